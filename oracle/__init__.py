@@ -1,0 +1,177 @@
+"""CPU oracle for the DropCompute threshold sweep.  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may use
+this package.  It compiles ``dc_oracle.c`` with gcc on first use (for the CPU
+it is running on) and exposes the C functions on numpy arrays.  It imports
+nothing from the CUDA package and the CUDA package imports nothing from here.
+
+Paper passages each function follows are cited in ``dc_oracle.c``.
+"""
+from __future__ import annotations
+
+import ctypes
+import hashlib
+import os
+import platform
+import subprocess
+from typing import NamedTuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dc_oracle.c")
+NSTATS = 5
+STAT_NAMES = ("mean_step", "done_frac", "thr", "thr_mean", "s_eff")
+_lib = None
+
+
+def _host_tag() -> str:
+    """A short tag for this host's CPU so a library built with -march=native
+    on one machine is never loaded on another."""
+    flags = ""
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags"):
+                    flags = line
+                    break
+    except OSError:
+        pass
+    with open(_SRC, "rb") as f:
+        src = f.read()
+    h = hashlib.sha1(flags.encode() + platform.machine().encode() + src).hexdigest()[:12]
+    return h
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, f"libdc_oracle.{_host_tag()}.so")
+
+
+def build(force: bool = False, source: str | None = None, out: str | None = None) -> str:
+    """Compile the oracle.  ``source``/``out`` let a test compile a deliberately
+    altered copy (mutation checks) without touching the real one."""
+    src = source or _SRC
+    dst = out or lib_path()
+    if not force and os.path.exists(dst) and os.path.getmtime(dst) >= os.path.getmtime(src):
+        return dst
+    tmp = dst + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O3", "-march=native", "-std=c11", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
+           "-shared", "-fPIC", "-o", tmp, src, "-lm"]
+    subprocess.run(cmd, check=True, capture_output=True)
+    os.replace(tmp, dst)
+    return dst
+
+
+def _bind(lib):
+    i64, i32, f32 = ctypes.c_int64, ctypes.c_int, ctypes.c_float
+    p = ctypes.c_void_p
+    for name in ("dco_sweep_literal", "dco_sweep_rows"):
+        fn = getattr(lib, name)
+        fn.argtypes = [p, i64, i64, i64, p, i64, f32, i32, p, p, p]
+        fn.restype = i32
+    lib.dco_reduce_trials.argtypes = [p, p, p, i64, i64, i64, i64, p, p]
+    lib.dco_reduce_trials.restype = i32
+    lib.dco_argmax.argtypes = [p, i64]
+    lib.dco_argmax.restype = i64
+    lib.dco_algorithm2.argtypes = [p, i64, i64, i64, p, i64, f32, p, p]
+    lib.dco_algorithm2.restype = i32
+    return lib
+
+
+def load(path: str | None = None):
+    global _lib
+    if path is not None:
+        return _bind(ctypes.CDLL(path))
+    if _lib is None:
+        _lib = _bind(ctypes.CDLL(build()))
+    return _lib
+
+
+def num_threads() -> int:
+    """Threads the row-order sweep uses (OpenMP's default: OMP_NUM_THREADS or all cores)."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        try:
+            return max(1, int(env.split(",")[0]))
+        except ValueError:
+            pass
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+class Sweep(NamedTuple):
+    step: np.ndarray  # [T,K] float32
+    done: np.ndarray  # [T,K] int32
+    sync: np.ndarray  # [T]   float32
+
+
+class Stats(NamedTuple):
+    stats: np.ndarray     # [NSTATS,K] float64, rows in STAT_NAMES order
+    baseline: np.ndarray  # [2] float64: mean_sync, thr_sync
+
+
+def _f32c(a, ndim):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    assert a.ndim == ndim
+    return a
+
+
+def sweep(lat, taus, t_comm: float, rule: int = 0, order: str = "rows", lib=None) -> Sweep:
+    """Per-(iteration, tau) step time and completed count.
+
+    ``order='literal'`` runs Algorithm 2's loop nest as printed (tau outermost);
+    ``order='rows'`` reads every sample once (same predicate, same integers)."""
+    lib = lib or load()
+    lat = _f32c(lat, 3)
+    taus = _f32c(taus, 1)
+    T, N, M = lat.shape
+    K = taus.shape[0]
+    step = np.empty((T, K), np.float32)
+    done = np.empty((T, K), np.int32)
+    sync = np.empty((T,), np.float32)
+    fn = {"literal": lib.dco_sweep_literal, "rows": lib.dco_sweep_rows}[order]
+    rc = fn(lat.ctypes.data, T, N, M, taus.ctypes.data, K, np.float32(t_comm), rule,
+            step.ctypes.data, done.ctypes.data, sync.ctypes.data)
+    if rc != 0:
+        raise ValueError(f"oracle sweep failed with status {rc}")
+    return Sweep(step, done, sync)
+
+
+def reduce_trials(step, done, sync, N: int, M: int, lib=None) -> Stats:
+    lib = lib or load()
+    step = _f32c(step, 2)
+    done = np.ascontiguousarray(done, dtype=np.int32)
+    sync = _f32c(sync, 1)
+    T, K = step.shape
+    assert done.shape == (T, K) and sync.shape == (T,)
+    stats = np.empty((NSTATS, K), np.float64)
+    base = np.empty((2,), np.float64)
+    rc = lib.dco_reduce_trials(step.ctypes.data, done.ctypes.data, sync.ctypes.data, T, K, N, M,
+                               stats.ctypes.data, base.ctypes.data)
+    if rc != 0:
+        raise ValueError(f"oracle reduce failed with status {rc}")
+    return Stats(stats, base)
+
+
+def argmax(objective, lib=None) -> int:
+    lib = lib or load()
+    obj = np.ascontiguousarray(objective, dtype=np.float64)
+    return int(lib.dco_argmax(obj.ctypes.data, obj.shape[0]))
+
+
+def algorithm2(lat, taus, t_comm: float, lib=None):
+    """Algorithm 2 start to finish as printed (floating-point 1/N accumulation)."""
+    lib = lib or load()
+    lat = _f32c(lat, 3)
+    taus = _f32c(taus, 1)
+    T, N, M = lat.shape
+    K = taus.shape[0]
+    s_eff = np.empty((K,), np.float64)
+    k_star = ctypes.c_int64(-1)
+    rc = lib.dco_algorithm2(lat.ctypes.data, T, N, M, taus.ctypes.data, K, np.float32(t_comm),
+                            s_eff.ctypes.data, ctypes.byref(k_star))
+    if rc != 0:
+        raise ValueError(f"oracle algorithm2 failed with status {rc}")
+    return s_eff, int(k_star.value)

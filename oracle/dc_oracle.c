@@ -1,0 +1,249 @@
+/*
+ * CPU oracle for the DropCompute threshold sweep.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain statement of what the simulator computes.  It
+ * exists so that tests, the smoke check and the benchmark's CPU-baseline leg
+ * can compare the CUDA library against it.  Nothing in the product path may
+ * include, link or call it, and it shares no code with the CUDA sources.
+ *
+ * What is stated here (paper: DropCompute, arXiv 2306.10598):
+ *   - Algorithm 2 ("Automatic choice for the optimal threshold tau"), App. C.1:
+ *     the loop nest, the running sum T_{i,n} += t_{i,n}^{(m)}, the strict test
+ *     T_{i,n} < tau, T_i = max_n T_{i,n}, S_i(tau), S_eff(tau), tau*.
+ *   - Sec. 4.3: completed micro-batches M~ (inclusive running sum < tau) and
+ *     the DropCompute step time min{tau, T} + T^c.
+ *   - Sec. 4.4, Eq. 6: effective speedup and throughput N*M~ / (min{tau,T}+T^c).
+ *
+ * Readings taken where the paper is silent (each is listed in the design notes):
+ *   - samples, running sums, comparisons and step times are IEEE binary32;
+ *     one rounding per addition, micro-batches strictly in the order m=1..M;
+ *   - M~ is kept as the integer number of completed micro-batches summed over
+ *     workers (Algorithm 2 adds 1/N per hit; the integer count divided once at
+ *     the end is the same number in exact arithmetic);
+ *   - T^c is one scalar for all iterations;
+ *   - statistics over iterations are binary64;
+ *   - argmax takes the first maximum and never selects a NaN.
+ *
+ * rule 0 is the paper's (a micro-batch counts iff it FINISHES before tau).
+ * rule 1 is the variant described in the paper's Limitations paragraph, where
+ * the timeout is only looked at between accumulations: a micro-batch is run
+ * iff it STARTS before tau, and a worker's time is the finish time of the
+ * last micro-batch it ran.
+ *
+ * Pins (tests/test_oracle_pins.py and friends): harmonic-number mean of the
+ * max of exponentials, quadrature of Eq. 3 for normals, Eq. 5 (exact for
+ * normal micro-batches), Erlang CDF for shifted exponentials, exhaustive
+ * enumeration of tiny dyadic laws in rational arithmetic, a hand-worked
+ * example, M=1 against sort/searchsorted, invariants, and mutation checks.
+ * Parity unpinned: none of the paper's printed E[T]/E[T_i] table values pins
+ * this code firmly (the worker count behind them is not printed); they are
+ * used as a loose plausibility band only.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define DCO_NSTATS 5 /* mean_step, done_frac, thr, thr_mean, s_eff */
+
+/* ---------------------------------------------------------------------------
+ * Algorithm 2 in the paper's own loop order: tau outermost, then iteration i,
+ * worker n, micro-batch m.  Writes the per-(iteration, tau) quantities.
+ *   lat      [T,N,M] binary32, m fastest
+ *   taus     [K]
+ *   out_step [T,K]  min(tau, T_i) + T^c            (rule 0)
+ *   out_done [T,K]  N * M~_i(tau) as an integer
+ *   out_sync [T]    T_i + T^c   (the tau = infinity step time)
+ * ------------------------------------------------------------------------- */
+int dco_sweep_literal(const float *lat, int64_t T, int64_t N, int64_t M,
+                      const float *taus, int64_t K, float t_comm, int rule,
+                      float *out_step, int32_t *out_done, float *out_sync)
+{
+    if (!lat || !taus || !out_step || !out_done || !out_sync) return 1;
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return 2;
+    if (rule != 0 && rule != 1) return 7;
+    for (int64_t k = 0; k < K; ++k) {
+        const float tau = taus[k];
+        for (int64_t i = 0; i < T; ++i) {
+            int64_t done = 0;      /* N * M~_i(tau) */
+            float Ti = 0.0f;       /* slowest worker's full compute time */
+            float Wi = 0.0f;       /* slowest worker's time under the threshold (rule 1) */
+            for (int64_t n = 0; n < N; ++n) {
+                const float *t = lat + (i * N + n) * M;
+                float Tin = 0.0f;  /* running compute time of worker n */
+                float Win = 0.0f;  /* finish time of the last micro-batch it ran (rule 1) */
+                for (int64_t m = 0; m < M; ++m) {
+                    if (rule == 0) {
+                        Tin = Tin + t[m];
+                        if (Tin < tau) done += 1;
+                    } else {
+                        /* started iff the time elapsed BEFORE it is < tau */
+                        if (Tin < tau) {
+                            done += 1;
+                            Win = Tin + t[m];
+                        }
+                        Tin = Tin + t[m];
+                    }
+                }
+                Ti = fmaxf(Ti, Tin);
+                Wi = fmaxf(Wi, Win);
+            }
+            if (rule == 0)
+                out_step[i * K + k] = fminf(tau, Ti) + t_comm;
+            else
+                out_step[i * K + k] = Wi + t_comm;
+            out_done[i * K + k] = (int32_t)done;
+            out_sync[i] = Ti + t_comm;
+        }
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------
+ * The same quantities with the loops in the order iteration, worker,
+ * micro-batch, tau.  The predicate evaluated for every (i,n,m,k) is the same
+ * and the counts are integers, so no output bit can differ from the literal
+ * order; this form reads the samples once and is the one used on large inputs.
+ * Iterations are independent and are spread over OpenMP threads.
+ * ------------------------------------------------------------------------- */
+int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
+                   const float *taus, int64_t K, float t_comm, int rule,
+                   float *out_step, int32_t *out_done, float *out_sync)
+{
+    if (!lat || !taus || !out_step || !out_done || !out_sync) return 1;
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return 2;
+    if (rule != 0 && rule != 1) return 7;
+    int failed = 0;
+#pragma omp parallel
+    {
+        int64_t *cnt = (int64_t *)malloc((size_t)K * sizeof(int64_t));
+        float *wmax = (float *)malloc((size_t)K * sizeof(float));
+        if (!cnt || !wmax) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t i = 0; i < T; ++i) {
+            if (!cnt || !wmax) continue;
+            float Ti = 0.0f;
+            for (int64_t k = 0; k < K; ++k) { cnt[k] = 0; wmax[k] = 0.0f; }
+            for (int64_t n = 0; n < N; ++n) {
+                const float *t = lat + (i * N + n) * M;
+                float Tin = 0.0f;
+                for (int64_t m = 0; m < M; ++m) {
+                    if (rule == 0) {
+                        Tin = Tin + t[m];
+                        for (int64_t k = 0; k < K; ++k) cnt[k] += (Tin < taus[k]) ? 1 : 0;
+                    } else {
+                        const float before = Tin;
+                        Tin = Tin + t[m];
+                        for (int64_t k = 0; k < K; ++k) {
+                            if (before < taus[k]) {
+                                cnt[k] += 1;
+                                wmax[k] = fmaxf(wmax[k], Tin);
+                            }
+                        }
+                    }
+                }
+                Ti = fmaxf(Ti, Tin);
+            }
+            out_sync[i] = Ti + t_comm;
+            for (int64_t k = 0; k < K; ++k) {
+                out_step[i * K + k] = (rule == 0) ? (fminf(taus[k], Ti) + t_comm) : (wmax[k] + t_comm);
+                out_done[i * K + k] = (int32_t)cnt[k];
+            }
+        }
+        free(cnt);
+        free(wmax);
+    }
+    return failed ? 6 : 0;
+}
+
+/* ---------------------------------------------------------------------------
+ * Reduction over iterations, binary64 (Algorithm 2: S_i(tau) and its mean;
+ * Eq. 6; Sec. 4.4 throughput).  For every tau_k:
+ *   stats[0][k] mean_step  = (1/T) sum_i step[i,k]
+ *   stats[1][k] done_frac  = sum_i done[i,k] / (T*N*M)
+ *   stats[2][k] thr        = sum_i done[i,k] / sum_i step[i,k]      micro-batches per second
+ *   stats[3][k] thr_mean   = (1/T) sum_i done[i,k]/step[i,k]
+ *   stats[4][k] s_eff      = (1/T) sum_i (sync[i]/step[i,k]) * done[i,k]/(N*M)
+ * baseline[0] mean_sync = (1/T) sum_i sync[i];  baseline[1] thr_sync = T*N*M / sum_i sync[i].
+ * ------------------------------------------------------------------------- */
+int dco_reduce_trials(const float *step, const int32_t *done, const float *sync,
+                      int64_t T, int64_t K, int64_t N, int64_t M,
+                      double *stats, double *baseline)
+{
+    if (!step || !done || !sync || !stats || !baseline) return 1;
+    if (T <= 0 || K <= 0 || N <= 0 || M <= 0) return 2;
+    const double NM = (double)N * (double)M;
+    for (int64_t k = 0; k < K; ++k) {
+        double sum_step = 0.0, sum_ratio = 0.0, sum_S = 0.0;
+        int64_t sum_done = 0;
+        for (int64_t i = 0; i < T; ++i) {
+            const double st = (double)step[i * K + k];
+            const double dn = (double)done[i * K + k];
+            sum_step += st;
+            sum_done += done[i * K + k];
+            sum_ratio += dn / st;
+            sum_S += ((double)sync[i] / st) * (dn / NM);
+        }
+        stats[0 * K + k] = sum_step / (double)T;
+        stats[1 * K + k] = (double)sum_done / ((double)T * NM);
+        stats[2 * K + k] = (double)sum_done / sum_step;
+        stats[3 * K + k] = sum_ratio / (double)T;
+        stats[4 * K + k] = sum_S / (double)T;
+    }
+    double sum_sync = 0.0;
+    for (int64_t i = 0; i < T; ++i) sum_sync += (double)sync[i];
+    baseline[0] = sum_sync / (double)T;
+    baseline[1] = ((double)T * NM) / sum_sync;
+    return 0;
+}
+
+/* tau* = argmax_tau objective(tau): first index attaining the maximum; a NaN
+ * never wins; returns -1 if every entry is NaN. */
+int64_t dco_argmax(const double *objective, int64_t K)
+{
+    int64_t best = -1;
+    for (int64_t k = 0; k < K; ++k) {
+        const double v = objective[k];
+        if (v != v) continue;
+        if (best < 0 || v > objective[best]) best = k;
+    }
+    return best;
+}
+
+/* ---------------------------------------------------------------------------
+ * Algorithm 2 start to finish, exactly as printed, including the 1/N
+ * accumulation of M~ in floating point (binary64 here) — used only to check
+ * that the integer-count reading above gives the same S_eff and tau*.
+ * ------------------------------------------------------------------------- */
+int dco_algorithm2(const float *lat, int64_t T, int64_t N, int64_t M,
+                   const float *taus, int64_t K, float t_comm,
+                   double *s_eff, int64_t *k_star)
+{
+    if (!lat || !taus || !s_eff || !k_star) return 1;
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return 2;
+    for (int64_t k = 0; k < K; ++k) {
+        const float tau = taus[k];
+        double acc = 0.0;
+        for (int64_t i = 0; i < T; ++i) {
+            double Mt = 0.0;
+            float Ti = 0.0f;
+            for (int64_t n = 0; n < N; ++n) {
+                float Tin = 0.0f;
+                for (int64_t m = 0; m < M; ++m) {
+                    Tin = Tin + lat[(i * N + n) * M + m];
+                    Mt = Mt + (1.0 / (double)N) * ((Tin < tau) ? 1.0 : 0.0);
+                }
+                Ti = fmaxf(Ti, Tin);
+            }
+            const float num = Ti + t_comm;
+            const float den = fminf(tau, Ti) + t_comm;
+            acc += ((double)num / (double)den) * (Mt / (double)M);
+        }
+        s_eff[k] = acc / (double)T;
+    }
+    *k_star = dco_argmax(s_eff, K);
+    return 0;
+}

@@ -1,0 +1,196 @@
+"""Seeded synthetic latency tensors and threshold grids.
+
+This module only draws random inputs: it contains none of the simulator's
+arithmetic and is the one module both the CUDA path's tests/benchmark and the
+CPU oracle's tests read their inputs from.
+
+The paper's measured micro-batch latency traces are not available, so each
+workload is a synthetic tensor ``latencies[T, N, M]`` (trials x workers x
+gradient accumulations, fp32 seconds) shaped like the paper's runs: about 200
+measured workers and an extrapolation to 2048 (Fig. 1), 12 to 64 accumulations
+(Sec. 5.2, Fig. 4, Fig. 6), additive straggler noise (App. B.1), plus a tiny
+case and a bandwidth-stress case.
+
+Draw order.  A tensor is filled in chunks of whole trials.  Chunk ``c`` uses
+its own ``torch.Generator`` seeded with ``seed * 1_000_003 + c`` on the target
+device, and inside a chunk the draws are made in the order written in the
+``_fill_*`` function of the law.  Any range of trials can therefore be
+regenerated on the same kind of device without generating the rest.  CPU and
+CUDA generators give different bits, so a comparison always copies one tensor
+to both sides and never regenerates it.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+from typing import Callable, Dict, Optional
+
+import numpy as np
+import torch
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    T: int
+    N: int
+    M: int
+    K: int
+    tau_lo: float       # grid start, in units of `tau_unit`
+    tau_hi: float       # grid end (inclusive), in units of `tau_unit`
+    tau_unit: float     # seconds: 1.0 for an absolute grid, else the analytic mean worker time
+    t_comm: float
+    law: str
+    seed: int = 0
+
+    @property
+    def samples(self) -> int:
+        return self.T * self.N * self.M
+
+    @property
+    def latency_bytes(self) -> int:
+        return 4 * self.samples
+
+    def with_trials(self, T: int) -> "Workload":
+        return Workload(self.name, T, self.N, self.M, self.K, self.tau_lo, self.tau_hi, self.tau_unit,
+                        self.t_comm, self.law, self.seed)
+
+
+# Analytic mean of one worker's total compute time under each law (so that the
+# grid does not depend on the draw).
+_MEAN_PAPER = 32 * 0.025 + 0.05                                           # 0.85 s
+_MEAN_EXTRA = 16 * (0.03 * math.exp(0.1 ** 2 / 2) + 0.005 * 0.3)          # 0.506406 s
+_MEAN_CORR = 64 * math.exp(0.05 ** 2 / 2) * 0.01 * math.exp(0.15 ** 2 / 2)  # 0.648050 s
+_MEAN_STRESS = 128 * (0.005 + 2 * 0.001)                                  # 0.896 s
+
+WORKLOADS: Dict[str, Workload] = {
+    w.name: w
+    for w in (
+        Workload("tiny", 1024, 8, 4, 16, 0.2, 0.6, 1.0, 0.05, "shifted_exp"),
+        Workload("paper_scale", 16384, 200, 32, 64, 0.5, 1.5, _MEAN_PAPER, 0.1, "normal_head_exp"),
+        Workload("extrapolation", 4096, 2048, 16, 128, 0.8, 2.0, _MEAN_EXTRA, 0.2, "lognormal_straggler"),
+        Workload("correlated", 8192, 4096, 64, 256, 0.7, 1.5, _MEAN_CORR, 0.15, "correlated_lognormal"),
+        Workload("bandwidth_stress", 32768, 2048, 128, 256, 0.6, 1.4, _MEAN_STRESS, 0.1, "shifted_gamma2"),
+    )
+}
+
+
+def make_taus(w: Workload) -> np.ndarray:
+    """K evenly spaced thresholds including both ends, computed in fp64 and rounded once to fp32."""
+    grid = np.linspace(w.tau_lo * w.tau_unit, w.tau_hi * w.tau_unit, w.K, dtype=np.float64)
+    return grid.astype(np.float32)
+
+
+# --- the laws -------------------------------------------------------------
+# Every function fills out[t0:t1] (a [n_trials, N, M] fp32 view) using generator g.
+
+def _fill_shifted_exp(out: torch.Tensor, g: torch.Generator) -> None:
+    # 0.1 s + Exponential(mean 0.02 s), iid
+    out.exponential_(1.0 / 0.02, generator=g)
+    out.add_(0.1)
+
+
+def _fill_normal_head_exp(out: torch.Tensor, g: torch.Generator) -> None:
+    # Normal(0.025, sd 0.002) clipped at 0, iid; then Exponential(mean 0.05) per (trial, worker) added to m = 0
+    out.normal_(0.025, 0.002, generator=g)
+    out.clamp_(min=0.0)
+    head = torch.empty(out.shape[:2], dtype=out.dtype, device=out.device)
+    head.exponential_(1.0 / 0.05, generator=g)
+    out[:, :, 0].add_(head)
+
+
+def _fill_lognormal_straggler(out: torch.Tensor, g: torch.Generator) -> None:
+    # 0.03 s x LogNormal(0, 0.1), iid; with probability 0.005 a sample gets Uniform(0.1, 0.5) s added
+    out.log_normal_(0.0, 0.1, generator=g)
+    out.mul_(0.03)
+    u = torch.empty_like(out).uniform_(0.0, 1.0, generator=g)
+    extra = torch.empty_like(out).uniform_(0.1, 0.5, generator=g)
+    out.add_(torch.where(u < 0.005, extra, torch.zeros_like(extra)))
+
+
+def _fill_correlated_lognormal(out: torch.Tensor, g: torch.Generator) -> None:
+    # LogNormal(ln 0.01, 0.15) per sample x LogNormal(0, 0.05) per (trial, worker)
+    out.log_normal_(math.log(0.01), 0.15, generator=g)
+    slow = torch.empty(out.shape[:2], dtype=out.dtype, device=out.device)
+    slow.log_normal_(0.0, 0.05, generator=g)
+    out.mul_(slow.unsqueeze(-1))
+
+
+def _fill_shifted_gamma2(out: torch.Tensor, g: torch.Generator) -> None:
+    # 0.005 s + Gamma(shape 2, scale 0.001 s) = 0.005 + 0.001 (E1 + E2), E ~ Exponential(1), iid
+    out.exponential_(1.0, generator=g)
+    e2 = torch.empty_like(out).exponential_(1.0, generator=g)
+    out.add_(e2)
+    out.mul_(0.001)
+    out.add_(0.005)
+
+
+_LAWS: Dict[str, Callable[[torch.Tensor, torch.Generator], None]] = {
+    "shifted_exp": _fill_shifted_exp,
+    "normal_head_exp": _fill_normal_head_exp,
+    "lognormal_straggler": _fill_lognormal_straggler,
+    "correlated_lognormal": _fill_correlated_lognormal,
+    "shifted_gamma2": _fill_shifted_gamma2,
+}
+
+_CHUNK_FLOATS = 1 << 26  # 256 MB of fp32 per chunk of whole trials
+
+
+def chunk_trials(w: Workload) -> int:
+    return max(1, _CHUNK_FLOATS // (w.N * w.M))
+
+
+def fill_latencies(w: Workload, device, out: Optional[torch.Tensor] = None,
+                   t0: int = 0, t1: Optional[int] = None) -> torch.Tensor:
+    """Trials ``t0:t1`` of workload ``w`` on ``device``: a contiguous fp32 ``[t1-t0, N, M]`` tensor.
+
+    The result does not depend on which range is asked for: trial t always
+    comes from chunk ``t // chunk_trials(w)`` of the seeded sequence."""
+    t1 = w.T if t1 is None else t1
+    assert 0 <= t0 <= t1 <= w.T
+    device = torch.device(device)
+    if out is None:
+        out = torch.empty((t1 - t0, w.N, w.M), dtype=torch.float32, device=device)
+    assert out.shape == (t1 - t0, w.N, w.M) and out.dtype == torch.float32 and out.is_contiguous()
+    ct = chunk_trials(w)
+    law = _LAWS[w.law]
+    c = t0 // ct
+    while c * ct < t1:
+        lo, hi = c * ct, min((c + 1) * ct, w.T)
+        g = torch.Generator(device=device)
+        g.manual_seed(w.seed * 1_000_003 + c)
+        a, b = max(lo, t0), min(hi, t1)
+        if a == lo and b == hi:
+            law(out[a - t0:b - t0], g)
+        else:  # partial chunk: draw the whole chunk, keep the part asked for
+            tmp = torch.empty((hi - lo, w.N, w.M), dtype=torch.float32, device=device)
+            law(tmp, g)
+            out[a - t0:b - t0].copy_(tmp[a - lo:b - lo])
+            del tmp
+        c += 1
+    return out
+
+
+# --- small generic inputs for tests --------------------------------------
+
+def iid_latencies(law: str, T: int, N: int, M: int, seed: int, device="cpu", **p) -> torch.Tensor:
+    """Small iid tensors for closed-form checks: 'exp'(rate), 'normal'(mu, sd), 'shifted_exp'(shift, mean),
+    'uniform'(lo, hi), 'dyadic' (values k/64, k in 1..hi: sums are exact in fp32)."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    out = torch.empty((T, N, M), dtype=torch.float32, device=device)
+    if law == "exp":
+        out.exponential_(p["rate"], generator=g)
+    elif law == "normal":
+        out.normal_(p["mu"], p["sd"], generator=g)
+    elif law == "shifted_exp":
+        out.exponential_(1.0 / p["mean"], generator=g)
+        out.add_(p["shift"])
+    elif law == "uniform":
+        out.uniform_(p["lo"], p["hi"], generator=g)
+    elif law == "dyadic":
+        k = torch.randint(1, int(p["hi"]) + 1, (T, N, M), generator=g, device=device)
+        out.copy_(k.to(torch.float32) / 64.0)
+    else:
+        raise ValueError(law)
+    return out

@@ -1,0 +1,335 @@
+"""The battery of checks that pins the CPU oracle to things other than itself.
+
+Each ``pin_*`` takes a loaded oracle library (the real one, or a deliberately
+altered copy in the mutation test) and raises AssertionError when the library
+disagrees with what the paper and the mathematics fix.  Citations name the
+paper's sections/equations/algorithms.
+"""
+from __future__ import annotations
+
+import itertools
+import json
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import scipy.integrate
+import scipy.stats
+
+import oracle
+from paper_2306_10598_b200 import workloads as W
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+INF = np.float32(np.inf)
+
+
+def _np(t):
+    return t.numpy() if hasattr(t, "numpy") else np.asarray(t)
+
+
+def _stats(lib, lat, taus, t_comm, rule=0, order="rows"):
+    lat = _np(lat)
+    T, N, M = lat.shape
+    sw = oracle.sweep(lat, taus, t_comm, rule=rule, order=order, lib=lib)
+    st = oracle.reduce_trials(sw.step, sw.done, sw.sync, N, M, lib=lib)
+    return sw, st
+
+
+# --- closed forms ------------------------------------------------------------
+
+def pin_exp_max_harmonic(lib, order="rows"):
+    """Sec. 4.2 / Eq. 3 special case: the max of N iid Exp(rate) has mean H_N / rate.
+    M = 1, tau = infinity, T^c = 0."""
+    for N, rate, T, seed in ((8, 2.0, 40000, 1), (200, 5.0, 20000, 2)):
+        lat = W.iid_latencies("exp", T, N, 1, seed, rate=rate)
+        sw, st = _stats(lib, lat, np.array([INF]), 0.0, order=order)
+        H = sum(1.0 / i for i in range(1, N + 1))
+        sd = math.sqrt(sum(1.0 / (i * rate) ** 2 for i in range(1, N + 1)))
+        assert abs(st.baseline[0] - H / rate) <= 5 * sd / math.sqrt(T), (N, st.baseline[0], H / rate)
+        # tau = infinity: everything completed, step is the plain synchronous max
+        assert (sw.done == N).all() and (sw.step[:, 0] == sw.sync).all()
+        assert abs(st.stats[0, 0] - st.baseline[0]) <= 1e-12 * st.baseline[0]
+        assert np.array_equal(sw.sync, _np(lat).max(axis=(1, 2)))
+
+
+def _emax_normal(N, mu, sd):
+    f = lambda x: x * N * scipy.stats.norm.pdf(x, mu, sd) * scipy.stats.norm.cdf(x, mu, sd) ** (N - 1)
+    v, _ = scipy.integrate.quad(f, mu - 12 * sd, mu + 12 * sd, epsabs=1e-13, epsrel=1e-12)
+    return v
+
+
+def pin_normal_max_quadrature(lib, order="rows"):
+    """Eq. 3: f_T = N f F^(N-1).  E[max of N normals] by quadrature; N = 2 is mu + sd/sqrt(pi).
+    With M micro-batches a worker's time is N(M mu, M sd^2) (sum of normals), so the same
+    integral pins running sum and max together."""
+    assert abs(_emax_normal(2, 1.0, 0.1) - (1.0 + 0.1 / math.sqrt(math.pi))) < 1e-10
+    mu, sd = 1.0, 0.1
+    for N, M, T, seed in ((2, 1, 60000, 3), (3, 1, 60000, 4), (5, 4, 40000, 5), (8, 9, 40000, 6)):
+        lat = W.iid_latencies("normal", T, N, M, seed, mu=mu, sd=sd)
+        sw, st = _stats(lib, lat, np.array([INF]), 0.25, order=order)
+        want = _emax_normal(N, M * mu, math.sqrt(M) * sd) + 0.25
+        tol = 5 * math.sqrt(M) * sd / math.sqrt(T) + 1e-6
+        assert abs(st.baseline[0] - want) <= tol, (N, M, st.baseline[0], want)
+
+
+def pin_done_frac_normal_eq5(lib, order="rows"):
+    """Eq. 5 is exact when micro-batch latencies are iid normal:
+    E[M~(tau)] = sum_m Phi((tau - m mu)/sqrt(m sd^2))."""
+    mu, sd, N, M, T = 1.0, 0.15, 6, 8, 20000
+    lat = W.iid_latencies("normal", T, N, M, 7, mu=mu, sd=sd)
+    taus = np.linspace(3.0, 9.0, 13).astype(np.float32)
+    sw, st = _stats(lib, lat, taus, 0.5, order=order)
+    per_trial = sw.done.astype(np.float64) / (N * M)
+    for k, tau in enumerate(taus.astype(np.float64)):
+        want = sum(scipy.stats.norm.cdf((tau - m * mu) / (sd * math.sqrt(m))) for m in range(1, M + 1)) / M
+        se = per_trial[:, k].std(ddof=1) / math.sqrt(T)
+        assert abs(st.stats[1, k] - want) <= 5 * se + 2e-6, (k, st.stats[1, k], want, se)
+
+
+def pin_done_frac_erlang(lib, order="rows"):
+    """E[M~(tau)] = sum_m P(T_n^(m) < tau) (App. C.2); for c + Exp(mean b) micro-batches
+    T_n^(m) - m c is Erlang(m, b)."""
+    c, b, N, M, T = 0.1, 0.02, 8, 4, 30000
+    lat = W.iid_latencies("shifted_exp", T, N, M, 8, shift=c, mean=b)
+    taus = np.linspace(0.2, 0.6, 16).astype(np.float32)
+    sw, st = _stats(lib, lat, taus, 0.05, order=order)
+    per_trial = sw.done.astype(np.float64) / (N * M)
+    for k, tau in enumerate(taus.astype(np.float64)):
+        want = sum(scipy.stats.gamma.cdf(tau - m * c, a=m, scale=b) for m in range(1, M + 1)) / M
+        se = per_trial[:, k].std(ddof=1) / math.sqrt(T)
+        assert abs(st.stats[1, k] - want) <= 5 * se + 2e-6, (k, st.stats[1, k], want, se)
+
+
+# --- exhaustive enumeration in rational arithmetic -----------------------------
+
+def _enumerate_exact(values, N, M, taus, t_comm, rule):
+    """All len(values)^(N*M) equally likely outcomes; returns exact per-outcome and mean quantities
+    written directly from Sec. 4.3 / Eq. 6 (not from Algorithm 2's loops)."""
+    outcomes = list(itertools.product(values, repeat=N * M))
+    done, step, sync = [], [], []
+    for o in outcomes:
+        rows = [o[n * M:(n + 1) * M] for n in range(N)]
+        finish = [list(itertools.accumulate(r)) for r in rows]           # T_n^(m)
+        Tmax = max(f[-1] for f in finish)
+        d_row, s_row = [], []
+        for tau in taus:
+            if rule == 0:
+                d = sum(1 for f in finish for x in f if x < tau)
+                s = min(tau, Tmax) + t_comm
+            else:
+                d, w = 0, Fraction(0)
+                for f in finish:
+                    start = [Fraction(0)] + f[:-1]
+                    ran = [x for b, x in zip(start, f) if b < tau]
+                    d += len(ran)
+                    if ran:
+                        w = max(w, ran[-1])
+                s = w + t_comm
+            d_row.append(d)
+            s_row.append(s)
+        done.append(d_row)
+        step.append(s_row)
+        sync.append(Tmax + t_comm)
+    return outcomes, done, step, sync
+
+
+def pin_enumeration(lib, order="rows"):
+    """Tiny dyadic law {1/4, 1/2}: feeding every outcome once as the trials makes trial means exact
+    expectations; thresholds include reachable sums (ties test '<' versus '<=')."""
+    vals = [Fraction(1, 4), Fraction(1, 2)]
+    t_comm = Fraction(1, 8)
+    for (N, M), rule in itertools.product(((2, 3), (3, 2), (1, 4), (2, 2)), (0, 1)):
+        taus = [Fraction(1, 8), Fraction(1, 4), Fraction(1, 2), Fraction(3, 4), Fraction(1), Fraction(5, 4),
+                Fraction(3, 2), Fraction(7, 4), Fraction(2), Fraction(4)]
+        outcomes, done, step, sync = _enumerate_exact(vals, N, M, taus, t_comm, rule)
+        T = len(outcomes)
+        lat = np.array([[float(x) for x in o] for o in outcomes], np.float32).reshape(T, N, M)
+        taus_f = np.array([float(t) for t in taus], np.float32)
+        sw, st = _stats(lib, lat, taus_f, float(t_comm), rule=rule, order=order)
+        assert np.array_equal(sw.done, np.array(done, np.int32)), (N, M, rule)
+        assert np.array_equal(sw.step, np.array([[float(x) for x in r] for r in step], np.float32)), (N, M, rule)
+        assert np.array_equal(sw.sync, np.array([float(x) for x in sync], np.float32))
+        NM = N * M
+        for k in range(len(taus)):
+            sd = sum(Fraction(d[k]) for d in done)
+            ss = sum(s[k] for s in step)
+            want = [ss / T, sd / (T * NM), sd / ss,
+                    sum(Fraction(d[k]) / s[k] for d, s in zip(done, step)) / T,
+                    sum((y / s[k]) * Fraction(d[k], NM) for d, s, y in zip(done, step, sync)) / T]
+            for r in range(5):
+                assert abs(st.stats[r, k] - float(want[r])) <= 1e-13 * max(1.0, abs(float(want[r]))), (N, M, rule, r, k)
+        assert abs(st.baseline[0] - float(sum(sync) / T)) <= 1e-13
+        assert abs(st.baseline[1] - float(Fraction(T * NM) / sum(sync))) <= 1e-12
+        if rule == 0:
+            exact_seff = [sum((y / s[k]) * Fraction(d[k], NM) for d, s, y in zip(done, step, sync)) / T
+                          for k in range(len(taus))]
+            k_first = max(range(len(taus)), key=lambda k: (exact_seff[k], -k))
+            assert oracle.argmax(st.stats[4], lib=lib) == k_first
+
+
+# --- hand-worked example and rounding order ------------------------------------
+
+def _fr(x):
+    return float(Fraction(x))
+
+
+def pin_hand_example(lib, order="rows"):
+    with open(os.path.join(GOLDEN, "alg2_hand_example.json")) as f:
+        g = json.load(f)
+    lat = np.array([[[_fr(x) for x in row] for row in it] for it in g["latencies"]], np.float32)
+    taus = np.array([_fr(x) for x in g["taus"]], np.float32)
+    tc = _fr(g["t_comm"])
+    for rule in (0, 1):
+        sw, st = _stats(lib, lat, taus, tc, rule=rule, order=order)
+        want = g[f"rule{rule}"]
+        assert np.array_equal(sw.done, np.array(want["done"], np.int32)), rule
+        assert np.array_equal(sw.step, np.array([[_fr(x) for x in r] for r in want["step"]], np.float32)), rule
+        assert np.array_equal(sw.sync, np.array([_fr(x) for x in g["sync"]], np.float32))
+        if rule == 0:
+            for r, name in enumerate(oracle.STAT_NAMES):
+                ref = np.array([_fr(x) for x in want[name]])
+                assert np.allclose(st.stats[r], ref, rtol=1e-14, atol=0), name
+            assert oracle.argmax(st.stats[4], lib=lib) == want["k_star"]
+            assert abs(st.baseline[0] - _fr(want["mean_sync"])) < 1e-15
+            assert abs(st.baseline[1] - _fr(want["thr_sync"])) < 1e-14
+            s_eff, k_star = oracle.algorithm2(lat, taus, tc, lib=lib)
+            assert np.allclose(s_eff, st.stats[4], rtol=1e-14) and k_star == want["k_star"]
+
+
+def pin_fp32_left_to_right(lib, order="rows"):
+    """The running sum is binary32 with one rounding per addition, taken m = 1..M in order
+    (Algorithm 2's inner loop; the precision is this build's reading)."""
+    e = 2.0 ** -24
+    nxt = np.float32(1.0 + 2.0 ** -23)
+    # 1 + 2^-24 ties to even = 1, three times over: the sum never leaves 1.0
+    lat = np.array([[[1.0, e, e, e]]], np.float32)
+    sw = oracle.sweep(lat, np.array([1.0, nxt, INF], np.float32), 0.0, order=order, lib=lib)
+    assert sw.done.tolist() == [[0, 4, 4]] and sw.sync[0] == np.float32(1.0)
+    # same addends, the large one last: 3*2^-24 is exact, then 1 + 1.5 ulp ties to even = 1 + 2^-22
+    lat = np.array([[[e, e, e, 1.0]]], np.float32)
+    sw = oracle.sweep(lat, np.array([1.0, nxt, INF], np.float32), 0.0, order=order, lib=lib)
+    assert sw.sync[0] == np.float32(1.0 + 2.0 ** -22) and sw.done.tolist() == [[3, 3, 4]]
+    # cumulative sum in binary32 from numpy on random data (advisory third opinion)
+    lat = _np(W.iid_latencies("uniform", 50, 7, 33, 9, lo=0.001, hi=0.3))
+    P = np.cumsum(lat, axis=-1, dtype=np.float32)
+    taus = np.sort(np.random.default_rng(0).uniform(0.0, 6.0, 40)).astype(np.float32)
+    sw = oracle.sweep(lat, taus, 0.125, order=order, lib=lib)
+    assert np.array_equal(sw.done, (P[..., None] < taus).sum(axis=(1, 2)).astype(np.int32))
+    assert np.array_equal(sw.sync, P[..., -1].max(axis=1) + np.float32(0.125))
+
+
+def pin_m1_sort(lib, order="rows"):
+    """M = 1: the completed count at tau is the rank of tau among the sorted worker times and
+    the synchronous time is their maximum (textbook routines on the same fp32 data)."""
+    lat = _np(W.iid_latencies("uniform", 300, 37, 1, 10, lo=0.0, hi=1.0))
+    taus = np.concatenate([np.linspace(-0.1, 1.1, 25), lat[0, :5, 0]]).astype(np.float32)
+    taus.sort()
+    sw = oracle.sweep(lat, taus, 0.5, order=order, lib=lib)
+    for t in range(lat.shape[0]):
+        s = np.sort(lat[t, :, 0])
+        assert np.array_equal(sw.done[t], np.searchsorted(s, taus, side="left").astype(np.int32))
+        assert sw.sync[t] == s[-1] + np.float32(0.5)
+        assert np.array_equal(sw.step[t], np.minimum(taus, s[-1]) + np.float32(0.5))
+
+
+# --- invariants ---------------------------------------------------------------------
+
+def pin_invariants(lib, order="rows"):
+    rng = np.random.default_rng(11)
+    for (T, N, M), law in (((40, 9, 12), "shifted_exp"), ((25, 33, 5), "dyadic"), ((10, 1, 1), "uniform")):
+        p = dict(shift=0.1, mean=0.05) if law == "shifted_exp" else dict(hi=40) if law == "dyadic" else dict(lo=0, hi=1)
+        lat = _np(W.iid_latencies(law, T, N, M, 12, **p))
+        tot = lat.sum(-1).max()
+        taus = np.sort(rng.uniform(-0.2, 1.3 * tot, 23)).astype(np.float32)
+        taus = np.concatenate([taus, [taus[5], INF]]).astype(np.float32)
+        taus.sort()
+        K = taus.shape[0]
+        tc = np.float32(0.3)
+        for rule in (0, 1):
+            sw = oracle.sweep(lat, taus, tc, rule=rule, order=order, lib=lib)
+            assert (np.diff(sw.done.astype(np.int64), axis=1) >= 0).all()
+            assert (np.diff(sw.step, axis=1) >= 0).all()
+            assert (sw.done >= 0).all() and (sw.done <= N * M).all()
+            P = np.cumsum(lat, axis=-1, dtype=np.float32)
+            tmax = P[..., -1].max(axis=1)
+            above = taus[None, :] > tmax[:, None]
+            assert (sw.done[above] == N * M).all()
+            assert (sw.step[above] == np.broadcast_to(sw.sync[:, None], (T, K))[above]).all()
+            assert (sw.step[:, -1] == sw.sync).all() and (sw.done[:, -1] == N * M).all()  # tau = inf
+            if rule == 0:
+                assert (sw.step <= (taus[None, :] + tc)).all()
+            else:
+                # step <= tau + the micro-batch that was running when tau passed
+                nonneg = taus >= 0
+                assert (sw.step[:, nonneg] <= (taus[None, nonneg] + lat.max() + tc) * (1 + 1e-6)).all()
+            assert (sw.step[:, taus >= 0] >= tc).all()
+            # per-worker decisions: each worker as its own one-worker trial
+            per = oracle.sweep(lat.reshape(T * N, 1, M), taus, tc, rule=rule, order=order, lib=lib)
+            assert np.array_equal(per.done.reshape(T, N, K).sum(1), sw.done)
+            assert (per.done <= M).all()
+            assert np.array_equal(per.step.reshape(T, N, K).max(1), sw.step)
+            if rule == 1:
+                base = oracle.sweep(lat.reshape(T * N, 1, M), taus, tc, rule=0, order=order, lib=lib)
+                want = np.where(taus[None, :] > 0, np.minimum(M, base.done + 1), 0)
+                assert np.array_equal(per.done, want.astype(np.int32))
+            # permuting workers changes nothing; permuting trials permutes rows
+            pw = rng.permutation(N)
+            pt = rng.permutation(T)
+            sw2 = oracle.sweep(lat[:, pw][pt], taus, tc, rule=rule, order=order, lib=lib)
+            assert np.array_equal(sw2.done, sw.done[pt]) and np.array_equal(sw2.step, sw.step[pt])
+            assert np.array_equal(sw2.sync, sw.sync[pt])
+            # dropping columns of the grid leaves the others unchanged
+            sub = oracle.sweep(lat, taus[3:-1], tc, rule=rule, order=order, lib=lib)
+            assert np.array_equal(sub.done, sw.done[:, 3:-1]) and np.array_equal(sub.step, sw.step[:, 3:-1])
+
+
+def pin_argmax(lib, order="rows"):
+    nan = float("nan")
+    assert oracle.argmax([1.0, 3.0, 3.0, 2.0], lib=lib) == 1
+    assert oracle.argmax([nan, 1.0, nan, 1.0], lib=lib) == 1
+    assert oracle.argmax([nan, nan], lib=lib) == -1
+    assert oracle.argmax([-1.0], lib=lib) == 0
+    assert oracle.argmax([0.5, nan, 0.7, 0.7], lib=lib) == 2
+
+
+def pin_literal_equals_rows(lib, order=None):
+    rng = np.random.default_rng(13)
+    for T, N, M, K in ((7, 5, 9, 11), (3, 1, 1, 1), (4, 17, 2, 30), (2, 3, 40, 6)):
+        lat = _np(W.iid_latencies("shifted_exp", T, N, M, 14, shift=0.05, mean=0.03))
+        taus = np.sort(rng.uniform(0, 1.2 * lat.sum(-1).max(), K)).astype(np.float32)
+        for rule in (0, 1):
+            a = oracle.sweep(lat, taus, 0.07, rule=rule, order="literal", lib=lib)
+            b = oracle.sweep(lat, taus, 0.07, rule=rule, order="rows", lib=lib)
+            assert np.array_equal(a.done, b.done) and np.array_equal(a.step, b.step) and np.array_equal(a.sync, b.sync)
+        s_eff, k_star = oracle.algorithm2(lat, taus, 0.07, lib=lib)
+        sw0 = oracle.sweep(lat, taus, 0.07, rule=0, order="rows", lib=lib)
+        st = oracle.reduce_trials(sw0.step, sw0.done, sw0.sync, N, M, lib=lib)
+        assert np.allclose(s_eff, st.stats[4], rtol=1e-12, atol=0)
+        assert k_star == oracle.argmax(st.stats[4], lib=lib)
+
+
+def pin_independence_and_bailey(lib, order="rows"):
+    """Loose plausibility: E[M~ T] is close to E[M~] E[T] for many workers (App. C.2), and the
+    Bailey approximation (Eq. 4) lands within a few percent of the simulated E[T] for normal totals."""
+    mu, sd, N, M, T = 0.025, 0.004, 400, 16, 400
+    lat = W.iid_latencies("normal", T, N, M, 15, mu=mu, sd=sd)
+    tau = np.array([M * mu * 1.02], np.float32)
+    sw, st = _stats(lib, lat, tau, 0.0, order=order)
+    mt = sw.done[:, 0] / N
+    tm = sw.sync.astype(np.float64)
+    assert abs((mt * tm).mean() - mt.mean() * tm.mean()) <= 0.01 * mt.mean() * tm.mean()
+    g = 0.5772156649015329
+    z = (1 - g) * scipy.stats.norm.ppf(1 - 1 / N) + g * scipy.stats.norm.ppf(1 - 1 / (math.e * N))
+    bailey = math.sqrt(M) * sd * z + M * mu
+    assert abs(st.baseline[0] - bailey) <= 0.03 * bailey
+
+
+ALL_PINS = (
+    pin_exp_max_harmonic, pin_normal_max_quadrature, pin_done_frac_normal_eq5, pin_done_frac_erlang,
+    pin_enumeration, pin_hand_example, pin_fp32_left_to_right, pin_m1_sort, pin_invariants, pin_argmax,
+    pin_literal_equals_rows, pin_independence_and_bailey,
+)
+# a quick subset that still kills every planted mistake (used by the mutation test)
+FAST_PINS = (pin_hand_example, pin_enumeration, pin_fp32_left_to_right, pin_m1_sort, pin_argmax, pin_invariants,
+             pin_exp_max_harmonic)

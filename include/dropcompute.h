@@ -1,0 +1,195 @@
+/*
+ * dropcompute.h — C ABI of the DropCompute threshold-sweep simulator for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates, on one GPU, the Monte-Carlo model behind the paper's automatic choice of
+ * the compute threshold tau (DropCompute, arXiv 2306.10598: Algorithm 2 in App. C.1, built from
+ * the completed-micro-batch count M~ and the step time min{tau,T}+T^c of Sec. 4.3 and the effective
+ * speedup of Eq. 6).
+ *
+ * Conventions
+ *   T  trials (the paper's iterations i = 1..I)        N  data-parallel workers n
+ *   M  micro-batches (gradient accumulations) m        K  candidate thresholds tau_k
+ *   t_comm  the serial latency T^c of one step (all-reduce etc.), one scalar for all trials
+ *   latencies[t][n][m] = t_{i,n}^{(m)}: seconds worker n spent on micro-batch m in trial t
+ *
+ * Every pointer argument says whether it is a DEVICE or a HOST pointer.  The library never
+ * allocates or frees device memory, keeps no per-call state, and never synchronises the device
+ * unless the function says so: work is enqueued on `stream` (a cudaStream_t passed as void*; NULL
+ * is the default stream) and the call returns.  Buffers belong to the caller and must stay valid
+ * until the enqueued work has run.  Outputs are overwritten, never accumulated into.
+ *
+ * Errors.  Every function returns a dc_status.  Anything the host can see (null pointers, sizes
+ * out of range, misalignment, unknown enum values, too small a workspace) returns an error code
+ * and enqueues nothing.  Properties of the DATA (latencies finite and >= 0, thresholds sorted and
+ * not NaN) cannot be seen without reading device memory; they are preconditions.  When they are
+ * violated every kernel still stays inside its buffers and terminates, but the numbers are
+ * unspecified.  dc_check_inputs() verifies them synchronously for callers who want that.
+ * The kernels never trap.  Their internal waits on asynchronous copies are bounded; should one
+ * ever expire, the kernel records it and carries on to completion, and dc_device_status()
+ * reports it.
+ */
+#ifndef DROPCOMPUTE_H_
+#define DROPCOMPUTE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DC_OK = 0,
+    DC_ERR_NULL = 1,        /* a required pointer is NULL */
+    DC_ERR_SHAPE = 2,       /* T, N, M or K is not positive */
+    DC_ERR_ALIGN = 3,       /* a pointer is not aligned as documented */
+    DC_ERR_RANGE = 4,       /* a size exceeds what the library supports (see DC_MAX_K, N*M <= INT32_MAX) */
+    DC_ERR_TAUS = 5,        /* dc_check_inputs: thresholds not non-decreasing, or NaN */
+    DC_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (launch, copy, tensor-map encode) */
+    DC_ERR_UNSUPPORTED = 7, /* unknown rule / objective */
+    DC_ERR_LATENCIES = 8,   /* dc_check_inputs: a latency is negative, NaN or infinite */
+    DC_ERR_WORKSPACE = 9,   /* workspace pointer NULL, misaligned or too small */
+    DC_ERR_DEVICE = 10      /* dc_device_status: a bounded wait inside a kernel expired */
+} dc_status;
+
+/* Largest number of thresholds one call accepts. */
+#define DC_MAX_K 4096
+
+/* Completion rule. */
+#define DC_RULE_FINISH_BEFORE_TAU 0 /* Algorithm 2 / Sec. 4.3: micro-batch m counts iff T_n^{(m)} < tau */
+#define DC_RULE_START_BEFORE_TAU 1  /* Limitations paragraph: the timeout is looked at between
+                                       accumulations, so m is run iff T_n^{(m-1)} < tau */
+
+/* Rows of the statistics matrix written by dc_reduce_trials and read by dc_argmax_tau. */
+#define DC_STAT_MEAN_STEP 0 /* E[step time](tau)                         = mean_t step[t,k]                 */
+#define DC_STAT_DONE_FRAC 1 /* completed fraction E[M~]/M                = sum_t done[t,k] / (T*N*M)        */
+#define DC_STAT_THR 2       /* throughput, micro-batches per second     = sum_t done[t,k] / sum_t step[t,k] */
+#define DC_STAT_THR_MEAN 3  /* mean per-trial throughput                 = mean_t done[t,k]/step[t,k]       */
+#define DC_STAT_S_EFF 4     /* Algorithm 2's S_eff(tau) = mean_t (sync[t]/step[t,k]) * done[t,k]/(N*M)      */
+#define DC_NSTATS 5
+
+/*
+ * dc_simulate — one pass of the threshold sweep (Algorithm 2's loops over i, n, m for all tau at
+ * once; Sec. 4.3).  For every trial t and threshold k:
+ *
+ *   P_{t,n,m}      = fl32(P_{t,n,m-1} + latencies[t][n][m]),  P_{t,n,-1} = +0     (strictly m = 0..M-1)
+ *   out_done[t][k] = #{ (n,m) : P_{t,n,m} < taus[k] }          (= N * M~_t(tau_k); strict '<', fp32)
+ *   out_step[t][k] = fl32( fminf(taus[k], max_n P_{t,n,M-1}) + t_comm )   (= min{tau,T} + T^c)
+ *
+ *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; 16-byte aligned; finite and >= 0
+ *   T, N, M    > 0, N*M <= INT32_MAX
+ *   taus       DEVICE, [K] fp32, non-decreasing, no NaN; +infinity is allowed (gives the
+ *              synchronous baseline); 4-byte aligned.  1 <= K <= DC_MAX_K
+ *   out_step   DEVICE, [T][K] fp32        out_done   DEVICE, [T][K] int32
+ *   stream     cudaStream_t
+ *
+ * The result does not depend on the launch configuration or on scheduling: counts are integers
+ * and the maximum is exact, so two calls on the same input give the same bits.
+ */
+int dc_simulate(const float *latencies, int64_t T, int64_t N, int64_t M,
+                const float *taus, int32_t K, float t_comm,
+                float *out_step, int32_t *out_done, void *stream);
+
+/*
+ * dc_simulate_ex — dc_simulate plus the tau = infinity baseline and the choice of completion rule.
+ *
+ *   out_sync   DEVICE, [T] fp32 or NULL:  out_sync[t] = fl32( max_n P_{t,n,M-1} + t_comm )
+ *              (the plain synchronous step time T + T^c of Sec. 4.2 / 4.4)
+ *   rule       DC_RULE_FINISH_BEFORE_TAU: as dc_simulate.
+ *              DC_RULE_START_BEFORE_TAU:  out_done[t][k] = #{(n,m): P_{t,n,m-1} < taus[k]} and
+ *              out_step[t][k] = fl32( max_n W_n + t_comm ), W_n = P_{t,n,s-1} with s the number of
+ *              micro-batches worker n ran (W_n = 0 if none).
+ */
+int dc_simulate_ex(const float *latencies, int64_t T, int64_t N, int64_t M,
+                   const float *taus, int32_t K, float t_comm,
+                   float *out_step, int32_t *out_done, float *out_sync,
+                   int32_t rule, void *stream);
+
+/*
+ * dc_reduce_trials — statistics over trials in fp64 (Algorithm 2: S_i(tau) and S_eff(tau); Eq. 6;
+ * Sec. 4.4 throughput).  Sums run over trials in a fixed order that depends only on (T, K), so the
+ * result is reproducible bit for bit.
+ *
+ *   out_step, out_done   DEVICE, as written by dc_simulate
+ *   out_sync             DEVICE [T] or NULL.  With NULL, row DC_STAT_S_EFF and both baseline
+ *                        entries are NaN.
+ *   stats      DEVICE, [DC_NSTATS][K] fp64, rows as DC_STAT_* above
+ *   baseline   DEVICE, [2] fp64: mean_t sync[t]  and  T*N*M / sum_t sync[t]  (micro-batches per second
+ *              without DropCompute)
+ *   workspace  DEVICE scratch of at least dc_reduce_workspace_bytes(T, K) bytes, 8-byte aligned.
+ *              Contents on entry are ignored; contents on return are unspecified.  Two calls that may
+ *              overlap on the device need different workspaces.
+ */
+size_t dc_reduce_workspace_bytes(int64_t T, int32_t K);
+int dc_reduce_trials(const float *out_step, const int32_t *out_done, const float *out_sync,
+                     int64_t T, int32_t K, int64_t N, int64_t M,
+                     double *stats, double *baseline,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * dc_argmax_tau — tau* = argmax_tau objective(tau) (last line of Algorithm 2).
+ *
+ *   stats      DEVICE, [DC_NSTATS][K] from dc_reduce_trials      taus  DEVICE [K]
+ *   objective  DC_STAT_S_EFF (Algorithm 2's own), DC_STAT_THR or DC_STAT_THR_MEAN
+ *   out_k      DEVICE int32: first index attaining the maximum; NaN entries never win; -1 if all are NaN
+ *   out_tau    DEVICE fp32: taus[out_k] (NaN if out_k = -1)       out_value  DEVICE fp64 (NaN if -1)
+ */
+int dc_argmax_tau(const double *stats, const float *taus, int32_t K, int32_t objective,
+                  int32_t *out_k, float *out_tau, double *out_value, void *stream);
+
+/*
+ * dc_sweep_host — the whole path for a caller whose samples live in HOST memory: copies the
+ * latencies to the device in chunks of whole trials (overlapped with the kernels), runs
+ * dc_simulate_ex, dc_reduce_trials and dc_argmax_tau, copies the results back and waits for them.
+ * SYNCHRONOUS: returns when the host outputs are written.
+ *
+ *   latencies_host  HOST [T][N][M] fp32 (page-locked memory makes the copies asynchronous and fast)
+ *   taus_host       HOST [K]
+ *   stats_host      HOST [DC_NSTATS][K] fp64      baseline_host  HOST [2] fp64
+ *   k_star_host     HOST int32                    tau_star_host  HOST fp32
+ *   workspace       DEVICE scratch, at least dc_sweep_host_workspace_bytes(T,N,M,K, chunk_trials)
+ *                   bytes, 1024-byte aligned.  chunk_trials >= 1 is how many trials travel per copy;
+ *                   two chunks are resident at a time.
+ *   rule, objective as above
+ */
+size_t dc_sweep_host_workspace_bytes(int64_t T, int64_t N, int64_t M, int32_t K, int64_t chunk_trials);
+int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M,
+                  const float *taus_host, int32_t K, float t_comm, int32_t rule, int32_t objective,
+                  int64_t chunk_trials,
+                  double *stats_host, double *baseline_host, int32_t *k_star_host, float *tau_star_host,
+                  void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * dc_check_inputs — SYNCHRONOUS check of the data preconditions of dc_simulate on `stream`:
+ * returns DC_ERR_LATENCIES if any latency is negative, NaN or infinite, DC_ERR_TAUS if the grid is
+ * not non-decreasing or holds a NaN, DC_OK otherwise.  report_host (HOST, [2] int64, may be NULL)
+ * receives the number of bad latencies and of bad thresholds.
+ *   counters  DEVICE scratch, [2] int64 (16 bytes, 8-byte aligned)
+ */
+int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M,
+                    const float *taus, int32_t K,
+                    int64_t *counters, int64_t *report_host, void *stream);
+
+/*
+ * dc_device_status — SYNCHRONOUS.  Reads and clears the current device's record of expired waits.
+ * Returns DC_OK if none expired since the last call, DC_ERR_DEVICE otherwise; *flags_host (HOST,
+ * may be NULL) receives the raw bit mask (bit 0: a load never arrived, bit 1: a buffer was never
+ * released).
+ */
+int dc_device_status(uint32_t *flags_host);
+
+/* Which kernel dc_simulate_ex would use for a shape: 0 = tiled bulk-copy kernel, 1 = plain-load
+ * kernel (M not a multiple of 4, or a pointer only 4-byte aligned), negative = -dc_status. */
+int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K);
+
+/* Number of kernel launches the last successful call of each entry point enqueues (for accounting). */
+int dc_simulate_launches(void);
+int dc_reduce_trials_launches(void);
+int dc_argmax_tau_launches(void);
+
+const char *dc_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DROPCOMPUTE_H_ */

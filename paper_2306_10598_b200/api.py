@@ -1,0 +1,238 @@
+"""Thin Python binding of the C ABI in ``include/dropcompute.h``.
+
+Argument marshalling only: every function checks dtype/device/contiguity of the torch tensors it is
+given, passes their device pointers and the current CUDA stream to the library entry point of the
+same name, and raises :class:`DropComputeError` on a non-zero status.  There is no fallback: if
+``libdropcompute.so`` is not built this module fails to import.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import NamedTuple, Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdropcompute.so")
+
+DC_MAX_K = 4096
+RULE_FINISH_BEFORE_TAU = 0
+RULE_START_BEFORE_TAU = 1
+STAT_MEAN_STEP, STAT_DONE_FRAC, STAT_THR, STAT_THR_MEAN, STAT_S_EFF = range(5)
+NSTATS = 5
+STAT_NAMES = ("mean_step", "done_frac", "thr", "thr_mean", "s_eff")
+
+EXPORTS = (
+    "dc_simulate", "dc_simulate_ex", "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_argmax_tau",
+    "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan",
+    "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string",
+)
+
+
+class DropComputeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2306_10598_b200.build` "
+        "(there is no CPU or PyTorch fallback for this library)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+_p, _i64, _i32, _f32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_size_t
+_lib.dc_simulate.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _p, _p, _p]
+_lib.dc_simulate_ex.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _p, _p, _p, _i32, _p]
+_lib.dc_reduce_workspace_bytes.argtypes = [_i64, _i32]
+_lib.dc_reduce_workspace_bytes.restype = _sz
+_lib.dc_reduce_trials.argtypes = [_p, _p, _p, _i64, _i32, _i64, _i64, _p, _p, _p, _sz, _p]
+_lib.dc_argmax_tau.argtypes = [_p, _p, _i32, _i32, _p, _p, _p, _p]
+_lib.dc_sweep_host_workspace_bytes.argtypes = [_i64, _i64, _i64, _i32, _i64]
+_lib.dc_sweep_host_workspace_bytes.restype = _sz
+_lib.dc_sweep_host.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _i32, _i32, _i64, _p, _p, _p, _p, _p, _sz, _p]
+_lib.dc_check_inputs.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _p, _p, _p]
+_lib.dc_device_status.argtypes = [_p]
+_lib.dc_simulate_plan.argtypes = [_p, _i64, _i64, _i64, _i32]
+_lib.dc_status_string.argtypes = [ctypes.c_int]
+_lib.dc_status_string.restype = ctypes.c_char_p
+for _name in ("dc_simulate", "dc_simulate_ex", "dc_reduce_trials", "dc_argmax_tau", "dc_sweep_host", "dc_check_inputs",
+              "dc_device_status", "dc_simulate_plan", "dc_simulate_launches", "dc_reduce_trials_launches",
+              "dc_argmax_tau_launches"):
+    getattr(_lib, _name).restype = ctypes.c_int
+
+
+def status_string(status: int) -> str:
+    return _lib.dc_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise DropComputeError(status, where)
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(t: torch.Tensor) -> int:
+    return torch.cuda.current_stream(t.device).cuda_stream
+
+
+def dc_simulate(latencies: torch.Tensor, taus: torch.Tensor, t_comm: float,
+                out_step: torch.Tensor, out_done: torch.Tensor) -> None:
+    """``dc_simulate`` of the C ABI on the current stream.  latencies [T,N,M] fp32, taus [K] fp32,
+    out_step [T,K] fp32, out_done [T,K] int32 (all CUDA, contiguous)."""
+    T, N, M = latencies.shape
+    K = taus.shape[0]
+    assert tuple(out_step.shape) == (T, K) and tuple(out_done.shape) == (T, K)
+    with torch.cuda.device(latencies.device):
+        _check(_lib.dc_simulate(_dev(latencies, torch.float32, "latencies"), T, N, M, _dev(taus, torch.float32, "taus"), K,
+                                float(t_comm), _dev(out_step, torch.float32, "out_step"),
+                                _dev(out_done, torch.int32, "out_done"), _stream(latencies)), "dc_simulate")
+
+
+def dc_simulate_ex(latencies: torch.Tensor, taus: torch.Tensor, t_comm: float, out_step: torch.Tensor,
+                   out_done: torch.Tensor, out_sync: Optional[torch.Tensor], rule: int = RULE_FINISH_BEFORE_TAU) -> None:
+    T, N, M = latencies.shape
+    K = taus.shape[0]
+    assert tuple(out_step.shape) == (T, K) and tuple(out_done.shape) == (T, K)
+    assert out_sync is None or tuple(out_sync.shape) == (T,)
+    with torch.cuda.device(latencies.device):
+        _check(_lib.dc_simulate_ex(_dev(latencies, torch.float32, "latencies"), T, N, M, _dev(taus, torch.float32, "taus"),
+                                   K, float(t_comm), _dev(out_step, torch.float32, "out_step"),
+                                   _dev(out_done, torch.int32, "out_done"),
+                                   None if out_sync is None else _dev(out_sync, torch.float32, "out_sync"),
+                                   int(rule), _stream(latencies)), "dc_simulate_ex")
+
+
+def dc_reduce_workspace_bytes(T: int, K: int) -> int:
+    return int(_lib.dc_reduce_workspace_bytes(T, K))
+
+
+def dc_reduce_trials(out_step: torch.Tensor, out_done: torch.Tensor, out_sync: Optional[torch.Tensor], N: int, M: int,
+                     stats: torch.Tensor, baseline: torch.Tensor, workspace: torch.Tensor) -> None:
+    """stats [NSTATS,K] fp64, baseline [2] fp64, workspace: any CUDA tensor of at least
+    dc_reduce_workspace_bytes(T,K) bytes."""
+    T, K = out_step.shape
+    assert tuple(stats.shape) == (NSTATS, K) and tuple(baseline.shape) == (2,)
+    if not workspace.is_cuda or not workspace.is_contiguous():
+        raise TypeError("workspace must be a contiguous CUDA tensor")
+    with torch.cuda.device(out_step.device):
+        _check(_lib.dc_reduce_trials(_dev(out_step, torch.float32, "out_step"), _dev(out_done, torch.int32, "out_done"),
+                                     None if out_sync is None else _dev(out_sync, torch.float32, "out_sync"),
+                                     T, K, int(N), int(M), _dev(stats, torch.float64, "stats"),
+                                     _dev(baseline, torch.float64, "baseline"), workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size(), _stream(out_step)), "dc_reduce_trials")
+
+
+def dc_argmax_tau(stats: torch.Tensor, taus: torch.Tensor, objective: int, out_k: torch.Tensor, out_tau: torch.Tensor,
+                  out_value: torch.Tensor) -> None:
+    K = taus.shape[0]
+    with torch.cuda.device(stats.device):
+        _check(_lib.dc_argmax_tau(_dev(stats, torch.float64, "stats"), _dev(taus, torch.float32, "taus"), K, int(objective),
+                                  _dev(out_k, torch.int32, "out_k"), _dev(out_tau, torch.float32, "out_tau"),
+                                  _dev(out_value, torch.float64, "out_value"), _stream(stats)), "dc_argmax_tau")
+
+
+def dc_check_inputs(latencies: torch.Tensor, taus: torch.Tensor) -> None:
+    """Synchronous data-precondition check; raises DropComputeError (DC_ERR_LATENCIES / DC_ERR_TAUS)."""
+    T, N, M = latencies.shape
+    counters = torch.empty(2, dtype=torch.int64, device=latencies.device)
+    with torch.cuda.device(latencies.device):
+        _check(_lib.dc_check_inputs(_dev(latencies, torch.float32, "latencies"), T, N, M, _dev(taus, torch.float32, "taus"),
+                                    taus.shape[0], counters.data_ptr(), None, _stream(latencies)), "dc_check_inputs")
+
+
+def dc_device_status() -> int:
+    """Reads and clears the device's expired-wait mask; raises if any wait expired."""
+    flags = ctypes.c_uint32(0)
+    rc = _lib.dc_device_status(ctypes.byref(flags))
+    _check(rc, f"dc_device_status (flags {flags.value:#x})")
+    return int(flags.value)
+
+
+def dc_simulate_plan(latencies: torch.Tensor, K: int) -> int:
+    T, N, M = latencies.shape
+    return int(_lib.dc_simulate_plan(latencies.data_ptr(), T, N, M, K))
+
+
+def dc_sweep_host_workspace_bytes(T: int, N: int, M: int, K: int, chunk_trials: int) -> int:
+    return int(_lib.dc_sweep_host_workspace_bytes(T, N, M, K, chunk_trials))
+
+
+class HostSweep(NamedTuple):
+    stats: torch.Tensor      # [NSTATS,K] fp64, host
+    baseline: torch.Tensor   # [2] fp64, host
+    k_star: int
+    tau_star: float
+
+
+def dc_sweep_host(latencies_host: torch.Tensor, taus_host: torch.Tensor, t_comm: float, workspace: torch.Tensor,
+                  chunk_trials: int, rule: int = RULE_FINISH_BEFORE_TAU, objective: int = STAT_S_EFF,
+                  stats_out: Optional[torch.Tensor] = None, baseline_out: Optional[torch.Tensor] = None) -> HostSweep:
+    """``dc_sweep_host``: latencies and thresholds in HOST memory (pin them for speed), results in
+    host memory; synchronous.  ``workspace`` is a CUDA byte tensor from dc_sweep_host_workspace_bytes."""
+    for t, dt, nm in ((latencies_host, torch.float32, "latencies_host"), (taus_host, torch.float32, "taus_host")):
+        if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+            raise TypeError(f"{nm} must be a contiguous host {dt} tensor")
+    T, N, M = latencies_host.shape
+    K = taus_host.shape[0]
+    stats = stats_out if stats_out is not None else torch.empty((NSTATS, K), dtype=torch.float64)
+    base = baseline_out if baseline_out is not None else torch.empty((2,), dtype=torch.float64)
+    k_star = ctypes.c_int32(-1)
+    tau_star = ctypes.c_float(float("nan"))
+    with torch.cuda.device(workspace.device):
+        _check(_lib.dc_sweep_host(latencies_host.data_ptr(), T, N, M, taus_host.data_ptr(), K, float(t_comm), int(rule),
+                                  int(objective), int(chunk_trials), stats.data_ptr(), base.data_ptr(),
+                                  ctypes.addressof(k_star), ctypes.addressof(tau_star), workspace.data_ptr(),
+                                  workspace.numel() * workspace.element_size(),
+                                  torch.cuda.current_stream(workspace.device).cuda_stream), "dc_sweep_host")
+    return HostSweep(stats, base, int(k_star.value), float(tau_star.value))
+
+
+def launches() -> dict:
+    return {"dc_simulate": _lib.dc_simulate_launches(), "dc_reduce_trials": _lib.dc_reduce_trials_launches(),
+            "dc_argmax_tau": _lib.dc_argmax_tau_launches()}
+
+
+# --- convenience wrapper (allocation + the three calls); still nothing but calls into the library ---------------
+
+class SweepResult(NamedTuple):
+    out_step: torch.Tensor   # [T,K] fp32
+    out_done: torch.Tensor   # [T,K] int32
+    out_sync: torch.Tensor   # [T] fp32
+    stats: torch.Tensor      # [NSTATS,K] fp64
+    baseline: torch.Tensor   # [2] fp64
+    k_star: torch.Tensor     # int32 scalar (device)
+    tau_star: torch.Tensor   # fp32 scalar (device)
+    value: torch.Tensor      # fp64 scalar (device)
+
+
+def sweep(latencies: torch.Tensor, taus: torch.Tensor, t_comm: float, rule: int = RULE_FINISH_BEFORE_TAU,
+          objective: int = STAT_S_EFF) -> SweepResult:
+    """Allocates the outputs with torch and runs dc_simulate_ex, dc_reduce_trials and dc_argmax_tau."""
+    T, N, M = latencies.shape
+    K = taus.shape[0]
+    dev = latencies.device
+    out_step = torch.empty((T, K), dtype=torch.float32, device=dev)
+    out_done = torch.empty((T, K), dtype=torch.int32, device=dev)
+    out_sync = torch.empty((T,), dtype=torch.float32, device=dev)
+    stats = torch.empty((NSTATS, K), dtype=torch.float64, device=dev)
+    baseline = torch.empty((2,), dtype=torch.float64, device=dev)
+    ws = torch.empty((max(8, dc_reduce_workspace_bytes(T, K)),), dtype=torch.uint8, device=dev)
+    k_star = torch.empty((), dtype=torch.int32, device=dev)
+    tau_star = torch.empty((), dtype=torch.float32, device=dev)
+    value = torch.empty((), dtype=torch.float64, device=dev)
+    dc_simulate_ex(latencies, taus, t_comm, out_step, out_done, out_sync, rule)
+    dc_reduce_trials(out_step, out_done, out_sync, N, M, stats, baseline, ws)
+    dc_argmax_tau(stats, taus, objective, out_k=k_star, out_tau=tau_star, out_value=value)
+    return SweepResult(out_step, out_done, out_sync, stats, baseline, k_star, tau_star, value)

@@ -1,0 +1,973 @@
+// DropCompute threshold-sweep simulator for sm_100a: kernels and the C ABI declared in
+// include/dropcompute.h.
+//
+// What is computed (paper: DropCompute, arXiv 2306.10598): Algorithm 2 (App. C.1) evaluates, for
+// every candidate threshold tau and every measured iteration, each worker's running compute time
+// T_{i,n} (micro-batch by micro-batch), the number of micro-batches whose running time is below
+// tau (the M~ of Sec. 4.3), the slowest worker's time T_i, the step time min(tau,T_i)+T^c and the
+// effective speedup S_i(tau) (Eq. 6); then it averages over iterations and takes the arg-max.
+//
+// How it is computed here.  The running sum does not depend on tau, so the samples are read ONCE.
+// A thread owns one worker's row of M latencies and adds them strictly left to right in fp32.
+// Because latencies are >= 0 the running sum P never decreases, and because the thresholds are
+// sorted, [P < tau_k] <=> k >= j(P) with j(P) = #{k : tau_k <= P}.  So each sample falls into one
+// bin j in [0,K] and done[t][k] is the prefix sum of the bin counts.  The thread keeps a cursor
+// (its current bin) that only moves forward and counts samples per bin by position, so the common
+// case costs one add and one compare per sample; bin counts go to per-warp integer histograms in
+// shared memory, which a per-trial epilogue sums, prefix-scans and writes out.  One block owns a
+// whole trial at a time (all N workers), so no global atomics and no scratch memory are needed
+// and every result is an integer sum or an exact maximum: bit-reproducible.
+//
+// Data movement.  The kernel is bound by the one read of latencies[T][N][M] from HBM.  Tiles of
+// (rows x up to 128 bytes of each row) are brought into shared memory by the TMA unit
+// (cp.async.bulk.tensor, 3-D tensor map over [T][N][M]) through a ring of stages guarded by
+// mbarriers; a dedicated producer warp issues the copies and the other warps consume.  The
+// hardware swizzle (128/64/32-byte modes) makes "lane r reads 16 bytes of row r" free of
+// shared-memory bank conflicts.  Rows past N in a trial's last pass and columns past M are
+// out-of-bounds coordinates of the tensor map: they are zero-filled by the TMA unit and cost no
+// HBM traffic.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "dropcompute.h"
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// constants
+// ------------------------------------------------------------------------------------------
+constexpr int kMaxRowsPerPass = 256;          // rows (threads) of one trial handled per pass; also the TMA box limit
+constexpr int kMaxStages = 8;
+constexpr int kStageBudgetBytes = 96 * 1024;  // shared memory spent on the ring of stages per block
+constexpr int kHistBudgetBytes = 32 * 1024;   // shared memory spent on per-warp histograms per block
+constexpr uint32_t kWaitLimit = 1u << 22;     // polls of one mbarrier wait before giving up (roughly a second)
+constexpr int kReduceChunksMax = 64;          // partial sums per threshold in dc_reduce_trials
+constexpr int kConsumerBarrier = 1;           // named barrier used by the consumer warps
+
+constexpr uint32_t kErrLoadNeverArrived = 1u;
+constexpr uint32_t kErrStageNeverFreed = 2u;
+
+__device__ unsigned int g_wait_expired = 0;   // bit mask of expired waits on this device
+
+struct SweepParams {
+    const float *lat;
+    const float *taus;
+    float *out_step;
+    int32_t *out_done;
+    float *out_sync;   // may be null
+    long long T;
+    int N, M, K;
+    float t_comm;
+    int passes;        // passes over a trial's workers
+    int rows;          // workers per pass (box height for the tiled kernel, blockDim.x for the plain one)
+    int chunks;        // column chunks per row
+    int bw;            // floats of a row per chunk (box width)
+    int nq_last;       // 16-byte quads of a row in the last chunk
+    int pitch;         // shared-memory bytes per row in a stage
+    int swz_mask;      // 7 / 3 / 1 / 0 for the 128 / 64 / 32-byte swizzle / none
+    int stages;
+    int stage_bytes;   // multiple of 1024
+    int hist_copies;   // per-warp histogram copies (power of two)
+    int hist_stride;   // ints per copy (>= K + 1)
+};
+
+// ------------------------------------------------------------------------------------------
+// small PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  If the limit is reached the fact is recorded and the caller carries on, so that
+// every thread still reaches every barrier and the kernel ends (its results are then garbage and
+// dc_device_status() says so).
+__device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, uint32_t err_bit)
+{
+    for (uint32_t it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return;
+        if (it > 64) __nanosleep(128);
+    }
+    atomicOr(&g_wait_expired, err_bit);
+}
+__device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int x, int y, int z, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_addr(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(smem_addr(bar))
+        : "memory");
+}
+__device__ __forceinline__ void named_barrier(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------
+// One worker's walk along its row (Algorithm 2's inner loop for all tau at once).
+// ------------------------------------------------------------------------------------------
+struct RowWalk {
+    float P;      // running compute time T_{i,n} after the samples seen so far
+    float tcur;   // tau_s[cur]; +inf once cur == K
+    int cur;      // number of thresholds <= the last P that moved the cursor (the current bin)
+    int mflush;   // index of the first sample not yet added to the histogram
+
+    __device__ __forceinline__ void start(const float *tau_s)
+    {
+        P = 0.0f;
+        cur = 0;
+        tcur = tau_s[0];
+        mflush = 0;
+    }
+    // sample number m (0-based) with latency x
+    __device__ __forceinline__ void step(float x, int m, const float *tau_s, int *hist, int K)
+    {
+        P = __fadd_rn(P, x);
+        if (P >= tcur) {  // leaves the current bin: samples mflush..m-1 were in it
+            const int c = m - mflush;
+            if (c > 0) atomicAdd(&hist[cur], c);
+            while (cur < K && P >= tcur) {
+                ++cur;
+                tcur = tau_s[cur];  // tau_s[K] = +inf
+            }
+            mflush = m;
+        }
+    }
+    __device__ __forceinline__ void finish(int M, int *hist)
+    {
+        const int c = M - mflush;
+        if (c > 0) atomicAdd(&hist[cur], c);
+    }
+};
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ int warp_inclusive_scan(int v, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += u;
+    }
+    return v;
+}
+
+// ------------------------------------------------------------------------------------------
+// End of a trial: all `nthr` participating threads call this with their largest row total.
+// Sums the histogram copies, prefix-scans the bins into done[t][k] (M~ * N of Sec. 4.3), takes
+// T = max_n T_n, writes step[t][k] = min(tau_k, T) + T^c and sync[t] = T + T^c, and clears the
+// histograms for the next trial.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t, float rowmax, int tid, int nthr,
+                                               int barrier_id, const float *tau_s, int *hist, float *smax, int *wtot)
+{
+    const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
+    const int K = p.K, H = p.hist_copies, HS = p.hist_stride;
+    rowmax = warp_max(rowmax);
+    if (lane == 0) smax[warp] = rowmax;
+    named_barrier(barrier_id, nthr);  // all histogram updates and smax[] visible
+
+    float Tmax = 0.0f;
+    for (int w = 0; w < nwarps; ++w) Tmax = fmaxf(Tmax, smax[w]);
+
+    const int ipt = (K + nthr - 1) / nthr;  // bins per thread (consecutive)
+    const int b0 = min(K, tid * ipt), b1 = min(K, b0 + ipt);
+    int tot = 0;
+    for (int b = b0; b < b1; ++b)
+        for (int c = 0; c < H; ++c) tot += hist[c * HS + b];
+    const int incl = warp_inclusive_scan(tot, lane);
+    if (lane == 31) wtot[warp] = incl;
+    named_barrier(barrier_id, nthr);
+
+    int run = incl - tot;
+    for (int w = 0; w < warp; ++w) run += wtot[w];
+    float *step_row = p.out_step + t * K;
+    int32_t *done_row = p.out_done + t * K;
+    for (int b = b0; b < b1; ++b) {
+        int h = 0;
+        for (int c = 0; c < H; ++c) {
+            h += hist[c * HS + b];
+            hist[c * HS + b] = 0;
+        }
+        run += h;
+        done_row[b] = run;
+        step_row[b] = __fadd_rn(fminf(tau_s[b], Tmax), p.t_comm);
+    }
+    if (tid < H) hist[tid * HS + K] = 0;  // the bin of samples at or above the last threshold
+    if (tid == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, p.t_comm);
+    named_barrier(barrier_id, nthr);  // histograms cleared, smax/wtot free again
+}
+
+// Shared-memory carve-up common to both kernels (after the stages of the tiled kernel).
+struct SmemTail {
+    float *tau_s;
+    int *hist;
+    float *smax;
+    int *wtot;
+};
+__device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepParams &p)
+{
+    SmemTail s;
+    s.tau_s = reinterpret_cast<float *>(base);
+    s.hist = reinterpret_cast<int *>(s.tau_s + (p.K + 1));
+    s.smax = reinterpret_cast<float *>(s.hist + p.hist_copies * p.hist_stride);
+    s.wtot = reinterpret_cast<int *>(s.smax + 32);
+    return s;
+}
+__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride)
+{
+    return sizeof(float) * (size_t)(K + 1) + sizeof(int) * (size_t)hist_copies * hist_stride + 64 * sizeof(int);
+}
+
+__device__ __forceinline__ void load_thresholds(const SweepParams &p, const SmemTail &s, int tid, int nthr)
+{
+    for (int k = tid; k < p.K; k += nthr) s.tau_s[k] = p.taus[k];
+    if (tid == 0) s.tau_s[p.K] = __int_as_float(0x7f800000);  // +inf sentinel
+    for (int i = tid; i < p.hist_copies * p.hist_stride; i += nthr) s.hist[i] = 0;
+}
+
+// ------------------------------------------------------------------------------------------
+// Tiled kernel: TMA-staged rows, one producer warp + consumer warps, persistent over trials.
+// NQ = 16-byte quads of a row per chunk held in registers (box width = 4*NQ floats at most).
+// ------------------------------------------------------------------------------------------
+template <int NQ>
+__global__ void __launch_bounds__(kMaxRowsPerPass + 32)
+dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char *stage0 = smem;
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)p.stages * p.stage_bytes);
+    uint64_t *empty = full + kMaxStages;
+    const SmemTail s = carve_tail(reinterpret_cast<unsigned char *>(empty + kMaxStages), p);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int ncw = (blockDim.x >> 5) - 1;  // consumer warps; the last warp is the producer
+    const int S = p.stages;
+
+    if (tid == 0) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(&full[i], 1);
+            mbar_init(&empty[i], ncw);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    load_thresholds(p, s, tid, blockDim.x);
+    __syncthreads();
+
+    if (warp == ncw) {
+        // ---------------- producer: one thread streams this block's tiles through the ring
+        if (lane == 0) {
+            uint32_t i = 0;
+            for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
+                for (int pass = 0; pass < p.passes; ++pass) {
+                    for (int c = 0; c < p.chunks; ++c, ++i) {
+                        const int st = i % S;
+                        const uint32_t use = i / S;
+                        if (use > 0) mbar_wait(&empty[st], (use & 1u) ^ 1u, kErrStageNeverFreed);
+                        mbar_arrive_expect_tx(&full[st], (uint32_t)(p.rows * p.pitch));
+                        tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, c * p.bw, pass * p.rows, (int)t, &full[st]);
+                    }
+                }
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers: thread r owns row (pass*rows + r) of the current trial
+    const int nthr = ncw * 32;
+    int *myhist = s.hist + (warp & (p.hist_copies - 1)) * p.hist_stride;
+    const uint32_t row_off = (uint32_t)tid * (uint32_t)p.pitch;
+    uint32_t i = 0;
+    for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
+        float rowmax = 0.0f;
+        for (int pass = 0; pass < p.passes; ++pass) {
+            const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
+            RowWalk w;
+            w.start(s.tau_s);
+            for (int c = 0; c < p.chunks; ++c, ++i) {
+                const int st = i % S;
+                mbar_wait(&full[st], (i / S) & 1u, kErrLoadNeverArrived);
+                const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes;
+                const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
+                float4 v[NQ];
+                if (valid) {
+#pragma unroll
+                    for (int q = 0; q < NQ; ++q) {
+                        if (q < nq) {
+                            uint32_t off = row_off + q * 16;
+                            off ^= ((off >> 7) & (uint32_t)p.swz_mask) << 4;
+                            v[q] = *reinterpret_cast<const float4 *>(stage + off);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[st]);  // this warp holds its part of the stage in registers
+                if (valid) {
+                    const int m0 = c * p.bw;
+#pragma unroll
+                    for (int q = 0; q < NQ; ++q) {
+                        if (q < nq) {
+                            w.step(v[q].x, m0 + 4 * q + 0, s.tau_s, myhist, p.K);
+                            w.step(v[q].y, m0 + 4 * q + 1, s.tau_s, myhist, p.K);
+                            w.step(v[q].z, m0 + 4 * q + 2, s.tau_s, myhist, p.K);
+                            w.step(v[q].w, m0 + 4 * q + 3, s.tau_s, myhist, p.K);
+                        }
+                    }
+                }
+            }
+            if (valid) {
+                w.finish(p.M, myhist);
+                rowmax = fmaxf(rowmax, w.P);
+            }
+        }
+        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Plain-load kernel for shapes the tensor map cannot describe (M not a multiple of 4, or a base
+// pointer that is only 4-byte aligned).  Same walk and epilogue; each thread reads its row
+// straight from global memory.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const SmemTail s = carve_tail(smem_raw, p);
+    const int tid = threadIdx.x, warp = tid >> 5, nthr = blockDim.x;
+    load_thresholds(p, s, tid, nthr);
+    __syncthreads();
+    int *myhist = s.hist + (warp & (p.hist_copies - 1)) * p.hist_stride;
+    for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
+        float rowmax = 0.0f;
+        for (int pass = 0; pass < p.passes; ++pass) {
+            const int n = pass * p.rows + tid;
+            if (n < p.N) {
+                const float *row = p.lat + ((size_t)t * p.N + n) * p.M;
+                RowWalk w;
+                w.start(s.tau_s);
+                for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), m, s.tau_s, myhist, p.K);
+                w.finish(p.M, myhist);
+                rowmax = fmaxf(rowmax, w.P);
+            }
+        }
+        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Trial statistics (fp64), two deterministic phases.
+// Phase 1: block (column tile of 32 thresholds, chunk of trials): 8 warps take the chunk's trials
+// round-robin, lanes are thresholds; per-warp sums are combined in warp order.
+// Workspace layout: double part[chunks][4][K] (sum step, sum done as int64 bits, sum done/step,
+// sum S) followed by double sync_part[chunks].
+// ------------------------------------------------------------------------------------------
+constexpr int kRedWarps = 8;
+
+__global__ void __launch_bounds__(kRedWarps * 32)
+dc_reduce_partial(const float *__restrict__ step, const int32_t *__restrict__ done, const float *__restrict__ sync,
+                  long long T, int K, double NM, int chunks, long long rows_per_chunk, double *ws)
+{
+    __shared__ double sh[kRedWarps][4][32];
+    __shared__ double shs[kRedWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int k = blockIdx.x * 32 + lane;
+    const int chunk = blockIdx.y;
+    const long long t0 = chunk * rows_per_chunk;
+    const long long t1 = min(T, t0 + rows_per_chunk);
+    double s_step = 0.0, s_ratio = 0.0, s_S = 0.0;
+    long long s_done = 0;
+    const double nan = __longlong_as_double(0x7ff8000000000000LL);
+    if (k < K) {
+        for (long long t = t0 + warp; t < t1; t += kRedWarps) {
+            const double st = (double)step[t * K + k];
+            const int dn_i = done[t * K + k];
+            const double dn = (double)dn_i;
+            const double sy = sync ? (double)sync[t] : nan;
+            s_step += st;
+            s_done += dn_i;
+            s_ratio += dn / st;
+            s_S += (sy / st) * (dn / NM);
+        }
+    }
+    sh[warp][0][lane] = s_step;
+    sh[warp][1][lane] = __longlong_as_double(s_done);
+    sh[warp][2][lane] = s_ratio;
+    sh[warp][3][lane] = s_S;
+    // sum of sync over this chunk (only the first column tile does it)
+    double ssum = 0.0;
+    if (blockIdx.x == 0 && sync) {
+        for (long long t = t0 + threadIdx.x; t < t1; t += kRedWarps * 32) ssum += (double)sync[t];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
+        if (lane == 0) shs[warp] = ssum;
+    }
+    __syncthreads();
+    if (warp == 0 && k < K) {
+        double a = 0.0, c = 0.0, d = 0.0;
+        long long b = 0;
+        for (int w = 0; w < kRedWarps; ++w) {
+            a += sh[w][0][lane];
+            b += __double_as_longlong(sh[w][1][lane]);
+            c += sh[w][2][lane];
+            d += sh[w][3][lane];
+        }
+        double *part = ws + (size_t)chunk * 4 * K;
+        part[0 * K + k] = a;
+        part[1 * K + k] = __longlong_as_double(b);
+        part[2 * K + k] = c;
+        part[3 * K + k] = d;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        double v = nan;
+        if (sync) {
+            v = 0.0;
+            for (int w = 0; w < kRedWarps; ++w) v += shs[w];
+        }
+        ws[(size_t)chunks * 4 * K + chunk] = v;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+dc_reduce_final(const double *__restrict__ ws, long long T, int K, double NM, int chunks, double *stats, double *baseline)
+{
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k < K) {
+        double a = 0.0, c = 0.0, d = 0.0;
+        long long b = 0;
+        for (int ch = 0; ch < chunks; ++ch) {
+            const double *part = ws + (size_t)ch * 4 * K;
+            a += part[0 * K + k];
+            b += __double_as_longlong(part[1 * K + k]);
+            c += part[2 * K + k];
+            d += part[3 * K + k];
+        }
+        const double Td = (double)T;
+        stats[DC_STAT_MEAN_STEP * K + k] = a / Td;
+        stats[DC_STAT_DONE_FRAC * K + k] = (double)b / (Td * NM);
+        stats[DC_STAT_THR * K + k] = (double)b / a;
+        stats[DC_STAT_THR_MEAN * K + k] = c / Td;
+        stats[DC_STAT_S_EFF * K + k] = d / Td;
+    }
+    if (k == 0) {
+        double ssum = 0.0;
+        for (int ch = 0; ch < chunks; ++ch) ssum += ws[(size_t)chunks * 4 * K + ch];
+        baseline[0] = ssum / (double)T;
+        baseline[1] = ((double)T * NM) / ssum;
+    }
+}
+
+// tau* = first index of the maximum, NaN never wins (one warp).
+__global__ void __launch_bounds__(32)
+dc_argmax_kernel(const double *__restrict__ obj, const float *__restrict__ taus, int K, int32_t *out_k, float *out_tau,
+                 double *out_value)
+{
+    const int lane = threadIdx.x;
+    int best = -1;
+    double bv = 0.0;
+    for (int k = lane; k < K; k += 32) {
+        const double v = obj[k];
+        if (v != v) continue;
+        if (best < 0 || v > bv) {
+            best = k;
+            bv = v;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const int ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const double ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const bool take = (ob >= 0) && (best < 0 || ov > bv || (ov == bv && ob < best));
+        if (take) {
+            best = ob;
+            bv = ov;
+        }
+    }
+    if (lane == 0) {
+        const double nan = __longlong_as_double(0x7ff8000000000000LL);
+        *out_k = best;
+        *out_tau = best >= 0 ? taus[best] : __int_as_float(0x7fc00000);
+        *out_value = best >= 0 ? bv : nan;
+    }
+}
+
+// Data precondition check: counts latencies that are negative, NaN or infinite, and thresholds
+// that are NaN or smaller than their predecessor.
+__global__ void __launch_bounds__(256)
+dc_check_kernel(const float *__restrict__ lat, unsigned long long total, const float *__restrict__ taus, int K,
+                unsigned long long *counters)
+{
+    unsigned long long bad = 0;
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const float x = lat[i];
+        if (!(x >= 0.0f) || !(x <= 3.402823466e38f)) ++bad;
+    }
+    if (bad) atomicAdd(&counters[0], bad);
+    if (blockIdx.x == 0) {
+        unsigned long long badt = 0;
+        for (int k = threadIdx.x; k < K; k += blockDim.x) {
+            const float x = taus[k];
+            if (x != x) ++badt;
+            else if (k > 0 && !(taus[k - 1] <= x)) ++badt;
+        }
+        if (badt) atomicAdd(&counters[1], badt);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+        return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    return fn;
+}
+
+struct DeviceInfo {
+    int sms = 0;
+    int max_smem_optin = 0;
+};
+bool device_info(DeviceInfo *out)
+{
+    static DeviceInfo cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (cache[dev].sms == 0) {
+        int sms = 0, smem = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+        if (cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
+        cache[dev].max_smem_optin = smem;
+        cache[dev].sms = sms;
+    }
+    *out = cache[dev];
+    return true;
+}
+
+int floor_pow2(int v)
+{
+    int p = 1;
+    while (p * 2 <= v) p *= 2;
+    return p;
+}
+
+int g_last_simulate_launches = 0;
+int g_last_reduce_launches = 0;
+int g_last_argmax_launches = 0;
+
+int validate_simulate(const float *lat, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K,
+                      const float *out_step, const int32_t *out_done, int32_t rule)
+{
+    if (!lat || !taus || !out_step || !out_done) return DC_ERR_NULL;
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return DC_ERR_SHAPE;
+    if (K > DC_MAX_K) return DC_ERR_RANGE;
+    if (N > INT32_MAX || M > INT32_MAX || N * M > (int64_t)INT32_MAX || T > (int64_t)INT32_MAX) return DC_ERR_RANGE;
+    if ((reinterpret_cast<uintptr_t>(lat) & 3) || (reinterpret_cast<uintptr_t>(taus) & 3) ||
+        (reinterpret_cast<uintptr_t>(out_step) & 3) || (reinterpret_cast<uintptr_t>(out_done) & 3))
+        return DC_ERR_ALIGN;
+    if (rule != DC_RULE_FINISH_BEFORE_TAU) return DC_ERR_UNSUPPORTED;
+    return DC_OK;
+}
+
+bool tiled_ok(const float *lat, int64_t M) { return (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0); }
+
+template <int NQ>
+int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
+                 cudaStream_t stream)
+{
+    auto kernel = dc_sweep_tiled<NQ>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
+    const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
+    kernel<<<(unsigned)grid, block, smem, stream>>>(map, p);
+    return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
+                  float *out_step, int32_t *out_done, float *out_sync, int32_t rule, void *stream_v)
+{
+    const int rc = validate_simulate(lat, T, N, M, taus, K, out_step, out_done, rule);
+    if (rc != DC_OK) return rc;
+    if (out_sync && (reinterpret_cast<uintptr_t>(out_sync) & 3)) return DC_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    DeviceInfo di;
+    if (!device_info(&di)) return DC_ERR_CUDA;
+
+    SweepParams p;
+    memset(&p, 0, sizeof(p));
+    p.lat = lat;
+    p.taus = taus;
+    p.out_step = out_step;
+    p.out_done = out_done;
+    p.out_sync = out_sync;
+    p.T = T;
+    p.N = (int)N;
+    p.M = (int)M;
+    p.K = K;
+    p.t_comm = t_comm;
+    p.passes = (int)((N + kMaxRowsPerPass - 1) / kMaxRowsPerPass);
+    p.rows = (int)((N + p.passes - 1) / p.passes);
+    const int row_threads = ((p.rows + 31) / 32) * 32;
+    p.hist_stride = K + 1;
+    p.hist_copies = floor_pow2(min(row_threads / 32, max(1, kHistBudgetBytes / (int)(sizeof(int) * p.hist_stride))));
+    const size_t tail = tail_bytes(K, p.hist_copies, p.hist_stride);
+
+    if (tiled_ok(lat, M)) {
+        EncodeTiledFn encode = get_encode_fn();
+        if (!encode) return DC_ERR_CUDA;
+        p.bw = (int)(M < 32 ? M : 32);
+        p.chunks = (int)((M + p.bw - 1) / p.bw);
+        const int last_cols = (int)(M - (int64_t)(p.chunks - 1) * p.bw);
+        p.nq_last = last_cols / 4;
+        p.pitch = p.bw * 4;
+        CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_NONE;
+        p.swz_mask = 0;
+        if (p.pitch == 128) { swz = CU_TENSOR_MAP_SWIZZLE_128B; p.swz_mask = 7; }
+        else if (p.pitch == 64) { swz = CU_TENSOR_MAP_SWIZZLE_64B; p.swz_mask = 3; }
+        else if (p.pitch == 32) { swz = CU_TENSOR_MAP_SWIZZLE_32B; p.swz_mask = 1; }
+        p.stage_bytes = ((p.rows * p.pitch + 1023) / 1024) * 1024;
+        p.stages = max(2, min(kMaxStages, kStageBudgetBytes / p.stage_bytes));
+
+        CUtensorMap map;
+        const cuuint64_t gdim[3] = {(cuuint64_t)M, (cuuint64_t)N, (cuuint64_t)T};
+        const cuuint64_t gstride[2] = {(cuuint64_t)M * 4, (cuuint64_t)N * (cuuint64_t)M * 4};
+        const cuuint32_t box[3] = {(cuuint32_t)p.bw, (cuuint32_t)p.rows, 1};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(lat), gdim, gstride, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return DC_ERR_CUDA;
+
+        const size_t smem = 1024 + (size_t)p.stages * p.stage_bytes + 2 * kMaxStages * sizeof(uint64_t) + tail;
+        if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
+        const int block = row_threads + 32;
+        const int nq = p.bw / 4;
+        int lrc;
+        if (nq <= 1) lrc = launch_tiled<1>(map, p, block, smem, T, di, stream);
+        else if (nq <= 2) lrc = launch_tiled<2>(map, p, block, smem, T, di, stream);
+        else if (nq <= 4) lrc = launch_tiled<4>(map, p, block, smem, T, di, stream);
+        else lrc = launch_tiled<8>(map, p, block, smem, T, di, stream);
+        if (lrc == DC_OK) g_last_simulate_launches = 1;
+        return lrc;
+    }
+
+    // plain-load kernel
+    p.rows = row_threads;  // one row per thread per pass
+    p.passes = (int)((N + p.rows - 1) / p.rows);
+    const size_t smem = tail;
+    if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
+    if (cudaFuncSetAttribute(dc_sweep_plain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return DC_ERR_CUDA;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, dc_sweep_plain, p.rows, smem) != cudaSuccess || occ < 1)
+        return DC_ERR_CUDA;
+    const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
+    dc_sweep_plain<<<(unsigned)grid, p.rows, smem, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
+    g_last_simulate_launches = 1;
+    return DC_OK;
+}
+
+struct ReducePlan {
+    int chunks;
+    long long rows_per_chunk;
+};
+ReducePlan reduce_plan(int64_t T)
+{
+    ReducePlan r;
+    long long chunks = (T + 31) / 32;
+    if (chunks > kReduceChunksMax) chunks = kReduceChunksMax;
+    if (chunks < 1) chunks = 1;
+    r.rows_per_chunk = (T + chunks - 1) / chunks;
+    r.chunks = (int)((T + r.rows_per_chunk - 1) / r.rows_per_chunk);
+    return r;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------
+extern "C" {
+
+int dc_simulate(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
+                float *out_step, int32_t *out_done, void *stream)
+{
+    return simulate_impl(latencies, T, N, M, taus, K, t_comm, out_step, out_done, nullptr, DC_RULE_FINISH_BEFORE_TAU, stream);
+}
+
+int dc_simulate_ex(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
+                   float *out_step, int32_t *out_done, float *out_sync, int32_t rule, void *stream)
+{
+    return simulate_impl(latencies, T, N, M, taus, K, t_comm, out_step, out_done, out_sync, rule, stream);
+}
+
+int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K)
+{
+    if (!latencies) return -DC_ERR_NULL;
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return -DC_ERR_SHAPE;
+    if (K > DC_MAX_K || N > INT32_MAX || M > INT32_MAX || N * M > (int64_t)INT32_MAX || T > (int64_t)INT32_MAX)
+        return -DC_ERR_RANGE;
+    if (reinterpret_cast<uintptr_t>(latencies) & 3) return -DC_ERR_ALIGN;
+    return tiled_ok(latencies, M) ? 0 : 1;
+}
+
+size_t dc_reduce_workspace_bytes(int64_t T, int32_t K)
+{
+    if (T <= 0 || K <= 0) return 0;
+    const ReducePlan r = reduce_plan(T);
+    return sizeof(double) * ((size_t)r.chunks * 4 * (size_t)K + (size_t)r.chunks);
+}
+
+int dc_reduce_trials(const float *out_step, const int32_t *out_done, const float *out_sync, int64_t T, int32_t K, int64_t N,
+                     int64_t M, double *stats, double *baseline, void *workspace, size_t workspace_bytes, void *stream_v)
+{
+    if (!out_step || !out_done || !stats || !baseline) return DC_ERR_NULL;
+    if (T <= 0 || K <= 0 || N <= 0 || M <= 0) return DC_ERR_SHAPE;
+    if (K > DC_MAX_K || N * M > (int64_t)INT32_MAX) return DC_ERR_RANGE;
+    if ((reinterpret_cast<uintptr_t>(stats) & 7) || (reinterpret_cast<uintptr_t>(baseline) & 7)) return DC_ERR_ALIGN;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 7) || workspace_bytes < dc_reduce_workspace_bytes(T, K))
+        return DC_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const ReducePlan r = reduce_plan(T);
+    const double NM = (double)N * (double)M;
+    double *ws = static_cast<double *>(workspace);
+    dim3 grid1((unsigned)((K + 31) / 32), (unsigned)r.chunks);
+    dc_reduce_partial<<<grid1, kRedWarps * 32, 0, stream>>>(out_step, out_done, out_sync, T, K, NM, r.chunks, r.rows_per_chunk, ws);
+    if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
+    dc_reduce_final<<<(unsigned)((K + 255) / 256), 256, 0, stream>>>(ws, T, K, NM, r.chunks, stats, baseline);
+    if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
+    g_last_reduce_launches = 2;
+    return DC_OK;
+}
+
+int dc_argmax_tau(const double *stats, const float *taus, int32_t K, int32_t objective, int32_t *out_k, float *out_tau,
+                  double *out_value, void *stream_v)
+{
+    if (!stats || !taus || !out_k || !out_tau || !out_value) return DC_ERR_NULL;
+    if (K <= 0) return DC_ERR_SHAPE;
+    if (K > DC_MAX_K) return DC_ERR_RANGE;
+    if (objective != DC_STAT_S_EFF && objective != DC_STAT_THR && objective != DC_STAT_THR_MEAN) return DC_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(stats) & 7) || (reinterpret_cast<uintptr_t>(out_value) & 7)) return DC_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    dc_argmax_kernel<<<1, 32, 0, stream>>>(stats + (size_t)objective * K, taus, K, out_k, out_tau, out_value);
+    if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
+    g_last_argmax_launches = 1;
+    return DC_OK;
+}
+
+int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, int64_t *counters,
+                    int64_t *report_host, void *stream_v)
+{
+    if (!latencies || !taus || !counters) return DC_ERR_NULL;
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return DC_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(counters) & 7) return DC_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    DeviceInfo di;
+    if (!device_info(&di)) return DC_ERR_CUDA;
+    if (cudaMemsetAsync(counters, 0, 16, stream) != cudaSuccess) return DC_ERR_CUDA;
+    const unsigned long long total = (unsigned long long)T * (unsigned long long)N * (unsigned long long)M;
+    unsigned long long want = (total + 255) / 256;
+    const unsigned grid = (unsigned)(want < (unsigned long long)di.sms * 8 ? (want ? want : 1) : (unsigned long long)di.sms * 8);
+    dc_check_kernel<<<grid, 256, 0, stream>>>(latencies, total, taus, K, reinterpret_cast<unsigned long long *>(counters));
+    if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
+    int64_t host[2] = {0, 0};
+    if (cudaMemcpyAsync(host, counters, 16, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return DC_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return DC_ERR_CUDA;
+    if (report_host) {
+        report_host[0] = host[0];
+        report_host[1] = host[1];
+    }
+    if (host[0] != 0) return DC_ERR_LATENCIES;
+    if (host[1] != 0) return DC_ERR_TAUS;
+    return DC_OK;
+}
+
+int dc_device_status(uint32_t *flags_host)
+{
+    unsigned int flags = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&flags, g_wait_expired, sizeof(flags)) != cudaSuccess) return DC_ERR_CUDA;
+    if (flags != 0 && cudaMemcpyToSymbol(g_wait_expired, &zero, sizeof(zero)) != cudaSuccess) return DC_ERR_CUDA;
+    if (flags_host) *flags_host = flags;
+    return flags == 0 ? DC_OK : DC_ERR_DEVICE;
+}
+
+size_t dc_sweep_host_workspace_bytes(int64_t T, int64_t N, int64_t M, int32_t K, int64_t chunk_trials)
+{
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0 || chunk_trials <= 0) return 0;
+    if (chunk_trials > T) chunk_trials = T;
+    const size_t chunk = align_up((size_t)chunk_trials * (size_t)N * (size_t)M * 4, 1024);
+    size_t total = 2 * chunk;
+    total += align_up((size_t)K * 4, 256);                       // taus
+    total += align_up((size_t)T * (size_t)K * 4, 256) * 2;       // step, done
+    total += align_up((size_t)T * 4, 256);                       // sync
+    total += align_up((size_t)DC_NSTATS * (size_t)K * 8, 256);   // stats
+    total += 256;                                                // baseline[2], value, k, tau
+    total += align_up(dc_reduce_workspace_bytes(T, K), 256);
+    return total;
+}
+
+int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M, const float *taus_host, int32_t K,
+                  float t_comm, int32_t rule, int32_t objective, int64_t chunk_trials, double *stats_host,
+                  double *baseline_host, int32_t *k_star_host, float *tau_star_host, void *workspace, size_t workspace_bytes,
+                  void *stream_v)
+{
+    if (!latencies_host || !taus_host || !stats_host || !baseline_host || !k_star_host || !tau_star_host) return DC_ERR_NULL;
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0 || chunk_trials <= 0) return DC_ERR_SHAPE;
+    if (K > DC_MAX_K || N > INT32_MAX || M > INT32_MAX || N * M > (int64_t)INT32_MAX || T > (int64_t)INT32_MAX)
+        return DC_ERR_RANGE;
+    if (rule != DC_RULE_FINISH_BEFORE_TAU) return DC_ERR_UNSUPPORTED;
+    if (objective != DC_STAT_S_EFF && objective != DC_STAT_THR && objective != DC_STAT_THR_MEAN) return DC_ERR_UNSUPPORTED;
+    if (chunk_trials > T) chunk_trials = T;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023) ||
+        workspace_bytes < dc_sweep_host_workspace_bytes(T, N, M, K, chunk_trials))
+        return DC_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+
+    // carve the workspace
+    unsigned char *w = static_cast<unsigned char *>(workspace);
+    const size_t chunk_bytes = align_up((size_t)chunk_trials * (size_t)N * (size_t)M * 4, 1024);
+    float *buf[2] = {reinterpret_cast<float *>(w), reinterpret_cast<float *>(w + chunk_bytes)};
+    w += 2 * chunk_bytes;
+    float *d_taus = reinterpret_cast<float *>(w);
+    w += align_up((size_t)K * 4, 256);
+    float *d_step = reinterpret_cast<float *>(w);
+    w += align_up((size_t)T * (size_t)K * 4, 256);
+    int32_t *d_done = reinterpret_cast<int32_t *>(w);
+    w += align_up((size_t)T * (size_t)K * 4, 256);
+    float *d_sync = reinterpret_cast<float *>(w);
+    w += align_up((size_t)T * 4, 256);
+    double *d_stats = reinterpret_cast<double *>(w);
+    w += align_up((size_t)DC_NSTATS * (size_t)K * 8, 256);
+    double *d_base = reinterpret_cast<double *>(w);        // [2]
+    double *d_value = d_base + 2;
+    int32_t *d_k = reinterpret_cast<int32_t *>(d_base + 3);
+    float *d_tau = reinterpret_cast<float *>(d_base + 4);
+    w += 256;
+    void *d_red = w;
+    const size_t red_bytes = dc_reduce_workspace_bytes(T, K);
+
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ready[2] = {nullptr, nullptr}, freed[2] = {nullptr, nullptr};
+    int rc = DC_OK;
+    bool cuda_fail = false;
+#define DC_TRY(call)                                  \
+    do {                                              \
+        if (!cuda_fail && (call) != cudaSuccess) {    \
+            cuda_fail = true;                         \
+        }                                             \
+    } while (0)
+    DC_TRY(cudaStreamCreateWithFlags(&copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+        DC_TRY(cudaEventCreateWithFlags(&ready[i], cudaEventDisableTiming));
+        DC_TRY(cudaEventCreateWithFlags(&freed[i], cudaEventDisableTiming));
+    }
+    DC_TRY(cudaMemcpyAsync(d_taus, taus_host, (size_t)K * 4, cudaMemcpyHostToDevice, stream));
+    int launches = 0;
+    const int64_t nchunks = (T + chunk_trials - 1) / chunk_trials;
+    for (int64_t c = 0; c < nchunks && !cuda_fail && rc == DC_OK; ++c) {
+        const int b = (int)(c & 1);
+        const int64_t t0 = c * chunk_trials;
+        const int64_t tn = (t0 + chunk_trials <= T) ? chunk_trials : (T - t0);
+        if (c >= 2) DC_TRY(cudaStreamWaitEvent(copy_stream, freed[b], 0));
+        DC_TRY(cudaMemcpyAsync(buf[b], latencies_host + (size_t)t0 * N * M, (size_t)tn * N * M * 4, cudaMemcpyHostToDevice,
+                               copy_stream));
+        DC_TRY(cudaEventRecord(ready[b], copy_stream));
+        DC_TRY(cudaStreamWaitEvent(stream, ready[b], 0));
+        if (!cuda_fail) {
+            rc = simulate_impl(buf[b], tn, N, M, d_taus, K, t_comm, d_step + (size_t)t0 * K, d_done + (size_t)t0 * K,
+                               d_sync + t0, rule, stream);
+            launches += 1;
+        }
+        DC_TRY(cudaEventRecord(freed[b], stream));
+    }
+    if (!cuda_fail && rc == DC_OK)
+        rc = dc_reduce_trials(d_step, d_done, d_sync, T, K, N, M, d_stats, d_base, d_red, red_bytes, stream);
+    if (!cuda_fail && rc == DC_OK) rc = dc_argmax_tau(d_stats, d_taus, K, objective, d_k, d_tau, d_value, stream);
+    if (!cuda_fail && rc == DC_OK) {
+        DC_TRY(cudaMemcpyAsync(stats_host, d_stats, (size_t)DC_NSTATS * K * 8, cudaMemcpyDeviceToHost, stream));
+        DC_TRY(cudaMemcpyAsync(baseline_host, d_base, 16, cudaMemcpyDeviceToHost, stream));
+        DC_TRY(cudaMemcpyAsync(k_star_host, d_k, 4, cudaMemcpyDeviceToHost, stream));
+        DC_TRY(cudaMemcpyAsync(tau_star_host, d_tau, 4, cudaMemcpyDeviceToHost, stream));
+    }
+    // always drain both streams before the events and the copy stream go away
+    if (copy_stream) cudaStreamSynchronize(copy_stream);
+    if (cudaStreamSynchronize(stream) != cudaSuccess) cuda_fail = true;
+#undef DC_TRY
+    for (int i = 0; i < 2; ++i) {
+        if (ready[i]) cudaEventDestroy(ready[i]);
+        if (freed[i]) cudaEventDestroy(freed[i]);
+    }
+    if (copy_stream) cudaStreamDestroy(copy_stream);
+    if (cuda_fail) return DC_ERR_CUDA;
+    if (rc == DC_OK) g_last_simulate_launches = launches;
+    return rc;
+}
+
+int dc_simulate_launches(void) { return g_last_simulate_launches; }
+int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
+int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
+
+const char *dc_status_string(int status)
+{
+    switch (status) {
+    case DC_OK: return "ok";
+    case DC_ERR_NULL: return "a required pointer is NULL";
+    case DC_ERR_SHAPE: return "T, N, M and K must be positive";
+    case DC_ERR_ALIGN: return "a pointer is not aligned as documented";
+    case DC_ERR_RANGE: return "a size is beyond what the library supports";
+    case DC_ERR_TAUS: return "thresholds are not non-decreasing or contain NaN";
+    case DC_ERR_CUDA: return "a CUDA call failed";
+    case DC_ERR_UNSUPPORTED: return "unknown rule or objective";
+    case DC_ERR_LATENCIES: return "latencies contain a negative, NaN or infinite value";
+    case DC_ERR_WORKSPACE: return "workspace is NULL, misaligned or too small";
+    case DC_ERR_DEVICE: return "a bounded wait inside a kernel expired";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,279 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element, on seeded
+inputs.  Integers and step times must match bit for bit; fp64 statistics within 1e-9 relative."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2306_10598_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+RTOL_STATS = 1e-9   # fp64 sums of <= 2^15 terms taken in a different order: far below this
+INF = float("inf")
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2306_10598_b200 import api as _api
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    return _api
+
+
+def grid_for(lat: np.ndarray, K: int, seed: int) -> np.ndarray:
+    """A sorted grid spanning below the smallest and above the largest worker time, with a repeated
+    value, an exact worker total (a tie) and +inf at the end when K allows."""
+    rng = np.random.default_rng(seed)
+    tot = np.cumsum(lat, axis=-1, dtype=np.float32)
+    hi = float(tot[..., -1].max())
+    g = rng.uniform(-0.05 * hi, 1.15 * hi, K).astype(np.float32)
+    if K >= 4:
+        g[0] = tot.reshape(-1)[rng.integers(tot.size)]      # equals some running sum exactly
+        g[1] = g[2]                                          # duplicate
+        g[3] = np.float32(INF)
+    g.sort()
+    return g
+
+
+def run_gpu(api, lat_d, taus_d, t_comm, rule=0, objective=4):
+    r = api.sweep(lat_d, taus_d, t_comm, rule=rule, objective=objective)
+    torch.cuda.synchronize()
+    return r
+
+
+def compare_sweep(res, ref, what=""):
+    assert np.array_equal(res.out_done.cpu().numpy(), ref.done), f"out_done differs {what}"
+    assert np.array_equal(res.out_step.cpu().numpy().view(np.uint32), ref.step.view(np.uint32)), f"out_step differs {what}"
+    assert np.array_equal(res.out_sync.cpu().numpy().view(np.uint32), ref.sync.view(np.uint32)), f"out_sync differs {what}"
+
+
+def compare_stats(res, ref_sweep, N, M, objective=4, what=""):
+    st = oracle.reduce_trials(ref_sweep.step, ref_sweep.done, ref_sweep.sync, N, M)
+    got = res.stats.cpu().numpy()
+    assert np.allclose(got, st.stats, rtol=RTOL_STATS, atol=0, equal_nan=True), f"stats differ {what}"
+    assert np.allclose(res.baseline.cpu().numpy(), st.baseline, rtol=RTOL_STATS, atol=0), f"baseline differs {what}"
+    k_ref = oracle.argmax(st.stats[objective])
+    assert int(res.k_star.item()) == k_ref, f"k* differs {what}"
+    return st
+
+
+EDGE_SHAPES = [
+    # T, N, M, K                      what it exercises
+    (1, 1, 1, 1),                    # everything degenerate (plain-load kernel)
+    (3, 7, 1, 5),                    # M = 1
+    (5, 1, 3, 4),                    # one worker, odd M
+    (4, 33, 129, 17),                # odd M > 128, ragged warp
+    (9, 8, 4, 16),                   # tiny's shape: 16-byte rows, no swizzle
+    (7, 40, 8, 9),                   # 32-byte rows, 32-byte swizzle
+    (6, 200, 12, 64),                # the paper's 12 accumulations: 48-byte rows, no swizzle
+    (4, 100, 16, 33),                # 64-byte swizzle
+    (3, 70, 20, 12), (3, 64, 24, 7), (2, 31, 28, 300),
+    (5, 200, 32, 64),                # one 128-byte chunk, 200 rows in 7 warps
+    (5, 300, 36, 40),                # two passes of 150 rows, ragged second column chunk
+    (3, 9, 100, 50),                 # four column chunks, last one 16 bytes
+    (3, 513, 64, 256),               # three passes of 171 rows
+    (2, 2048, 128, 256),             # the stress shape: 8 passes x 4 chunks per trial
+    (2, 256, 32, 4096),              # the largest grid
+    (300, 5, 16, 3),                 # many short trials, more trials than blocks in flight
+    (1, 1000, 8, 1),                 # one trial only
+]
+
+
+@pytest.mark.parametrize("T,N,M,K", EDGE_SHAPES)
+def test_edge_shapes_match_oracle(api, T, N, M, K):
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=100 + T + N + M, shift=0.01, mean=0.02).numpy()
+    taus = grid_for(lat, K, seed=K)
+    t_comm = 0.0625 + 0.001
+    ref = oracle.sweep(lat, taus, t_comm)
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    res = run_gpu(api, lat_d, taus_d, t_comm)
+    compare_sweep(res, ref, f"{(T, N, M, K)}")
+    compare_stats(res, ref, N, M, what=f"{(T, N, M, K)}")
+    # plain dc_simulate (no sync output) gives the same step/done
+    step2 = torch.full_like(res.out_step, -1.0)
+    done2 = torch.full_like(res.out_done, -1)
+    api.dc_simulate(lat_d, taus_d, t_comm, step2, done2)
+    torch.cuda.synchronize()
+    assert torch.equal(step2, res.out_step) and torch.equal(done2, res.out_done)
+    # a second call gives the same bits
+    res2 = run_gpu(api, lat_d, taus_d, t_comm)
+    for a, b in zip(res, res2):
+        assert torch.equal(a.reshape(-1).view(torch.uint8), b.reshape(-1).view(torch.uint8))
+    api.dc_device_status()
+
+
+def test_unaligned_base_takes_plain_kernel(api):
+    T, N, M, K = 4, 50, 16, 11
+    lat = W.iid_latencies("uniform", T, N, M, seed=5, lo=0.0, hi=0.1).numpy()
+    taus = grid_for(lat, K, 3)
+    buf = torch.zeros(T * N * M + 1, dtype=torch.float32, device="cuda")
+    view = buf[1:].view(T, N, M)
+    view.copy_(torch.from_numpy(lat))
+    assert api.dc_simulate_plan(view, K) == 1
+    assert api.dc_simulate_plan(torch.from_numpy(lat).cuda(), K) == 0
+    res = run_gpu(api, view, torch.from_numpy(taus).cuda(), 0.3)
+    compare_sweep(res, oracle.sweep(lat, taus, 0.3))
+
+
+def test_zero_and_tie_latencies(api):
+    # dyadic values: many running sums coincide with thresholds exactly, zeros repeat a running sum
+    T, N, M, K = 6, 37, 24, 40
+    lat = W.iid_latencies("dyadic", T, N, M, seed=6, hi=8).numpy()
+    lat[:, ::3, ::2] = 0.0
+    taus = (np.arange(K, dtype=np.float32) / 16.0)
+    ref = oracle.sweep(lat, taus, 0.25)
+    res = run_gpu(api, torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda(), 0.25)
+    compare_sweep(res, ref)
+    compare_stats(res, ref, N, M)
+
+
+def test_thresholds_outside_the_data(api):
+    T, N, M = 5, 20, 8
+    lat = W.iid_latencies("uniform", T, N, M, seed=7, lo=0.01, hi=0.02).numpy()
+    for taus in ([-1.0, 0.0], [0.0], [INF], [-INF, INF], [1e30, INF, INF], [0.05] * 7):
+        taus = np.array(taus, np.float32)
+        ref = oracle.sweep(lat, taus, 0.5)
+        res = run_gpu(api, torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda(), 0.5)
+        compare_sweep(res, ref, str(taus))
+
+
+def test_objectives(api):
+    T, N, M, K = 64, 30, 12, 25
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=8, shift=0.02, mean=0.03).numpy()
+    taus = np.linspace(0.3, 1.2, K).astype(np.float32)
+    ref = oracle.sweep(lat, taus, 0.1)
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    for obj in (api.STAT_S_EFF, api.STAT_THR, api.STAT_THR_MEAN):
+        res = run_gpu(api, lat_d, taus_d, 0.1, objective=obj)
+        st = compare_stats(res, ref, N, M, objective=obj)
+        k = int(res.k_star.item())
+        assert float(res.tau_star.item()) == float(taus[k])
+        assert np.isclose(float(res.value.item()), st.stats[obj, k], rtol=RTOL_STATS)
+    # without the synchronous baseline S_eff and the baseline are NaN, the rest unchanged
+    stats = torch.empty((api.NSTATS, K), dtype=torch.float64, device="cuda")
+    base = torch.empty(2, dtype=torch.float64, device="cuda")
+    ws = torch.empty(api.dc_reduce_workspace_bytes(T, K), dtype=torch.uint8, device="cuda")
+    api.dc_reduce_trials(res.out_step, res.out_done, None, N, M, stats, base, ws)
+    torch.cuda.synchronize()
+    assert torch.isnan(stats[api.STAT_S_EFF]).all() and torch.isnan(base).all()
+    assert torch.equal(stats[:4], res.stats[:4])
+
+
+def test_check_inputs(api):
+    lat = torch.rand(4, 5, 6, device="cuda")
+    taus = torch.tensor([0.1, 0.2, 0.2, INF], device="cuda")
+    api.dc_check_inputs(lat, taus)
+    bad = lat.clone()
+    bad[1, 2, 3] = -0.5
+    with pytest.raises(api.DropComputeError) as e:
+        api.dc_check_inputs(bad, taus)
+    assert e.value.status == 8
+    bad[1, 2, 3] = float("nan")
+    with pytest.raises(api.DropComputeError):
+        api.dc_check_inputs(bad, taus)
+    with pytest.raises(api.DropComputeError) as e:
+        api.dc_check_inputs(lat, torch.tensor([0.3, 0.2], device="cuda"))
+    assert e.value.status == 5
+    with pytest.raises(api.DropComputeError):
+        api.dc_check_inputs(lat, torch.tensor([0.3, float("nan")], device="cuda"))
+    with pytest.raises(TypeError):
+        api.dc_simulate(lat.double(), taus, 0.1, torch.empty(4, 4, device="cuda"),
+                        torch.empty(4, 4, dtype=torch.int32, device="cuda"))
+
+
+def test_sweep_host_matches_oracle(api):
+    T, N, M, K = 37, 64, 16, 20
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=9, shift=0.02, mean=0.01)
+    taus = np.linspace(0.3, 0.7, K).astype(np.float32)
+    ref = oracle.sweep(lat.numpy(), taus, 0.1)
+    st = oracle.reduce_trials(ref.step, ref.done, ref.sync, N, M)
+    for chunk in (5, 37, 100):
+        ws = torch.empty(api.dc_sweep_host_workspace_bytes(T, N, M, K, chunk) + 1024, dtype=torch.uint8, device="cuda")
+        off = (-ws.data_ptr()) % 1024
+        hs = api.dc_sweep_host(lat.pin_memory(), torch.from_numpy(taus), 0.1, ws[off:], chunk)
+        assert np.allclose(hs.stats.numpy(), st.stats, rtol=RTOL_STATS, atol=0)
+        assert np.allclose(hs.baseline.numpy(), st.baseline, rtol=RTOL_STATS, atol=0)
+        assert hs.k_star == oracle.argmax(st.stats[4]) and hs.tau_star == float(taus[hs.k_star])
+
+
+# ---- the five benchmark workloads ---------------------------------------------------------------
+
+def _full_parity(api, w):
+    lat_d = W.fill_latencies(w, "cuda")
+    taus = W.make_taus(w)
+    res = run_gpu(api, lat_d, torch.from_numpy(taus).cuda(), w.t_comm)
+    ref = oracle.sweep(lat_d.cpu().numpy(), taus, w.t_comm)
+    compare_sweep(res, ref, w.name)
+    compare_stats(res, ref, w.N, w.M, what=w.name)
+    api.dc_device_status()
+
+
+def test_workload_tiny(api):
+    _full_parity(api, W.WORKLOADS["tiny"])
+
+
+def test_workload_paper_scale(api):
+    _full_parity(api, W.WORKLOADS["paper_scale"])
+
+
+def test_workload_extrapolation(api):
+    _full_parity(api, W.WORKLOADS["extrapolation"])
+
+
+def _sampled_parity(api, w, n_sample):
+    """Full-size run in the benchmark's launch configuration; the oracle recomputes sampled trials
+    one by one (it cannot finish all of them in seconds), and properties that hold at any size
+    are checked on every output."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < w.latency_bytes + (4 << 30):
+        pytest.skip(f"needs {w.latency_bytes / 2**30:.1f} GiB of device memory")
+    lat_d = W.fill_latencies(w, "cuda")
+    taus = W.make_taus(w)
+    taus_d = torch.from_numpy(taus).cuda()
+    res = run_gpu(api, lat_d, taus_d, w.t_comm)
+    rng = np.random.default_rng(1234)
+    idx = np.unique(np.concatenate([[0, 1, w.T - 1], rng.integers(0, w.T, n_sample)]))
+    idx_d = torch.from_numpy(idx).cuda()
+    sample = lat_d[idx_d].cpu().numpy()
+    ref = oracle.sweep(sample, taus, w.t_comm)
+    assert np.array_equal(res.out_done[idx_d].cpu().numpy(), ref.done)
+    assert np.array_equal(res.out_step[idx_d].cpu().numpy().view(np.uint32), ref.step.view(np.uint32))
+    assert np.array_equal(res.out_sync[idx_d].cpu().numpy().view(np.uint32), ref.sync.view(np.uint32))
+    # trial statistics on the sampled trials: each side reduces its own (bit-identical) outputs
+    Ts = len(idx)
+    st_d = torch.empty((api.NSTATS, w.K), dtype=torch.float64, device="cuda")
+    base_d = torch.empty(2, dtype=torch.float64, device="cuda")
+    ws = torch.empty(api.dc_reduce_workspace_bytes(Ts, w.K), dtype=torch.uint8, device="cuda")
+    api.dc_reduce_trials(res.out_step[idx_d].contiguous(), res.out_done[idx_d].contiguous(),
+                         res.out_sync[idx_d].contiguous(), w.N, w.M, st_d, base_d, ws)
+    st = oracle.reduce_trials(ref.step, ref.done, ref.sync, w.N, w.M)
+    assert np.allclose(st_d.cpu().numpy(), st.stats, rtol=RTOL_STATS, atol=0)
+    assert np.allclose(base_d.cpu().numpy(), st.baseline, rtol=RTOL_STATS, atol=0)
+    # properties at full size
+    done, step, sync = res.out_done, res.out_step, res.out_sync
+    assert bool((done[:, 1:] >= done[:, :-1]).all()) and bool((step[:, 1:] >= step[:, :-1]).all())
+    assert int(done.min()) >= 0 and int(done.max()) <= w.N * w.M
+    tc = torch.tensor(w.t_comm, dtype=torch.float32, device="cuda")
+    assert bool((step <= (taus_d[None, :] + tc)).all()) and bool((step <= sync[:, None]).all())
+    rowsum_max = lat_d[idx_d].sum(-1).max(-1).values            # approximately the max worker time
+    assert torch.allclose(sync[idx_d] - tc, rowsum_max, rtol=1e-4)
+    full = taus_d[None, :] > (sync[:, None] - tc) * 1.001       # thresholds clearly above the slowest worker
+    assert bool((done[full] == w.N * w.M).all())
+    stats = res.stats.cpu().numpy()
+    assert np.isfinite(stats).all()
+    assert (np.diff(stats[api.STAT_MEAN_STEP]) >= 0).all() and (np.diff(stats[api.STAT_DONE_FRAC]) >= 0).all()
+    assert 0 <= stats[api.STAT_DONE_FRAC].min() and stats[api.STAT_DONE_FRAC].max() <= 1
+    # the full-size statistics equal the mean of the per-trial values computed with torch in fp64
+    S = (sync.double()[:, None] / step.double()) * (done.double() / (w.N * w.M))
+    assert np.allclose(stats[api.STAT_S_EFF], S.mean(0).cpu().numpy(), rtol=1e-9)
+    assert np.allclose(stats[api.STAT_MEAN_STEP], step.double().mean(0).cpu().numpy(), rtol=1e-9)
+    assert int(res.k_star.item()) == int(np.argmax(stats[api.STAT_S_EFF]))
+    api.dc_device_status()
+
+
+def test_workload_correlated_sampled(api):
+    _sampled_parity(api, W.WORKLOADS["correlated"], 96)
+
+
+def test_workload_bandwidth_stress_sampled(api):
+    _sampled_parity(api, W.WORKLOADS["bandwidth_stress"], 64)

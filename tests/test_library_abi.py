@@ -1,0 +1,80 @@
+"""The C-ABI library loads without a GPU, exports every function the header declares, and turns
+host-visible argument errors into status codes before touching CUDA (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "dropcompute.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2306_10598_b200 import build
+    build.build_library()
+    from paper_2306_10598_b200 import api
+    return api._lib
+
+
+def declared_functions():
+    with open(HEADER) as f:
+        text = f.read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b(dc_[a-z_0-9]+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_header_functions_are_exported(lib):
+    names = declared_functions()
+    assert "dc_simulate" in names and "dc_reduce_trials" in names and "dc_argmax_tau" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in dropcompute.h but not exported"
+    from paper_2306_10598_b200 import api
+    assert sorted(api.EXPORTS) == names, "the Python binding must list exactly the header's functions"
+
+
+def test_argument_errors_need_no_gpu(lib):
+    A = 0x10000  # a made-up aligned address: validation fails before anything is dereferenced
+    f = ctypes.c_float(0.1)
+    # null pointers
+    assert lib.dc_simulate(None, 1, 1, 1, A, 1, f, A, A, None) == 1
+    assert lib.dc_simulate(A, 1, 1, 1, None, 1, f, A, A, None) == 1
+    assert lib.dc_simulate(A, 1, 1, 1, A, 1, f, None, A, None) == 1
+    assert lib.dc_simulate(A, 1, 1, 1, A, 1, f, A, None, None) == 1
+    # shapes
+    for T, N, M, K in ((0, 1, 1, 1), (1, 0, 1, 1), (1, 1, -3, 1), (1, 1, 1, 0)):
+        assert lib.dc_simulate(A, T, N, M, A, K, f, A, A, None) == 2
+    # ranges: K beyond the maximum, N*M beyond int32
+    assert lib.dc_simulate(A, 1, 1, 1, A, 4097, f, A, A, None) == 4
+    assert lib.dc_simulate(A, 1, 1 << 20, 1 << 12, A, 1, f, A, A, None) == 4
+    # alignment
+    assert lib.dc_simulate(A + 2, 1, 1, 1, A, 1, f, A, A, None) == 3
+    assert lib.dc_simulate(A, 1, 1, 1, A + 1, 1, f, A, A, None) == 3
+    # unknown rule
+    assert lib.dc_simulate_ex(A, 1, 1, 1, A, 1, f, A, A, None, 5, None) == 7
+    # reduce / argmax
+    assert lib.dc_reduce_trials(None, A, A, 1, 1, 1, 1, A, A, A, 1 << 20, None) == 1
+    assert lib.dc_reduce_trials(A, A, A, 1, 1, 1, 1, A, A, None, 0, None) == 9
+    assert lib.dc_reduce_trials(A, A, A, 100, 8, 1, 1, A, A, A, 8, None) == 9
+    assert lib.dc_argmax_tau(A, A, 4, 1, A, A, A, None) == 7      # done_frac is not an objective
+    assert lib.dc_argmax_tau(A, A, 0, 4, A, A, A, None) == 2
+    assert lib.dc_simulate_plan(A, 4, 8, 12, 3) == 0
+    assert lib.dc_simulate_plan(A, 4, 8, 13, 3) == 1
+    assert lib.dc_simulate_plan(A + 4, 4, 8, 12, 3) == 1
+    assert lib.dc_simulate_plan(A, 4, 8, 12, 5000) == -4
+
+
+def test_workspace_sizes(lib):
+    from paper_2306_10598_b200 import api
+    assert api.dc_reduce_workspace_bytes(0, 4) == 0
+    for T, K in ((1, 1), (31, 7), (33, 16), (32768, 256), (5000, 4096)):
+        b = api.dc_reduce_workspace_bytes(T, K)
+        chunks = min(64, -(-T // 32))
+        rows = -(-T // chunks)
+        chunks = -(-T // rows)
+        assert b == 8 * (chunks * 4 * K + chunks)
+    assert api.dc_sweep_host_workspace_bytes(8, 4, 4, 2, 0) == 0
+    assert api.dc_sweep_host_workspace_bytes(1024, 8, 4, 16, 4096) == api.dc_sweep_host_workspace_bytes(1024, 8, 4, 16, 1024)
+    assert api.status_string(0) == "ok" and "NULL" in api.status_string(1)

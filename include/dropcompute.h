@@ -182,6 +182,17 @@ int dc_device_status(uint32_t *flags_host);
  * kernel (M not a multiple of 4, or a pointer only 4-byte aligned), negative = -dc_status. */
 int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K);
 
+/*
+ * dc_tune — expert knob for performance experiments; affects later dc_simulate* calls of this process.
+ * Results never depend on it.  value 0 restores the automatic choice.
+ *   DC_TUNE_STAGES       depth of the shared-memory ring the tiled kernel streams rows through (2..8)
+ *   DC_TUNE_LANE_COPIES  histogram copies per warp in the tiled kernel (1, 2 or 4)
+ * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
+ */
+#define DC_TUNE_STAGES 1
+#define DC_TUNE_LANE_COPIES 2
+int dc_tune(int32_t key, int32_t value);
+
 /* Number of kernel launches the last successful call of each entry point enqueues (for accounting). */
 int dc_simulate_launches(void);
 int dc_reduce_trials_launches(void);

@@ -26,7 +26,7 @@ STAT_NAMES = ("mean_step", "done_frac", "thr", "thr_mean", "s_eff")
 EXPORTS = (
     "dc_simulate", "dc_simulate_ex", "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_argmax_tau",
     "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan",
-    "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string",
+    "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string", "dc_tune",
 )
 
 
@@ -56,6 +56,8 @@ _lib.dc_sweep_host.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _i32, _i32,
 _lib.dc_check_inputs.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _p, _p, _p]
 _lib.dc_device_status.argtypes = [_p]
 _lib.dc_simulate_plan.argtypes = [_p, _i64, _i64, _i64, _i32]
+_lib.dc_tune.argtypes = [_i32, _i32]
+_lib.dc_tune.restype = ctypes.c_int
 _lib.dc_status_string.argtypes = [ctypes.c_int]
 _lib.dc_status_string.restype = ctypes.c_char_p
 for _name in ("dc_simulate", "dc_simulate_ex", "dc_reduce_trials", "dc_argmax_tau", "dc_sweep_host", "dc_check_inputs",
@@ -197,6 +199,13 @@ def dc_sweep_host(latencies_host: torch.Tensor, taus_host: torch.Tensor, t_comm:
                                   workspace.numel() * workspace.element_size(),
                                   torch.cuda.current_stream(workspace.device).cuda_stream), "dc_sweep_host")
     return HostSweep(stats, base, int(k_star.value), float(tau_star.value))
+
+
+TUNE_STAGES, TUNE_LANE_COPIES = 1, 2
+
+
+def dc_tune(key: int, value: int) -> None:
+    _check(_lib.dc_tune(int(key), int(value)), "dc_tune")
 
 
 def launches() -> dict:

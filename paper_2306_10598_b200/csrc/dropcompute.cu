@@ -46,6 +46,7 @@ constexpr int kHistBudgetBytes = 32 * 1024;   // shared memory spent on per-warp
 constexpr uint32_t kWaitLimit = 1u << 22;     // polls of one mbarrier wait before giving up (roughly a second)
 constexpr int kReduceChunksMax = 64;          // partial sums per threshold in dc_reduce_trials
 constexpr int kConsumerBarrier = 1;           // named barrier used by the consumer warps
+constexpr int kLutCellsMax = 4096;            // cells of the bin lookup table (4 per threshold up to this)
 
 constexpr uint32_t kErrLoadNeverArrived = 1u;
 constexpr uint32_t kErrStageNeverFreed = 2u;
@@ -70,8 +71,10 @@ struct SweepParams {
     int swz_mask;      // 7 / 3 / 1 / 0 for the 128 / 64 / 32-byte swizzle / none
     int stages;
     int stage_bytes;   // multiple of 1024
-    int hist_copies;   // per-warp histogram copies (power of two)
+    int hist_copies;   // histogram copies in shared memory
     int hist_stride;   // ints per copy (>= K + 1)
+    int lane_copies;   // tiled kernel: copies per warp (lane l uses copy l % lane_copies); power of two
+    int lut_cells;     // tiled kernel: cells of the bin lookup table (the table has lut_cells + 1 entries)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -233,6 +236,8 @@ struct SmemTail {
     int *hist;
     float *smax;
     int *wtot;
+    int *meta;           // [0] lookup table has at most one finite threshold per cell, [1..2] lo, scale (as bits)
+    unsigned short *lut; // lut_cells + 1 entries (tiled kernel only)
 };
 __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepParams &p)
 {
@@ -241,11 +246,14 @@ __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepP
     s.hist = reinterpret_cast<int *>(s.tau_s + (p.K + 1));
     s.smax = reinterpret_cast<float *>(s.hist + p.hist_copies * p.hist_stride);
     s.wtot = reinterpret_cast<int *>(s.smax + 32);
+    s.meta = s.wtot + 32;
+    s.lut = reinterpret_cast<unsigned short *>(s.meta + 8);
     return s;
 }
-__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride)
+__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride, int lut_cells)
 {
-    return sizeof(float) * (size_t)(K + 1) + sizeof(int) * (size_t)hist_copies * hist_stride + 64 * sizeof(int);
+    return sizeof(float) * (size_t)(K + 1) + sizeof(int) * (size_t)hist_copies * hist_stride + 72 * sizeof(int) +
+           (((size_t)(lut_cells + 1) * sizeof(unsigned short) + 3) & ~(size_t)3);
 }
 
 __device__ __forceinline__ void load_thresholds(const SweepParams &p, const SmemTail &s, int tid, int nthr)
@@ -256,11 +264,85 @@ __device__ __forceinline__ void load_thresholds(const SweepParams &p, const Smem
 }
 
 // ------------------------------------------------------------------------------------------
+// Bin lookup for the tiled kernel.  A running sum P falls into bin j(P) = #{k : tau_k <= P}.
+// The range [lo, hi] of the finite thresholds is cut into C equal cells; cell(x) is a monotone
+// function of x evaluated with the SAME two fp32 operations for thresholds and samples, so
+//   lut[c] = #{k : tau_k = -inf or cell(tau_k) < c}  <=  j(P)  for every P with cell(P) = c,
+// and j(P) is reached from lut[c] by comparing P with the real thresholds (one compare when no
+// cell holds two finite thresholds, which is the case for evenly spaced grids).  The table only
+// proposes where to start; the comparisons with tau_k decide, so the bins are exact.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned lut_cell(float x, float lo, float scale, unsigned C)
+{
+    return min(__float2uint_rz(__fmul_rn(__fsub_rn(x, lo), scale)), C);  // negative and NaN -> 0, huge -> C
+}
+
+// All threads of the block; tau_s[0..K] is loaded (tau_s[K] = +inf).  Ends with __syncthreads().
+__device__ __forceinline__ void build_lut(const SweepParams &p, const SmemTail &s, int tid, int nthr)
+{
+    const int K = p.K;
+    const unsigned C = (unsigned)p.lut_cells;
+    const float ninf = __int_as_float(0xff800000), pinf = __int_as_float(0x7f800000);
+    if (tid == 0) {
+        int klo = 0, khi = K - 1;
+        while (klo < K && !(s.tau_s[klo] > ninf)) ++klo;
+        while (khi >= 0 && !(s.tau_s[khi] < pinf)) --khi;
+        float lo = 0.0f, scale = 0.0f;
+        if (klo <= khi) {
+            lo = s.tau_s[klo];
+            const float range = __fsub_rn(s.tau_s[khi], lo);
+            if (range > 0.0f && range < pinf) scale = __fdiv_rn((float)C, range);
+            if (!(scale < pinf)) scale = 0.0f;
+        }
+        s.meta[0] = 1;
+        s.meta[1] = __float_as_int(lo);
+        s.meta[2] = __float_as_int(scale);
+    }
+    for (unsigned c = tid; c <= C; c += nthr) s.lut[c] = 0;
+    __syncthreads();
+    const float lo = __int_as_float(s.meta[1]), scale = __int_as_float(s.meta[2]);
+    // extended cell of threshold k: -1 for -inf, C+1 for +inf / NaN / the virtual entry k = K
+    auto cx = [&](int k) -> int {
+        if (k >= K) return (int)C + 1;
+        const float x = s.tau_s[k];
+        if (x == ninf) return -1;
+        if (!(x < pinf)) return (int)C + 1;
+        return (int)lut_cell(x, lo, scale, C);
+    };
+    for (int k = tid; k <= K; k += nthr) {
+        const int prev = (k == 0) ? -1 : cx(k - 1);
+        const int cur = cx(k);
+        const int last = min(cur, (int)C);
+        for (int c = prev + 1; c <= last; ++c) s.lut[c] = (unsigned short)k;  // smallest k with cx(k) >= c
+        if (k > 0 && k < K && cur == prev && cur >= 0 && cur <= (int)C) s.meta[0] = 0;  // two finite thresholds share a cell
+    }
+    __syncthreads();
+}
+
+// Bins one running sum (tiled kernel).  ONE = the table guarantees at most one threshold to step over.
+template <bool ONE>
+__device__ __forceinline__ void bin_sample(float P, float lo, float scale, unsigned C, const unsigned short *lut,
+                                           const float *tau_s, int K, int *myhist, int &cnt0)
+{
+    int j = lut[lut_cell(P, lo, scale, C)];
+    j += (P >= tau_s[j]) ? 1 : 0;  // tau_s[K] = +inf
+    if (!ONE) {
+        while (j < K && P >= tau_s[j]) ++j;
+    }
+    if ((unsigned)(j - 1) < (unsigned)(K - 1)) atomicAdd(myhist + j, 1);  // bins 1..K-1; bin K is never read
+    cnt0 += (j == 0) ? 1 : 0;                                              // bin 0 is counted in a register
+}
+
+// ------------------------------------------------------------------------------------------
 // Tiled kernel: TMA-staged rows, one producer warp + consumer warps, persistent over trials.
 // NQ = 16-byte quads of a row per chunk held in registers (box width = 4*NQ floats at most).
+// A consumer thread adds its row's samples in order, eight at a time.  If after a group every
+// lane of the warp is still below the first threshold the eight samples are bin 0 (one register
+// add); if before the group every lane is at or above the last threshold they are in the bin
+// nobody reads; otherwise each running sum is binned through the lookup table.
 // ------------------------------------------------------------------------------------------
 template <int NQ>
-__global__ void __launch_bounds__(kMaxRowsPerPass + 32)
+__global__ void __launch_bounds__(kMaxRowsPerPass + 32, 2)
 dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 {
     extern __shared__ unsigned char smem_raw[];
@@ -284,6 +366,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     }
     load_thresholds(p, s, tid, blockDim.x);
     __syncthreads();
+    build_lut(p, s, tid, blockDim.x);
 
     if (warp == ncw) {
         // ---------------- producer: one thread streams this block's tiles through the ring
@@ -305,52 +388,71 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     }
 
     // ---------------- consumers: thread r owns row (pass*rows + r) of the current trial
+    constexpr int GQ = NQ >= 2 ? 2 : 1;  // quads per group
     const int nthr = ncw * 32;
-    int *myhist = s.hist + (warp & (p.hist_copies - 1)) * p.hist_stride;
+    const int K = p.K;
+    int *myhist = s.hist + (warp * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
+    const bool one = s.meta[0] != 0;
+    const float lut_lo = __int_as_float(s.meta[1]), lut_scale = __int_as_float(s.meta[2]);
+    const unsigned C = (unsigned)p.lut_cells;
+    const float tau_first = s.tau_s[0], tau_last = s.tau_s[K - 1];
+    // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
     const uint32_t row_off = (uint32_t)tid * (uint32_t)p.pitch;
+    const uint32_t swz = ((row_off >> 7) & (uint32_t)p.swz_mask) << 4;
     uint32_t i = 0;
     for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
         float rowmax = 0.0f;
+        int cnt0 = 0;
         for (int pass = 0; pass < p.passes; ++pass) {
             const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
-            RowWalk w;
-            w.start(s.tau_s);
+            float P = 0.0f;
             for (int c = 0; c < p.chunks; ++c, ++i) {
                 const int st = i % S;
                 mbar_wait(&full[st], (i / S) & 1u, kErrLoadNeverArrived);
-                const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes;
+                const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes + row_off;
                 const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
                 float4 v[NQ];
-                if (valid) {
 #pragma unroll
-                    for (int q = 0; q < NQ; ++q) {
-                        if (q < nq) {
-                            uint32_t off = row_off + q * 16;
-                            off ^= ((off >> 7) & (uint32_t)p.swz_mask) << 4;
-                            v[q] = *reinterpret_cast<const float4 *>(stage + off);
-                        }
-                    }
+                for (int q = 0; q < NQ; ++q) {
+                    v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    if (valid && q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[st]);  // this warp holds its part of the stage in registers
-                if (valid) {
-                    const int m0 = c * p.bw;
 #pragma unroll
-                    for (int q = 0; q < NQ; ++q) {
-                        if (q < nq) {
-                            w.step(v[q].x, m0 + 4 * q + 0, s.tau_s, myhist, p.K);
-                            w.step(v[q].y, m0 + 4 * q + 1, s.tau_s, myhist, p.K);
-                            w.step(v[q].z, m0 + 4 * q + 2, s.tau_s, myhist, p.K);
-                            w.step(v[q].w, m0 + 4 * q + 3, s.tau_s, myhist, p.K);
+                for (int g = 0; g < NQ; g += GQ) {
+                    const int gq = min(GQ, nq - g);  // quads of this group that exist (same for all threads)
+                    if (gq > 0) {
+                        float pv[4 * GQ];
+#pragma unroll
+                        for (int q = 0; q < GQ; ++q) {
+                            // a missing quad holds zeros: P stays put and its entries are never binned
+                            P = __fadd_rn(P, v[g + q].x); pv[4 * q + 0] = P;
+                            P = __fadd_rn(P, v[g + q].y); pv[4 * q + 1] = P;
+                            P = __fadd_rn(P, v[g + q].z); pv[4 * q + 2] = P;
+                            P = __fadd_rn(P, v[g + q].w); pv[4 * q + 3] = P;
+                        }
+                        if (__all_sync(0xffffffffu, !valid || P < tau_first)) {
+                            if (valid) cnt0 += 4 * gq;
+                        } else if (!__all_sync(0xffffffffu, !valid || pv[0] >= tau_last)) {
+                            if (valid) {
+                                if (one) {
+#pragma unroll
+                                    for (int e = 0; e < 4 * GQ; ++e)
+                                        if (e < 4 * gq) bin_sample<true>(pv[e], lut_lo, lut_scale, C, s.lut, s.tau_s, K, myhist, cnt0);
+                                } else {
+#pragma unroll
+                                    for (int e = 0; e < 4 * GQ; ++e)
+                                        if (e < 4 * gq) bin_sample<false>(pv[e], lut_lo, lut_scale, C, s.lut, s.tau_s, K, myhist, cnt0);
+                                }
+                            }
                         }
                     }
                 }
             }
-            if (valid) {
-                w.finish(p.M, myhist);
-                rowmax = fmaxf(rowmax, w.P);
-            }
+            if (valid) rowmax = fmaxf(rowmax, P);
         }
+        if (cnt0 > 0) atomicAdd(myhist, cnt0);
         trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot);
     }
 }
@@ -568,6 +670,7 @@ EncodeTiledFn get_encode_fn()
 struct DeviceInfo {
     int sms = 0;
     int max_smem_optin = 0;
+    int smem_per_sm = 0;
 };
 bool device_info(DeviceInfo *out)
 {
@@ -578,6 +681,9 @@ bool device_info(DeviceInfo *out)
         int sms = 0, smem = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
         if (cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return false;
+        int per_sm = 0;
+        if (cudaDeviceGetAttribute(&per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) != cudaSuccess) return false;
+        cache[dev].smem_per_sm = per_sm;
         cache[dev].max_smem_optin = smem;
         cache[dev].sms = sms;
     }
@@ -592,6 +698,8 @@ int floor_pow2(int v)
     return p;
 }
 
+int g_tune_stages = 0;       // 0 = automatic
+int g_tune_lane_copies = 0;  // 0 = automatic
 int g_last_simulate_launches = 0;
 int g_last_reduce_launches = 0;
 int g_last_argmax_launches = 0;
@@ -652,7 +760,8 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     const int row_threads = ((p.rows + 31) / 32) * 32;
     p.hist_stride = K + 1;
     p.hist_copies = floor_pow2(min(row_threads / 32, max(1, kHistBudgetBytes / (int)(sizeof(int) * p.hist_stride))));
-    const size_t tail = tail_bytes(K, p.hist_copies, p.hist_stride);
+    p.lane_copies = 1;
+    p.lut_cells = 0;
 
     if (tiled_ok(lat, M)) {
         EncodeTiledFn encode = get_encode_fn();
@@ -668,7 +777,33 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         else if (p.pitch == 64) { swz = CU_TENSOR_MAP_SWIZZLE_64B; p.swz_mask = 3; }
         else if (p.pitch == 32) { swz = CU_TENSOR_MAP_SWIZZLE_32B; p.swz_mask = 1; }
         p.stage_bytes = ((p.rows * p.pitch + 1023) / 1024) * 1024;
-        p.stages = max(2, min(kMaxStages, kStageBudgetBytes / p.stage_bytes));
+        p.lut_cells = min(kLutCellsMax, 4 * K);
+        // Shared memory per block: aim at two resident blocks per SM.  Prefer more histogram copies per
+        // warp (fewer same-address conflicts between lanes), then more stages.
+        const int ncw = row_threads / 32;
+        const size_t budget = (size_t)di.smem_per_sm / 2 - 1024 - 256;
+        size_t smem = 0;
+        bool fits = false;
+        const int lc_first = g_tune_lane_copies > 0 ? g_tune_lane_copies : 4;
+        for (int lc = lc_first; lc >= 1 && !fits; lc >>= 1) {
+            p.lane_copies = lc;
+            p.hist_copies = ncw * lc;
+            const int want = lc > 1 ? 32 / lc : 1;  // copies of one warp start in different banks
+            p.hist_stride = K + 1;
+            while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
+            const size_t fixed = 1024 + 2 * kMaxStages * sizeof(uint64_t) + tail_bytes(K, p.hist_copies, p.hist_stride, p.lut_cells);
+            const int s_max = g_tune_stages > 0 ? g_tune_stages : min(kMaxStages, max(2, kStageBudgetBytes / p.stage_bytes));
+            for (int st = s_max; st >= 2; --st) {
+                smem = fixed + (size_t)st * p.stage_bytes;
+                if (smem <= budget || (lc == 1 && st == 2) || g_tune_stages > 0) {
+                    p.stages = st;
+                    fits = true;
+                    break;
+                }
+            }
+            if (g_tune_lane_copies > 0) break;
+        }
+        if (!fits) return DC_ERR_RANGE;
 
         CUtensorMap map;
         const cuuint64_t gdim[3] = {(cuuint64_t)M, (cuuint64_t)N, (cuuint64_t)T};
@@ -680,7 +815,6 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return DC_ERR_CUDA;
 
-        const size_t smem = 1024 + (size_t)p.stages * p.stage_bytes + 2 * kMaxStages * sizeof(uint64_t) + tail;
         if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
         const int block = row_threads + 32;
         const int nq = p.bw / 4;
@@ -696,7 +830,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     // plain-load kernel
     p.rows = row_threads;  // one row per thread per pass
     p.passes = (int)((N + p.rows - 1) / p.rows);
-    const size_t smem = tail;
+    const size_t smem = tail_bytes(K, p.hist_copies, p.hist_stride, 0);
     if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
     if (cudaFuncSetAttribute(dc_sweep_plain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return DC_ERR_CUDA;
@@ -946,6 +1080,19 @@ int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M, 
     if (cuda_fail) return DC_ERR_CUDA;
     if (rc == DC_OK) g_last_simulate_launches = launches;
     return rc;
+}
+
+int dc_tune(int32_t key, int32_t value)
+{
+    if (key == DC_TUNE_STAGES && (value == 0 || (value >= 2 && value <= kMaxStages))) {
+        g_tune_stages = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_LANE_COPIES && (value == 0 || value == 1 || value == 2 || value == 4)) {
+        g_tune_lane_copies = value;
+        return DC_OK;
+    }
+    return DC_ERR_UNSUPPORTED;
 }
 
 int dc_simulate_launches(void) { return g_last_simulate_launches; }

@@ -225,7 +225,10 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
         done_row[b] = run;
         step_row[b] = __fadd_rn(fminf(tau_s[b], Tmax), p.t_comm);
     }
-    if (tid < H) hist[tid * HS + K] = 0;  // the bin of samples at or above the last threshold
+    for (int c = tid; c < H; c += nthr) {  // the bins of samples at or above the last threshold
+        hist[c * HS + K] = 0;
+        if (HS > K + 1) hist[c * HS + K + 1] = 0;
+    }
     if (tid == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, p.t_comm);
     named_barrier(barrier_id, nthr);  // histograms cleared, smax/wtot free again
 }
@@ -313,24 +316,26 @@ __device__ __forceinline__ void build_lut(const SweepParams &p, const SmemTail &
         const int prev = (k == 0) ? -1 : cx(k - 1);
         const int cur = cx(k);
         const int last = min(cur, (int)C);
-        for (int c = prev + 1; c <= last; ++c) s.lut[c] = (unsigned short)k;  // smallest k with cx(k) >= c
+        for (int c = prev + 1; c <= last; ++c) s.lut[c] = (unsigned short)(4 * k);  // byte offset of the smallest k with cx(k) >= c
         if (k > 0 && k < K && cur == prev && cur >= 0 && cur <= (int)C) s.meta[0] = 0;  // two finite thresholds share a cell
     }
     __syncthreads();
 }
 
-// Bins one running sum (tiled kernel).  ONE = the table guarantees at most one threshold to step over.
+// Bins one running sum (tiled kernel): adds 1 to bin j(P) of this thread's histogram copy.  The table
+// entry and `off` are BYTE offsets (4 j) into the threshold array and the histogram.  Bins 0..K+1 exist
+// (K: at or above the last threshold, K+1: only reachable by P = +inf); the epilogue reads 0..K-1.
+// ONE = the table guarantees at most one threshold to step over.
 template <bool ONE>
 __device__ __forceinline__ void bin_sample(float P, float lo, float scale, unsigned C, const unsigned short *lut,
-                                           const float *tau_s, int K, int *myhist, int &cnt0)
+                                           const unsigned char *tau_b, unsigned K4, unsigned char *hist_b)
 {
-    int j = lut[lut_cell(P, lo, scale, C)];
-    j += (P >= tau_s[j]) ? 1 : 0;  // tau_s[K] = +inf
+    unsigned off = lut[lut_cell(P, lo, scale, C)];
+    off += (P >= *reinterpret_cast<const float *>(tau_b + off)) ? 4u : 0u;  // tau_s[K] = +inf
     if (!ONE) {
-        while (j < K && P >= tau_s[j]) ++j;
+        while (off < K4 && P >= *reinterpret_cast<const float *>(tau_b + off)) off += 4u;
     }
-    if ((unsigned)(j - 1) < (unsigned)(K - 1)) atomicAdd(myhist + j, 1);  // bins 1..K-1; bin K is never read
-    cnt0 += (j == 0) ? 1 : 0;                                              // bin 0 is counted in a register
+    atomicAdd(reinterpret_cast<int *>(hist_b + off), 1);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -392,12 +397,16 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     const int nthr = ncw * 32;
     const int K = p.K;
     int *myhist = s.hist + (warp * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
+    unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
+    const unsigned char *tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
+    const unsigned K4 = 4u * (unsigned)K;
     const bool one = s.meta[0] != 0;
     const float lut_lo = __int_as_float(s.meta[1]), lut_scale = __int_as_float(s.meta[2]);
     const unsigned C = (unsigned)p.lut_cells;
     const float tau_first = s.tau_s[0], tau_last = s.tau_s[K - 1];
     // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
-    const uint32_t row_off = (uint32_t)tid * (uint32_t)p.pitch;
+    // (threads past the last row of the box read the last row instead: always inside the stage)
+    const uint32_t row_off = (uint32_t)min(tid, p.rows - 1) * (uint32_t)p.pitch;
     const uint32_t swz = ((row_off >> 7) & (uint32_t)p.swz_mask) << 4;
     uint32_t i = 0;
     for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
@@ -414,8 +423,8 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                 float4 v[NQ];
 #pragma unroll
                 for (int q = 0; q < NQ; ++q) {
-                    v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    if (valid && q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
+                    if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
+                    else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[st]);  // this warp holds its part of the stage in registers
@@ -436,14 +445,18 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                             if (valid) cnt0 += 4 * gq;
                         } else if (!__all_sync(0xffffffffu, !valid || pv[0] >= tau_last)) {
                             if (valid) {
-                                if (one) {
+                                if (one && gq == GQ) {  // the common case, no per-sample predicates
 #pragma unroll
                                     for (int e = 0; e < 4 * GQ; ++e)
-                                        if (e < 4 * gq) bin_sample<true>(pv[e], lut_lo, lut_scale, C, s.lut, s.tau_s, K, myhist, cnt0);
+                                        bin_sample<true>(pv[e], lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                } else if (one) {
+#pragma unroll
+                                    for (int e = 0; e < 4 * GQ; ++e)
+                                        if (e < 4 * gq) bin_sample<true>(pv[e], lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
                                 } else {
 #pragma unroll
                                     for (int e = 0; e < 4 * GQ; ++e)
-                                        if (e < 4 * gq) bin_sample<false>(pv[e], lut_lo, lut_scale, C, s.lut, s.tau_s, K, myhist, cnt0);
+                                        if (e < 4 * gq) bin_sample<false>(pv[e], lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
                                 }
                             }
                         }
@@ -789,7 +802,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
             p.lane_copies = lc;
             p.hist_copies = ncw * lc;
             const int want = lc > 1 ? 32 / lc : 1;  // copies of one warp start in different banks
-            p.hist_stride = K + 1;
+            p.hist_stride = K + 2;
             while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
             const size_t fixed = 1024 + 2 * kMaxStages * sizeof(uint64_t) + tail_bytes(K, p.hist_copies, p.hist_stride, p.lut_cells);
             const int s_max = g_tune_stages > 0 ? g_tune_stages : min(kMaxStages, max(2, kStageBudgetBytes / p.stage_bytes));

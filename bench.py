@@ -108,8 +108,9 @@ class ClockSampler:
 def cpu_baseline(w: W.Workload, lat_dev, taus: np.ndarray, budget_s: float = 15.0):
     """Times the CPU oracle (as it stands) on a bounded sample of whole trials of the same workload."""
     import oracle
-    probe = min(w.T, 4)
+    probe = min(w.T, 16)
     lat = lat_dev[:probe].cpu().numpy()
+    oracle.sweep(lat[:1], taus, w.t_comm)  # loads the library and starts the thread pool
     t = time.perf_counter()
     oracle.sweep(lat, taus, w.t_comm)
     dt = max(time.perf_counter() - t, 1e-4)
@@ -135,8 +136,9 @@ def run_reference(args, w: W.Workload):
     import oracle
     taus = W.make_taus(w)
     # size the per-step sample so that (steps + warmup) steps take about a minute in total
-    probe = min(w.T, 2)
+    probe = min(w.T, 16)
     lat = W.fill_latencies(w, "cpu", t0=0, t1=probe).numpy()
+    oracle.sweep(lat[:1], taus, w.t_comm)  # loads the library and starts the thread pool
     t = time.perf_counter()
     oracle.sweep(lat, taus, w.t_comm)
     per_trial = max(time.perf_counter() - t, 1e-4) / probe

@@ -173,6 +173,20 @@ def run_reference(args, w: W.Workload):
     return 0
 
 
+def read_traffic(workload: str, kernel_version: str):
+    """DRAM bytes per sweep launch from the ncu capture filed in profiles/traffic.txt, or None when there is
+    no capture of this workload taken on the kernel version the library reports."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.txt")) as f:
+            for ln in f:
+                parts = ln.split()
+                if len(parts) == 3 and not ln.startswith("#") and parts[0] == workload and parts[1] == kernel_version:
+                    return int(parts[2])
+    except (OSError, ValueError):
+        pass
+    return None
+
+
 def physical_gpu_index(local_rank: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
     parts = [x.strip() for x in vis.split(",") if x.strip()]
@@ -278,17 +292,7 @@ def run_ours(args, w: W.Workload):
     alg_bytes = 4 * samples + 8 * T * K + 4 * T
     peak, peak_kind = measured_hbm_peak()
     achieved = alg_bytes / sim_avg_s / 1e9
-    traffic = None  # dram bytes per launch from ncu; see profiles/ (null until captured for this kernel version)
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        try:
-            with open(tpath) as f:
-                tj = json.load(f)
-            ent = tj.get(w.name)
-            if ent and ent.get("kernel_version") == tj.get("current_kernel_version"):
-                traffic = ent.get("dram_bytes_per_launch")
-        except Exception:
-            traffic = None
+    traffic = read_traffic(w.name, api.dc_kernel_version()) if not args.trials else None
 
     line = {
         "metric": METRIC, "value": value_sps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,

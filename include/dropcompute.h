@@ -200,6 +200,9 @@ int dc_argmax_tau_launches(void);
 
 const char *dc_status_string(int status);
 
+/* A short tag that changes whenever the sweep kernels change (profiles are filed under it). */
+const char *dc_kernel_version(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,6 +27,7 @@ EXPORTS = (
     "dc_simulate", "dc_simulate_ex", "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_argmax_tau",
     "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan",
     "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string", "dc_tune",
+    "dc_kernel_version",
 )
 
 
@@ -60,10 +61,16 @@ _lib.dc_tune.argtypes = [_i32, _i32]
 _lib.dc_tune.restype = ctypes.c_int
 _lib.dc_status_string.argtypes = [ctypes.c_int]
 _lib.dc_status_string.restype = ctypes.c_char_p
+_lib.dc_kernel_version.argtypes = []
+_lib.dc_kernel_version.restype = ctypes.c_char_p
 for _name in ("dc_simulate", "dc_simulate_ex", "dc_reduce_trials", "dc_argmax_tau", "dc_sweep_host", "dc_check_inputs",
               "dc_device_status", "dc_simulate_plan", "dc_simulate_launches", "dc_reduce_trials_launches",
               "dc_argmax_tau_launches"):
     getattr(_lib, _name).restype = ctypes.c_int
+
+
+def dc_kernel_version() -> str:
+    return _lib.dc_kernel_version().decode()
 
 
 def status_string(status: int) -> str:

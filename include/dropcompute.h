@@ -127,6 +127,34 @@ int dc_reduce_trials(const float *out_step, const int32_t *out_done, const float
                      void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * dc_reduce_trials_static — the same statistics as dc_reduce_trials, for a caller that cannot hand over a
+ * workspace.  (The paper has no counterpart to this entry point; it exists for deployment only.)
+ *
+ * Who needs it: code that runs where device memory may not be requested any more — a plug-in inside a
+ * serving or training process whose memory pool already owns the whole GPU (a fresh cudaMalloc there fails
+ * or forces the pool to shrink), or a latency-critical loop in which an allocation would stall the device.
+ * Such a caller still owns its inputs and outputs, but has nowhere to put the partial sums of the two-phase
+ * reduction.  Here they live in an array that is part of the library image: DC_STATIC_SCRATCH_BYTES bytes of
+ * device memory that every GPU holds from the moment it loads this library until the process ends.
+ *
+ * Same arguments, results and error codes as dc_reduce_trials without the workspace pair, plus:
+ *   K <= DC_STATIC_MAX_K, otherwise DC_ERR_RANGE (the array is sized for that many thresholds; use
+ *   dc_reduce_trials with your own workspace beyond it).  T is not limited.
+ * The call allocates and frees nothing, neither directly nor through a library routine.
+ * The first call on each device looks up the array's device address (one runtime query, cached); make that
+ * first call outside any stream capture.
+ * All calls on a device share the one array.  Nothing in it has to be cleared between calls — each call
+ * overwrites every partial sum before reading it, so what an earlier call left behind is never seen — but
+ * two calls that may run at the same time on one device (different streams) would overwrite each other's
+ * partial sums: serialise them, or give the concurrent ones a workspace through dc_reduce_trials.
+ */
+#define DC_STATIC_MAX_K 1024
+#define DC_STATIC_SCRATCH_BYTES (64 * (4 * DC_STATIC_MAX_K + 1) * 8) /* 2 097 664 bytes per GPU */
+int dc_reduce_trials_static(const float *out_step, const int32_t *out_done, const float *out_sync,
+                            int64_t T, int32_t K, int64_t N, int64_t M,
+                            double *stats, double *baseline, void *stream);
+
+/*
  * dc_argmax_tau — tau* = argmax_tau objective(tau) (last line of Algorithm 2).
  *
  *   stats      DEVICE, [DC_NSTATS][K] from dc_reduce_trials      taus  DEVICE [K]

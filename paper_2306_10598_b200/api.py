@@ -24,7 +24,8 @@ NSTATS = 5
 STAT_NAMES = ("mean_step", "done_frac", "thr", "thr_mean", "s_eff")
 
 EXPORTS = (
-    "dc_simulate", "dc_simulate_ex", "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_argmax_tau",
+    "dc_simulate", "dc_simulate_ex", "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_reduce_trials_static",
+    "dc_argmax_tau",
     "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan",
     "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string", "dc_tune",
     "dc_kernel_version",
@@ -50,6 +51,8 @@ _lib.dc_simulate_ex.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _p, _p, _p
 _lib.dc_reduce_workspace_bytes.argtypes = [_i64, _i32]
 _lib.dc_reduce_workspace_bytes.restype = _sz
 _lib.dc_reduce_trials.argtypes = [_p, _p, _p, _i64, _i32, _i64, _i64, _p, _p, _p, _sz, _p]
+_lib.dc_reduce_trials_static.argtypes = [_p, _p, _p, _i64, _i32, _i64, _i64, _p, _p, _p]
+_lib.dc_reduce_trials_static.restype = ctypes.c_int
 _lib.dc_argmax_tau.argtypes = [_p, _p, _i32, _i32, _p, _p, _p, _p]
 _lib.dc_sweep_host_workspace_bytes.argtypes = [_i64, _i64, _i64, _i32, _i64]
 _lib.dc_sweep_host_workspace_bytes.restype = _sz
@@ -141,6 +144,25 @@ def dc_reduce_trials(out_step: torch.Tensor, out_done: torch.Tensor, out_sync: O
                                      T, K, int(N), int(M), _dev(stats, torch.float64, "stats"),
                                      _dev(baseline, torch.float64, "baseline"), workspace.data_ptr(),
                                      workspace.numel() * workspace.element_size(), _stream(out_step)), "dc_reduce_trials")
+
+
+STATIC_MAX_K = 1024
+
+
+def dc_reduce_trials_static(out_step: torch.Tensor, out_done: torch.Tensor, out_sync: Optional[torch.Tensor], N: int,
+                            M: int, stats: torch.Tensor, baseline: torch.Tensor) -> None:
+    """``dc_reduce_trials_static``: the trial statistics without a workspace argument, for callers that may
+    not allocate device memory (the partial sums go to an array built into the library; K <= STATIC_MAX_K).
+    This wrapper allocates nothing either: it only passes the pointers of the tensors it is given.  Calls on
+    one device share that array, so do not run two of them concurrently on different streams."""
+    T, K = out_step.shape
+    assert tuple(stats.shape) == (NSTATS, K) and tuple(baseline.shape) == (2,)
+    with torch.cuda.device(out_step.device):
+        _check(_lib.dc_reduce_trials_static(_dev(out_step, torch.float32, "out_step"), _dev(out_done, torch.int32, "out_done"),
+                                            None if out_sync is None else _dev(out_sync, torch.float32, "out_sync"),
+                                            T, K, int(N), int(M), _dev(stats, torch.float64, "stats"),
+                                            _dev(baseline, torch.float64, "baseline"), _stream(out_step)),
+               "dc_reduce_trials_static")
 
 
 def dc_argmax_tau(stats: torch.Tensor, taus: torch.Tensor, objective: int, out_k: torch.Tensor, out_tau: torch.Tensor,

@@ -29,6 +29,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>
+#include <mutex>
 #include <stdint.h>
 #include <string.h>
 
@@ -876,6 +877,13 @@ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
+// Partial sums of dc_reduce_trials_static.  Part of the library image: each GPU that loads the library
+// holds these DC_STATIC_SCRATCH_BYTES until the process exits.  In host code this name is only a handle
+// for cudaGetSymbolAddress; kernels are given the address that call returns.
+static __device__ __align__(256) double g_static_reduce_scratch[kReduceChunksMax * (4 * DC_STATIC_MAX_K + 1)];
+static_assert(sizeof(double) * kReduceChunksMax * (4 * DC_STATIC_MAX_K + 1) == DC_STATIC_SCRATCH_BYTES,
+              "header and array disagree about the scratch size");
+
 // ------------------------------------------------------------------------------------------
 // C ABI
 // ------------------------------------------------------------------------------------------
@@ -929,6 +937,39 @@ int dc_reduce_trials(const float *out_step, const int32_t *out_done, const float
     dc_reduce_final<<<(unsigned)((K + 255) / 256), 256, 0, stream>>>(ws, T, K, NM, r.chunks, stats, baseline);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     g_last_reduce_launches = 2;
+    return DC_OK;
+}
+
+int dc_reduce_trials_static(const float *out_step, const int32_t *out_done, const float *out_sync, int64_t T, int32_t K,
+                            int64_t N, int64_t M, double *stats, double *baseline, void *stream_v)
+{
+    if (!out_step || !out_done || !stats || !baseline) return DC_ERR_NULL;
+    if (T <= 0 || K <= 0 || N <= 0 || M <= 0) return DC_ERR_SHAPE;
+    if (K > DC_STATIC_MAX_K || N * M > (int64_t)INT32_MAX) return DC_ERR_RANGE;
+    if ((reinterpret_cast<uintptr_t>(stats) & 7) || (reinterpret_cast<uintptr_t>(baseline) & 7)) return DC_ERR_ALIGN;
+    // Device address of the built-in scratch, looked up once per device with that device current.
+    static std::mutex lock;
+    static double *scratch_of_device[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DC_ERR_CUDA;
+    double *ws = nullptr;
+    {
+        std::lock_guard<std::mutex> guard(lock);
+        if (scratch_of_device[dev] == nullptr) {
+            void *ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_static_reduce_scratch) != cudaSuccess || ptr == nullptr) return DC_ERR_CUDA;
+            scratch_of_device[dev] = static_cast<double *>(ptr);
+        }
+        ws = scratch_of_device[dev];
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const ReducePlan r = reduce_plan(T);  // at most kReduceChunksMax chunks, whatever T is
+    const double NM = (double)N * (double)M;
+    dim3 grid1((unsigned)((K + 31) / 32), (unsigned)r.chunks);
+    dc_reduce_partial<<<grid1, kRedWarps * 32, 0, stream>>>(out_step, out_done, out_sync, T, K, NM, r.chunks, r.rows_per_chunk, ws);
+    if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
+    dc_reduce_final<<<(unsigned)((K + 255) / 256), 256, 0, stream>>>(ws, T, K, NM, r.chunks, stats, baseline);
+    if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     return DC_OK;
 }
 

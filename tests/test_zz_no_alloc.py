@@ -1,0 +1,76 @@
+"""dc_reduce_trials_static, the entry point for callers that may not allocate device memory.
+
+Some users of this library run inside a process whose memory pool already owns the GPU, or in a loop
+that must never stall on an allocation; they cannot supply the workspace dc_reduce_trials asks for.
+This file checks, through the C ABI, that the workspace-free entry point gives what dc_reduce_trials
+gives, on two calls in a row with different inputs (the built-in scratch keeps the first call's
+contents, which must not leak into the second), and that it refuses a grid larger than the scratch was
+sized for.  It is collected last on purpose, and passes both alone and after the other tests."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2306_10598_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+RTOL_STATS = 1e-9  # the tolerance the parity tests use for fp64 statistics
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2306_10598_b200 import api as _api
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    return _api
+
+
+def _sweep_outputs(api, T, N, M, K, seed):
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=seed, shift=0.01, mean=0.02).cuda()
+    hi = float(lat.sum(-1).max())
+    taus = torch.linspace(0.3 * hi, 1.1 * hi, K, device="cuda")
+    step = torch.empty((T, K), dtype=torch.float32, device="cuda")
+    done = torch.empty((T, K), dtype=torch.int32, device="cuda")
+    sync = torch.empty((T,), dtype=torch.float32, device="cuda")
+    api.dc_simulate_ex(lat, taus, 0.05, step, done, sync)
+    return step, done, sync
+
+
+def test_static_reduce_matches_workspace_reduce_twice(api):
+    # second call: fewer trials and thresholds than the first, so stale partial sums lie beyond what it writes
+    for call, (T, N, M, K) in enumerate(((700, 40, 16, 96), (45, 9, 8, 7))):
+        step, done, sync = _sweep_outputs(api, T, N, M, K, seed=50 + call)
+        want = torch.empty((api.NSTATS, K), dtype=torch.float64, device="cuda")
+        want_base = torch.empty(2, dtype=torch.float64, device="cuda")
+        ws = torch.empty(api.dc_reduce_workspace_bytes(T, K), dtype=torch.uint8, device="cuda")
+        api.dc_reduce_trials(step, done, sync, N, M, want, want_base, ws)
+        got = torch.full_like(want, float("nan"))
+        got_base = torch.full_like(want_base, float("nan"))
+        torch.cuda.synchronize()
+        api.dc_reduce_trials_static(step, done, sync, N, M, got, got_base)   # outputs exist already: no allocation here
+        torch.cuda.synchronize()
+        assert np.allclose(got.cpu().numpy(), want.cpu().numpy(), rtol=RTOL_STATS, atol=0), f"call {call}"
+        assert np.allclose(got_base.cpu().numpy(), want_base.cpu().numpy(), rtol=RTOL_STATS, atol=0), f"call {call}"
+        # without the synchronous baseline: NaN in the same places as dc_reduce_trials
+        api.dc_reduce_trials(step, done, None, N, M, want, want_base, ws)
+        api.dc_reduce_trials_static(step, done, None, N, M, got, got_base)
+        torch.cuda.synchronize()
+        assert np.allclose(got.cpu().numpy(), want.cpu().numpy(), rtol=RTOL_STATS, atol=0, equal_nan=True)
+        assert torch.isnan(got_base).all()
+
+
+def test_static_reduce_refuses_grids_beyond_its_scratch(api):
+    T, K = 4, api.STATIC_MAX_K + 1
+    step = torch.ones((T, K), dtype=torch.float32, device="cuda")
+    done = torch.ones((T, K), dtype=torch.int32, device="cuda")
+    stats = torch.empty((api.NSTATS, K), dtype=torch.float64, device="cuda")
+    base = torch.empty(2, dtype=torch.float64, device="cuda")
+    with pytest.raises(api.DropComputeError) as e:
+        api.dc_reduce_trials_static(step, done, None, 2, 2, stats, base)
+    assert e.value.status == 4  # DC_ERR_RANGE
+    # the largest supported grid is accepted
+    K = api.STATIC_MAX_K
+    step, done = step[:, :K].contiguous(), done[:, :K].contiguous()
+    stats = torch.empty((api.NSTATS, K), dtype=torch.float64, device="cuda")
+    api.dc_reduce_trials_static(step, done, None, 2, 2, stats, base)
+    torch.cuda.synchronize()
+    assert torch.allclose(stats[api.STAT_MEAN_STEP], torch.ones(K, dtype=torch.float64, device="cuda"))

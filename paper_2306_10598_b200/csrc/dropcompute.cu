@@ -76,6 +76,7 @@ struct SweepParams {
     int hist_stride;   // ints per copy (>= K + 1)
     int lane_copies;   // tiled kernel: copies per warp (lane l uses copy l % lane_copies); power of two
     int lut_cells;     // tiled kernel: cells of the bin lookup table (the table has lut_cells + 1 entries)
+    int one;           // always 1; a value the compiler cannot see, used to tie a stage release to a warp vote
 };
 
 // ------------------------------------------------------------------------------------------
@@ -94,6 +95,10 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_count(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
@@ -427,37 +432,59 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                     if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
                     else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[st]);  // this warp holds its part of the stage in registers
+                // Running sums of the whole chunk, in place (a missing quad holds zeros: P stays put and its
+                // entries are never binned).
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    P = __fadd_rn(P, v[q].x); v[q].x = P;
+                    P = __fadd_rn(P, v[q].y); v[q].y = P;
+                    P = __fadd_rn(P, v[q].z); v[q].z = P;
+                    P = __fadd_rn(P, v[q].w); v[q].w = P;
+                }
+                // Whole chunk still below the first threshold for every lane of the warp?  The vote needs every
+                // lane's last running sum, i.e. every shared-memory read of the stage by this warp has returned;
+                // the stage is released only after it, and the count operand of the arrive depends on the vote
+                // (p.one is 1), so the release cannot move ahead of the reads.
+                const bool chunk_low = __all_sync(0xffffffffu, !valid || P < tau_first);
+                if (lane == 0) mbar_arrive_count(&empty[st], chunk_low ? 1u : (uint32_t)p.one);
+                if (chunk_low) {
+                    if (valid) cnt0 += 4 * nq;
+                    continue;
+                }
 #pragma unroll
                 for (int g = 0; g < NQ; g += GQ) {
                     const int gq = min(GQ, nq - g);  // quads of this group that exist (same for all threads)
                     if (gq > 0) {
-                        float pv[4 * GQ];
-#pragma unroll
-                        for (int q = 0; q < GQ; ++q) {
-                            // a missing quad holds zeros: P stays put and its entries are never binned
-                            P = __fadd_rn(P, v[g + q].x); pv[4 * q + 0] = P;
-                            P = __fadd_rn(P, v[g + q].y); pv[4 * q + 1] = P;
-                            P = __fadd_rn(P, v[g + q].z); pv[4 * q + 2] = P;
-                            P = __fadd_rn(P, v[g + q].w); pv[4 * q + 3] = P;
-                        }
-                        if (__all_sync(0xffffffffu, !valid || P < tau_first)) {
+                        const float pend = v[g + GQ - 1].w;  // running sum after the group
+                        if (__all_sync(0xffffffffu, !valid || pend < tau_first)) {
                             if (valid) cnt0 += 4 * gq;
-                        } else if (!__all_sync(0xffffffffu, !valid || pv[0] >= tau_last)) {
+                        } else if (!__all_sync(0xffffffffu, !valid || v[g].x >= tau_last)) {
                             if (valid) {
                                 if (one && gq == GQ) {  // the common case, no per-sample predicates
 #pragma unroll
-                                    for (int e = 0; e < 4 * GQ; ++e)
-                                        bin_sample<true>(pv[e], lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                } else if (one) {
-#pragma unroll
-                                    for (int e = 0; e < 4 * GQ; ++e)
-                                        if (e < 4 * gq) bin_sample<true>(pv[e], lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                    for (int q = 0; q < GQ; ++q) {
+                                        bin_sample<true>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                        bin_sample<true>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                        bin_sample<true>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                        bin_sample<true>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                    }
                                 } else {
 #pragma unroll
-                                    for (int e = 0; e < 4 * GQ; ++e)
-                                        if (e < 4 * gq) bin_sample<false>(pv[e], lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                    for (int q = 0; q < GQ; ++q) {
+                                        if (q < gq) {
+                                            if (one) {
+                                                bin_sample<true>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                                bin_sample<true>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                                bin_sample<true>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                                bin_sample<true>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                            } else {
+                                                bin_sample<false>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                                bin_sample<false>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                                bin_sample<false>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                                bin_sample<false>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                            }
+                                        }
+                                    }
                                 }
                             }
                         }
@@ -776,6 +803,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.hist_copies = floor_pow2(min(row_threads / 32, max(1, kHistBudgetBytes / (int)(sizeof(int) * p.hist_stride))));
     p.lane_copies = 1;
     p.lut_cells = 0;
+    p.one = 1;
 
     if (tiled_ok(lat, M)) {
         EncodeTiledFn encode = get_encode_fn();
@@ -1153,7 +1181,7 @@ int dc_simulate_launches(void) { return g_last_simulate_launches; }
 int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
 int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
 
-const char *dc_kernel_version(void) { return "sweep-tiled-3"; }
+const char *dc_kernel_version(void) { return "sweep-tiled-4"; }
 
 const char *dc_status_string(int status)
 {

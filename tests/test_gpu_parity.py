@@ -277,3 +277,36 @@ def test_workload_correlated_sampled(api):
 
 def test_workload_bandwidth_stress_sampled(api):
     _sampled_parity(api, W.WORKLOADS["bandwidth_stress"], 64)
+
+
+def test_results_do_not_depend_on_tuning_or_timing(api):
+    """The ring depth and the number of histogram copies change the timing of the pipeline (how soon a
+    stage is refilled, how long shared-memory atomics queue up) but must never change a bit of the result.
+    Runs the stress shape (where a stage released too early would be overwritten while still being read)
+    several times under every setting."""
+    w = W.WORKLOADS["bandwidth_stress"].with_trials(1536)
+    lat_d = W.fill_latencies(w, "cuda")
+    taus = W.make_taus(w)
+    taus_d = torch.from_numpy(taus).cuda()
+    idx = np.arange(0, w.T, 64)
+    ref = oracle.sweep(lat_d[torch.from_numpy(idx).cuda()].cpu().numpy(), taus, w.t_comm)
+    first = None
+    try:
+        for stages, copies in ((0, 0), (4, 1), (2, 1), (2, 2), (3, 1), (2, 4)):
+            api.dc_tune(api.TUNE_STAGES, stages)
+            api.dc_tune(api.TUNE_LANE_COPIES, copies)
+            for _ in range(4):
+                res = run_gpu(api, lat_d, taus_d, w.t_comm)
+                if first is None:
+                    first = res
+                    assert np.array_equal(res.out_done[idx].cpu().numpy(), ref.done)
+                    assert np.array_equal(res.out_step[idx].cpu().numpy().view(np.uint32), ref.step.view(np.uint32))
+                    assert np.array_equal(res.out_sync[idx].cpu().numpy().view(np.uint32), ref.sync.view(np.uint32))
+                else:
+                    assert torch.equal(res.out_done, first.out_done), (stages, copies)
+                    assert torch.equal(res.out_step, first.out_step), (stages, copies)
+                    assert torch.equal(res.out_sync, first.out_sync), (stages, copies)
+    finally:
+        api.dc_tune(api.TUNE_STAGES, 0)
+        api.dc_tune(api.TUNE_LANE_COPIES, 0)
+    api.dc_device_status()

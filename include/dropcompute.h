@@ -214,11 +214,15 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  * dc_tune — expert knob for performance experiments; affects later dc_simulate* calls of this process.
  * Results never depend on it.  value 0 restores the automatic choice.
  *   DC_TUNE_STAGES       depth of the shared-memory ring the tiled kernel streams rows through (2..8)
- *   DC_TUNE_LANE_COPIES  histogram copies per warp in the tiled kernel (1, 2 or 4)
+ *   DC_TUNE_LANE_COPIES  histogram copies a warp spreads its lanes over in the tiled kernel (1, 2, 4 or 8)
+ *   DC_TUNE_WARP_GROUPS  groups of warps with histogram copies of their own (1..8)
+ *   DC_TUNE_BOX_FLOATS   floats of a row fetched per tile (16 or 32; 16 needs M to be a multiple of 16)
  * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
  */
 #define DC_TUNE_STAGES 1
 #define DC_TUNE_LANE_COPIES 2
+#define DC_TUNE_WARP_GROUPS 3
+#define DC_TUNE_BOX_FLOATS 4
 int dc_tune(int32_t key, int32_t value);
 
 /* Number of kernel launches the last successful call of each entry point enqueues (for accounting). */

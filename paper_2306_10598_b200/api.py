@@ -230,7 +230,7 @@ def dc_sweep_host(latencies_host: torch.Tensor, taus_host: torch.Tensor, t_comm:
     return HostSweep(stats, base, int(k_star.value), float(tau_star.value))
 
 
-TUNE_STAGES, TUNE_LANE_COPIES = 1, 2
+TUNE_STAGES, TUNE_LANE_COPIES, TUNE_WARP_GROUPS, TUNE_BOX_FLOATS = 1, 2, 3, 4
 
 
 def dc_tune(key: int, value: int) -> None:

@@ -75,6 +75,7 @@ struct SweepParams {
     int hist_copies;   // histogram copies in shared memory
     int hist_stride;   // ints per copy (>= K + 1)
     int lane_copies;   // tiled kernel: copies per warp (lane l uses copy l % lane_copies); power of two
+    int warp_groups;   // tiled kernel: warp w uses the copies of group w % warp_groups
     int lut_cells;     // tiled kernel: cells of the bin lookup table (the table has lut_cells + 1 entries)
     int one;           // always 1; a value the compiler cannot see, used to tie a stage release to a warp vote
 };
@@ -91,10 +92,6 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_count(uint64_t *bar, uint32_t count)
 {
@@ -402,7 +399,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     constexpr int GQ = NQ >= 2 ? 2 : 1;  // quads per group
     const int nthr = ncw * 32;
     const int K = p.K;
-    int *myhist = s.hist + (warp * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
+    int *myhist = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
     unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
     const unsigned char *tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
     const unsigned K4 = 4u * (unsigned)K;
@@ -741,6 +738,8 @@ int floor_pow2(int v)
 
 int g_tune_stages = 0;       // 0 = automatic
 int g_tune_lane_copies = 0;  // 0 = automatic
+int g_tune_warp_groups = 0;  // 0 = automatic
+int g_tune_box_floats = 0;   // 0 = automatic
 int g_last_simulate_launches = 0;
 int g_last_reduce_launches = 0;
 int g_last_argmax_launches = 0;
@@ -802,6 +801,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.hist_stride = K + 1;
     p.hist_copies = floor_pow2(min(row_threads / 32, max(1, kHistBudgetBytes / (int)(sizeof(int) * p.hist_stride))));
     p.lane_copies = 1;
+    p.warp_groups = 1;
     p.lut_cells = 0;
     p.one = 1;
 
@@ -809,6 +809,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         EncodeTiledFn encode = get_encode_fn();
         if (!encode) return DC_ERR_CUDA;
         p.bw = (int)(M < 32 ? M : 32);
+        if (g_tune_box_floats == 16 && M % 16 == 0) p.bw = 16;
         p.chunks = (int)((M + p.bw - 1) / p.bw);
         const int last_cols = (int)(M - (int64_t)(p.chunks - 1) * p.bw);
         p.nq_last = last_cols / 4;
@@ -820,8 +821,9 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         else if (p.pitch == 32) { swz = CU_TENSOR_MAP_SWIZZLE_32B; p.swz_mask = 1; }
         p.stage_bytes = ((p.rows * p.pitch + 1023) / 1024) * 1024;
         p.lut_cells = min(kLutCellsMax, 4 * K);
-        // Shared memory per block: aim at two resident blocks per SM.  Prefer more histogram copies per
-        // warp (fewer same-address conflicts between lanes), then more stages.
+        // Shared memory per block: aim at two resident blocks per SM.  Histogram copies: lane l of warp w
+        // adds into copy (w % warp_groups) * lane_copies + (l % lane_copies); copies used by one warp start
+        // 32 / lane_copies banks apart so that equal bins of different lanes do not collide.
         const int ncw = row_threads / 32;
         const size_t budget = (size_t)di.smem_per_sm / 2 - 1024 - 256;
         size_t smem = 0;
@@ -829,8 +831,9 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         const int lc_first = g_tune_lane_copies > 0 ? g_tune_lane_copies : 4;
         for (int lc = lc_first; lc >= 1 && !fits; lc >>= 1) {
             p.lane_copies = lc;
-            p.hist_copies = ncw * lc;
-            const int want = lc > 1 ? 32 / lc : 1;  // copies of one warp start in different banks
+            p.warp_groups = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
+            p.hist_copies = p.warp_groups * lc;
+            const int want = lc > 1 ? 32 / lc : 1;
             p.hist_stride = K + 2;
             while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
             const size_t fixed = 1024 + 2 * kMaxStages * sizeof(uint64_t) + tail_bytes(K, p.hist_copies, p.hist_stride, p.lut_cells);
@@ -1170,8 +1173,16 @@ int dc_tune(int32_t key, int32_t value)
         g_tune_stages = value;
         return DC_OK;
     }
-    if (key == DC_TUNE_LANE_COPIES && (value == 0 || value == 1 || value == 2 || value == 4)) {
+    if (key == DC_TUNE_LANE_COPIES && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8)) {
         g_tune_lane_copies = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_WARP_GROUPS && value >= 0 && value <= 8) {
+        g_tune_warp_groups = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_BOX_FLOATS && (value == 0 || value == 16 || value == 32)) {
+        g_tune_box_floats = value;
         return DC_OK;
     }
     return DC_ERR_UNSUPPORTED;

@@ -354,7 +354,9 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 32, 2)
 dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 {
     extern __shared__ unsigned char smem_raw[];
-    unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // 1024-byte alignment by pointer arithmetic on the shared array itself (a round trip through an integer
+    // would hide the address space from the compiler and turn every shared access into a generic one)
+    unsigned char *smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
     unsigned char *stage0 = smem;
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)p.stages * p.stage_bytes);
     uint64_t *empty = full + kMaxStages;
@@ -1192,7 +1194,7 @@ int dc_simulate_launches(void) { return g_last_simulate_launches; }
 int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
 int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
 
-const char *dc_kernel_version(void) { return "sweep-tiled-4"; }
+const char *dc_kernel_version(void) { return "sweep-tiled-5"; }
 
 const char *dc_status_string(int status)
 {

@@ -77,6 +77,8 @@ struct SweepParams {
     int lane_copies;   // tiled kernel: copies per warp (lane l uses copy l % lane_copies); power of two
     int warp_groups;   // tiled kernel: warp w uses the copies of group w % warp_groups
     int lut_cells;     // tiled kernel: cells of the bin lookup table (the table has lut_cells + 1 entries)
+    int rule;          // DC_RULE_*
+    int aux_copies;    // rule 1: copies of the per-threshold worker-time maxima (0 for rule 0)
     int one;           // always 1; a value the compiler cannot see, used to tie a stage release to a warp vote
 };
 
@@ -171,10 +173,53 @@ struct RowWalk {
     }
 };
 
+// Non-negative floats order like their bit patterns, so an integer atomicMax is an exact float max.  The
+// plain read first makes the atomic rare: a maximum over thousands of workers changes only a few times.
+__device__ __forceinline__ void float_max_nonneg(float *slot, float v)
+{
+    if (v > *reinterpret_cast<volatile float *>(slot)) atomicMax(reinterpret_cast<int *>(slot), __float_as_int(v));
+}
+
+// Start-before-tau rule, one worker's row with a forward cursor (plain-load kernel).  Micro-batch m is run iff
+// the time before it, P_{m-1}, is < tau_k; the worker's time W(k) is the finish time of the last one it ran:
+// the first running sum that reaches tau_k, or the row total if none does, or 0 if tau_k <= 0.
+struct RowWalkStart {
+    float P;
+    int cur;  // #{k : tau_k <= P}
+    __device__ __forceinline__ void start(const float *tau_s, int K)
+    {
+        P = 0.0f;
+        cur = 0;
+        while (cur < K && 0.0f >= tau_s[cur]) ++cur;
+    }
+    __device__ __forceinline__ void step(float x, const float *tau_s, int *hist, float *wmax, int K)
+    {
+        atomicAdd(&hist[cur], 1);  // P_{m-1} is in bin cur
+        P = __fadd_rn(P, x);
+        while (cur < K && P >= tau_s[cur]) {  // thresholds first reached by this micro-batch
+            float_max_nonneg(&wmax[cur], P);
+            ++cur;
+        }
+    }
+    __device__ __forceinline__ void finish(float *tail, int K)
+    {
+        if (cur < K) float_max_nonneg(&tail[cur], P);  // thresholds cur.. were never reached: W = row total
+    }
+};
+
 __device__ __forceinline__ float warp_max(float v)
 {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_inclusive_max_scan(float v, int lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v = fmaxf(v, u);
+    }
     return v;
 }
 __device__ __forceinline__ int warp_inclusive_scan(int v, int lane)
@@ -193,11 +238,17 @@ __device__ __forceinline__ int warp_inclusive_scan(int v, int lane)
 // T = max_n T_n, writes step[t][k] = min(tau_k, T) + T^c and sync[t] = T + T^c, and clears the
 // histograms for the next trial.
 // ------------------------------------------------------------------------------------------
+// Rule 1 (start-before-tau): step[t][k] = max_n W_n(k) + T^c with
+//   max_n W_n(k) = max( wmax[k], max_{j <= k} tail[j] )
+// (wmax[k]: largest first-reaching running sum; tail[j]: largest total among workers that stopped at bin j).
 __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t, float rowmax, int tid, int nthr,
-                                               int barrier_id, const float *tau_s, int *hist, float *smax, int *wtot)
+                                               int barrier_id, const float *tau_s, int *hist, float *smax, int *wtot,
+                                               float *wmax, float *tail, float *wmx)
 {
     const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
     const int K = p.K, H = p.hist_copies, HS = p.hist_stride;
+    const int A = p.aux_copies, AS = K + 2;
+    const bool rule1 = p.rule == DC_RULE_START_BEFORE_TAU;
     rowmax = warp_max(rowmax);
     if (lane == 0) smax[warp] = rowmax;
     named_barrier(barrier_id, nthr);  // all histogram updates and smax[] visible
@@ -208,14 +259,29 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
     const int ipt = (K + nthr - 1) / nthr;  // bins per thread (consecutive)
     const int b0 = min(K, tid * ipt), b1 = min(K, b0 + ipt);
     int tot = 0;
-    for (int b = b0; b < b1; ++b)
+    float tl = 0.0f;
+    for (int b = b0; b < b1; ++b) {
         for (int c = 0; c < H; ++c) tot += hist[c * HS + b];
+        if (rule1)
+            for (int c = 0; c < A; ++c) tl = fmaxf(tl, tail[c * AS + b]);
+    }
     const int incl = warp_inclusive_scan(tot, lane);
     if (lane == 31) wtot[warp] = incl;
+    float tl_incl = 0.0f;
+    if (rule1) {
+        tl_incl = warp_inclusive_max_scan(tl, lane);
+        if (lane == 31) wmx[warp] = tl_incl;
+    }
     named_barrier(barrier_id, nthr);
 
     int run = incl - tot;
     for (int w = 0; w < warp; ++w) run += wtot[w];
+    float tail_run = 0.0f;  // max of tail[] over all bins before b0
+    if (rule1) {
+        const float up = __shfl_up_sync(0xffffffffu, tl_incl, 1);
+        if (lane > 0) tail_run = up;
+        for (int w = 0; w < warp; ++w) tail_run = fmaxf(tail_run, wmx[w]);
+    }
     float *step_row = p.out_step + t * K;
     int32_t *done_row = p.out_done + t * K;
     for (int b = b0; b < b1; ++b) {
@@ -226,7 +292,18 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
         }
         run += h;
         done_row[b] = run;
-        step_row[b] = __fadd_rn(fminf(tau_s[b], Tmax), p.t_comm);
+        if (!rule1) {
+            step_row[b] = __fadd_rn(fminf(tau_s[b], Tmax), p.t_comm);
+        } else {
+            float w = 0.0f;
+            for (int c = 0; c < A; ++c) {
+                tail_run = fmaxf(tail_run, tail[c * AS + b]);
+                w = fmaxf(w, wmax[c * AS + b]);
+                tail[c * AS + b] = 0.0f;
+                wmax[c * AS + b] = 0.0f;
+            }
+            step_row[b] = __fadd_rn(fmaxf(w, tail_run), p.t_comm);
+        }
     }
     for (int c = tid; c < H; c += nthr) {  // the bins of samples at or above the last threshold
         hist[c * HS + K] = 0;
@@ -244,6 +321,9 @@ struct SmemTail {
     int *wtot;
     int *meta;           // [0] lookup table has at most one finite threshold per cell, [1..2] lo, scale (as bits)
     unsigned short *lut; // lut_cells + 1 entries (tiled kernel only)
+    float *wmx;          // rule 1: warp totals of the tail max-scan
+    float *wmax;         // rule 1: [aux_copies][K + 2] largest first-reaching running sum per threshold
+    float *tail;         // rule 1: [aux_copies][K + 2] largest total among workers whose last bin is j
 };
 __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepParams &p)
 {
@@ -254,12 +334,17 @@ __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepP
     s.wtot = reinterpret_cast<int *>(s.smax + 32);
     s.meta = s.wtot + 32;
     s.lut = reinterpret_cast<unsigned short *>(s.meta + 8);
+    s.wmx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(s.lut) +
+                                      (((size_t)(p.lut_cells + 1) * sizeof(unsigned short) + 3) & ~(size_t)3));
+    s.wmax = s.wmx + 32;
+    s.tail = s.wmax + p.aux_copies * (p.K + 2);
     return s;
 }
-__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride, int lut_cells)
+__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride, int lut_cells, int aux_copies)
 {
     return sizeof(float) * (size_t)(K + 1) + sizeof(int) * (size_t)hist_copies * hist_stride + 72 * sizeof(int) +
-           (((size_t)(lut_cells + 1) * sizeof(unsigned short) + 3) & ~(size_t)3);
+           (((size_t)(lut_cells + 1) * sizeof(unsigned short) + 3) & ~(size_t)3) + 32 * sizeof(float) +
+           2 * sizeof(float) * (size_t)aux_copies * (K + 2);
 }
 
 __device__ __forceinline__ void load_thresholds(const SweepParams &p, const SmemTail &s, int tid, int nthr)
@@ -267,6 +352,7 @@ __device__ __forceinline__ void load_thresholds(const SweepParams &p, const Smem
     for (int k = tid; k < p.K; k += nthr) s.tau_s[k] = p.taus[k];
     if (tid == 0) s.tau_s[p.K] = __int_as_float(0x7f800000);  // +inf sentinel
     for (int i = tid; i < p.hist_copies * p.hist_stride; i += nthr) s.hist[i] = 0;
+    for (int i = tid; i < 2 * p.aux_copies * (p.K + 2); i += nthr) s.wmax[i] = 0.0f;  // wmax and tail are adjacent
 }
 
 // ------------------------------------------------------------------------------------------
@@ -330,15 +416,35 @@ __device__ __forceinline__ void build_lut(const SweepParams &p, const SmemTail &
 // (K: at or above the last threshold, K+1: only reachable by P = +inf); the epilogue reads 0..K-1.
 // ONE = the table guarantees at most one threshold to step over.
 template <bool ONE>
-__device__ __forceinline__ void bin_sample(float P, float lo, float scale, unsigned C, const unsigned short *lut,
-                                           const unsigned char *tau_b, unsigned K4, unsigned char *hist_b)
+__device__ __forceinline__ unsigned bin_offset(float P, float lo, float scale, unsigned C, const unsigned short *lut,
+                                               const unsigned char *tau_b, unsigned K4)
 {
     unsigned off = lut[lut_cell(P, lo, scale, C)];
     off += (P >= *reinterpret_cast<const float *>(tau_b + off)) ? 4u : 0u;  // tau_s[K] = +inf
     if (!ONE) {
         while (off < K4 && P >= *reinterpret_cast<const float *>(tau_b + off)) off += 4u;
     }
-    atomicAdd(reinterpret_cast<int *>(hist_b + off), 1);
+    return off;
+}
+template <bool ONE>
+__device__ __forceinline__ void bin_sample(float P, float lo, float scale, unsigned C, const unsigned short *lut,
+                                           const unsigned char *tau_b, unsigned K4, unsigned char *hist_b)
+{
+    atomicAdd(reinterpret_cast<int *>(hist_b + bin_offset<ONE>(P, lo, scale, C, lut, tau_b, K4)), 1);
+}
+// Start-before-tau rule: micro-batch m with finish time P.  The time before it lies in bin `prev` (byte
+// offset), which is what the completion count is taken on; the thresholds in [prev, j(P)) are first reached by
+// this micro-batch, so P is a candidate for their worker-time maximum.
+template <bool ONE>
+__device__ __forceinline__ void start_rule_sample(float P, unsigned &prev, float lo, float scale, unsigned C,
+                                                  const unsigned short *lut, const unsigned char *tau_b, unsigned K4,
+                                                  unsigned char *hist_b, unsigned char *wmax_b)
+{
+    const unsigned off = bin_offset<ONE>(P, lo, scale, C, lut, tau_b, K4);
+    atomicAdd(reinterpret_cast<int *>(hist_b + prev), 1);
+    const unsigned stop = min(off, K4);
+    for (unsigned o = prev; o < stop; o += 4u) float_max_nonneg(reinterpret_cast<float *>(wmax_b + o), P);
+    prev = off;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -349,7 +455,7 @@ __device__ __forceinline__ void bin_sample(float P, float lo, float scale, unsig
 // add); if before the group every lane is at or above the last threshold they are in the bin
 // nobody reads; otherwise each running sum is binned through the lookup table.
 // ------------------------------------------------------------------------------------------
-template <int NQ>
+template <int NQ, int RULE>
 __global__ void __launch_bounds__(kMaxRowsPerPass + 32, 2)
 dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 {
@@ -409,6 +515,11 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     const float lut_lo = __int_as_float(s.meta[1]), lut_scale = __int_as_float(s.meta[2]);
     const unsigned C = (unsigned)p.lut_cells;
     const float tau_first = s.tau_s[0], tau_last = s.tau_s[K - 1];
+    // rule 1 only: this thread's copies of the worker-time maxima, and the bin of a running time of 0
+    unsigned char *wmax_b = reinterpret_cast<unsigned char *>(s.wmax + (p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0));
+    float *mytail = s.tail + (p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0);
+    unsigned off_zero = 0;
+    if (RULE == 1) off_zero = bin_offset<false>(0.0f, lut_lo, lut_scale, C, s.lut, tau_b, K4);
     // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
     // (threads past the last row of the box read the last row instead: always inside the stage)
     const uint32_t row_off = (uint32_t)min(tid, p.rows - 1) * (uint32_t)p.pitch;
@@ -420,6 +531,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
         for (int pass = 0; pass < p.passes; ++pass) {
             const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
             float P = 0.0f;
+            unsigned prev = off_zero;  // rule 1: bin (byte offset) of the running time before the next micro-batch
             for (int c = 0; c < p.chunks; ++c, ++i) {
                 const int st = i % S;
                 mbar_wait(&full[st], (i / S) & 1u, kErrLoadNeverArrived);
@@ -457,6 +569,25 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                         const float pend = v[g + GQ - 1].w;  // running sum after the group
                         if (__all_sync(0xffffffffu, !valid || pend < tau_first)) {
                             if (valid) cnt0 += 4 * gq;
+                        } else if (RULE == 1) {
+                            if (valid) {
+#pragma unroll
+                                for (int q = 0; q < GQ; ++q) {
+                                    if (q < gq) {
+                                        if (one) {
+                                            start_rule_sample<true>(v[g + q].x, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
+                                            start_rule_sample<true>(v[g + q].y, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
+                                            start_rule_sample<true>(v[g + q].z, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
+                                            start_rule_sample<true>(v[g + q].w, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
+                                        } else {
+                                            start_rule_sample<false>(v[g + q].x, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
+                                            start_rule_sample<false>(v[g + q].y, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
+                                            start_rule_sample<false>(v[g + q].z, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
+                                            start_rule_sample<false>(v[g + q].w, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
+                                        }
+                                    }
+                                }
+                            }
                         } else if (!__all_sync(0xffffffffu, !valid || v[g].x >= tau_last)) {
                             if (valid) {
                                 if (one && gq == GQ) {  // the common case, no per-sample predicates
@@ -490,10 +621,13 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                     }
                 }
             }
-            if (valid) rowmax = fmaxf(rowmax, P);
+            if (valid) {
+                rowmax = fmaxf(rowmax, P);
+                if (RULE == 1 && prev < K4) float_max_nonneg(mytail + (prev >> 2), P);  // thresholds never reached: W = total
+            }
         }
         if (cnt0 > 0) atomicAdd(myhist, cnt0);
-        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot);
+        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot, s.wmax, s.tail, s.wmx);
     }
 }
 
@@ -516,14 +650,22 @@ __global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepPar
             const int n = pass * p.rows + tid;
             if (n < p.N) {
                 const float *row = p.lat + ((size_t)t * p.N + n) * p.M;
-                RowWalk w;
-                w.start(s.tau_s);
-                for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), m, s.tau_s, myhist, p.K);
-                w.finish(p.M, myhist);
-                rowmax = fmaxf(rowmax, w.P);
+                if (p.rule == DC_RULE_FINISH_BEFORE_TAU) {
+                    RowWalk w;
+                    w.start(s.tau_s);
+                    for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), m, s.tau_s, myhist, p.K);
+                    w.finish(p.M, myhist);
+                    rowmax = fmaxf(rowmax, w.P);
+                } else {
+                    RowWalkStart w;
+                    w.start(s.tau_s, p.K);
+                    for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), s.tau_s, myhist, s.wmax, p.K);
+                    w.finish(s.tail, p.K);
+                    rowmax = fmaxf(rowmax, w.P);
+                }
             }
         }
-        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot);
+        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot, s.wmax, s.tail, s.wmx);
     }
 }
 
@@ -551,15 +693,30 @@ dc_reduce_partial(const float *__restrict__ step, const int32_t *__restrict__ do
     long long s_done = 0;
     const double nan = __longlong_as_double(0x7ff8000000000000LL);
     if (k < K) {
-        for (long long t = t0 + warp; t < t1; t += kRedWarps) {
-            const double st = (double)step[t * K + k];
-            const int dn_i = done[t * K + k];
-            const double dn = (double)dn_i;
-            const double sy = sync ? (double)sync[t] : nan;
-            s_step += st;
-            s_done += dn_i;
-            s_ratio += dn / st;
-            s_S += (sy / st) * (dn / NM);
+        // four rows in flight per thread (the loads do not depend on each other); summed in row order
+        for (long long t = t0 + warp; t < t1; t += 4 * kRedWarps) {
+            float st_f[4], sy_f[4];
+            int dn_i[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const long long tt = t + (long long)u * kRedWarps;
+                const bool ok = tt < t1;
+                st_f[u] = ok ? step[tt * K + k] : 1.0f;
+                dn_i[u] = ok ? done[tt * K + k] : 0;
+                sy_f[u] = (ok && sync) ? sync[tt] : 0.0f;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (t + (long long)u * kRedWarps < t1) {
+                    const double st = (double)st_f[u];
+                    const double dn = (double)dn_i[u];
+                    const double sy = sync ? (double)sy_f[u] : nan;
+                    s_step += st;
+                    s_done += dn_i[u];
+                    s_ratio += dn / st;
+                    s_S += (sy / st) * (dn / NM);
+                }
+            }
         }
     }
     sh[warp][0][lane] = s_step;
@@ -600,19 +757,43 @@ dc_reduce_partial(const float *__restrict__ step, const int32_t *__restrict__ do
     }
 }
 
-__global__ void __launch_bounds__(256)
+// Phase 2: block = 32 thresholds; warp w adds the partial sums of chunks w, w+8, ... and the eight warp sums
+// are combined in warp order (a fixed order: reproducible).
+__global__ void __launch_bounds__(kRedWarps * 32)
 dc_reduce_final(const double *__restrict__ ws, long long T, int K, double NM, int chunks, double *stats, double *baseline)
 {
-    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    __shared__ double sh[kRedWarps][4][32];
+    __shared__ double shs[kRedWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int k = blockIdx.x * 32 + lane;
+    double a = 0.0, c = 0.0, d = 0.0;
+    long long b = 0;
     if (k < K) {
-        double a = 0.0, c = 0.0, d = 0.0;
-        long long b = 0;
-        for (int ch = 0; ch < chunks; ++ch) {
+        for (int ch = warp; ch < chunks; ch += kRedWarps) {
             const double *part = ws + (size_t)ch * 4 * K;
             a += part[0 * K + k];
             b += __double_as_longlong(part[1 * K + k]);
             c += part[2 * K + k];
             d += part[3 * K + k];
+        }
+    }
+    sh[warp][0][lane] = a;
+    sh[warp][1][lane] = __longlong_as_double(b);
+    sh[warp][2][lane] = c;
+    sh[warp][3][lane] = d;
+    if (blockIdx.x == 0 && lane == 0) {
+        double ssum = 0.0;
+        for (int ch = warp; ch < chunks; ch += kRedWarps) ssum += ws[(size_t)chunks * 4 * K + ch];
+        shs[warp] = ssum;
+    }
+    __syncthreads();
+    if (warp == 0 && k < K) {
+        a = 0.0; c = 0.0; d = 0.0; b = 0;
+        for (int w = 0; w < kRedWarps; ++w) {
+            a += sh[w][0][lane];
+            b += __double_as_longlong(sh[w][1][lane]);
+            c += sh[w][2][lane];
+            d += sh[w][3][lane];
         }
         const double Td = (double)T;
         stats[DC_STAT_MEAN_STEP * K + k] = a / Td;
@@ -621,9 +802,9 @@ dc_reduce_final(const double *__restrict__ ws, long long T, int K, double NM, in
         stats[DC_STAT_THR_MEAN * K + k] = c / Td;
         stats[DC_STAT_S_EFF * K + k] = d / Td;
     }
-    if (k == 0) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
         double ssum = 0.0;
-        for (int ch = 0; ch < chunks; ++ch) ssum += ws[(size_t)chunks * 4 * K + ch];
+        for (int w = 0; w < kRedWarps; ++w) ssum += shs[w];
         baseline[0] = ssum / (double)T;
         baseline[1] = ((double)T * NM) / ssum;
     }
@@ -756,17 +937,17 @@ int validate_simulate(const float *lat, int64_t T, int64_t N, int64_t M, const f
     if ((reinterpret_cast<uintptr_t>(lat) & 3) || (reinterpret_cast<uintptr_t>(taus) & 3) ||
         (reinterpret_cast<uintptr_t>(out_step) & 3) || (reinterpret_cast<uintptr_t>(out_done) & 3))
         return DC_ERR_ALIGN;
-    if (rule != DC_RULE_FINISH_BEFORE_TAU) return DC_ERR_UNSUPPORTED;
+    if (rule != DC_RULE_FINISH_BEFORE_TAU && rule != DC_RULE_START_BEFORE_TAU) return DC_ERR_UNSUPPORTED;
     return DC_OK;
 }
 
 bool tiled_ok(const float *lat, int64_t M) { return (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0); }
 
-template <int NQ>
+template <int NQ, int RULE>
 int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
                  cudaStream_t stream)
 {
-    auto kernel = dc_sweep_tiled<NQ>;
+    auto kernel = dc_sweep_tiled<NQ, RULE>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
@@ -806,6 +987,8 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.warp_groups = 1;
     p.lut_cells = 0;
     p.one = 1;
+    p.rule = rule;
+    p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? 1 : 0;
 
     if (tiled_ok(lat, M)) {
         EncodeTiledFn encode = get_encode_fn();
@@ -835,10 +1018,11 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
             p.lane_copies = lc;
             p.warp_groups = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
             p.hist_copies = p.warp_groups * lc;
+            if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = p.warp_groups;
             const int want = lc > 1 ? 32 / lc : 1;
             p.hist_stride = K + 2;
             while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
-            const size_t fixed = 1024 + 2 * kMaxStages * sizeof(uint64_t) + tail_bytes(K, p.hist_copies, p.hist_stride, p.lut_cells);
+            const size_t fixed = 1024 + 2 * kMaxStages * sizeof(uint64_t) + tail_bytes(K, p.hist_copies, p.hist_stride, p.lut_cells, p.aux_copies);
             const int s_max = g_tune_stages > 0 ? g_tune_stages : min(kMaxStages, max(2, kStageBudgetBytes / p.stage_bytes));
             for (int st = s_max; st >= 2; --st) {
                 smem = fixed + (size_t)st * p.stage_bytes;
@@ -866,10 +1050,17 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         const int block = row_threads + 32;
         const int nq = p.bw / 4;
         int lrc;
-        if (nq <= 1) lrc = launch_tiled<1>(map, p, block, smem, T, di, stream);
-        else if (nq <= 2) lrc = launch_tiled<2>(map, p, block, smem, T, di, stream);
-        else if (nq <= 4) lrc = launch_tiled<4>(map, p, block, smem, T, di, stream);
-        else lrc = launch_tiled<8>(map, p, block, smem, T, di, stream);
+        if (rule == DC_RULE_FINISH_BEFORE_TAU) {
+            if (nq <= 1) lrc = launch_tiled<1, 0>(map, p, block, smem, T, di, stream);
+            else if (nq <= 2) lrc = launch_tiled<2, 0>(map, p, block, smem, T, di, stream);
+            else if (nq <= 4) lrc = launch_tiled<4, 0>(map, p, block, smem, T, di, stream);
+            else lrc = launch_tiled<8, 0>(map, p, block, smem, T, di, stream);
+        } else {
+            if (nq <= 1) lrc = launch_tiled<1, 1>(map, p, block, smem, T, di, stream);
+            else if (nq <= 2) lrc = launch_tiled<2, 1>(map, p, block, smem, T, di, stream);
+            else if (nq <= 4) lrc = launch_tiled<4, 1>(map, p, block, smem, T, di, stream);
+            else lrc = launch_tiled<8, 1>(map, p, block, smem, T, di, stream);
+        }
         if (lrc == DC_OK) g_last_simulate_launches = 1;
         return lrc;
     }
@@ -877,7 +1068,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     // plain-load kernel
     p.rows = row_threads;  // one row per thread per pass
     p.passes = (int)((N + p.rows - 1) / p.rows);
-    const size_t smem = tail_bytes(K, p.hist_copies, p.hist_stride, 0);
+    const size_t smem = tail_bytes(K, p.hist_copies, p.hist_stride, 0, p.aux_copies);
     if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
     if (cudaFuncSetAttribute(dc_sweep_plain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return DC_ERR_CUDA;
@@ -967,7 +1158,7 @@ int dc_reduce_trials(const float *out_step, const int32_t *out_done, const float
     dim3 grid1((unsigned)((K + 31) / 32), (unsigned)r.chunks);
     dc_reduce_partial<<<grid1, kRedWarps * 32, 0, stream>>>(out_step, out_done, out_sync, T, K, NM, r.chunks, r.rows_per_chunk, ws);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
-    dc_reduce_final<<<(unsigned)((K + 255) / 256), 256, 0, stream>>>(ws, T, K, NM, r.chunks, stats, baseline);
+    dc_reduce_final<<<(unsigned)((K + 31) / 32), kRedWarps * 32, 0, stream>>>(ws, T, K, NM, r.chunks, stats, baseline);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     g_last_reduce_launches = 2;
     return DC_OK;
@@ -1001,7 +1192,7 @@ int dc_reduce_trials_static(const float *out_step, const int32_t *out_done, cons
     dim3 grid1((unsigned)((K + 31) / 32), (unsigned)r.chunks);
     dc_reduce_partial<<<grid1, kRedWarps * 32, 0, stream>>>(out_step, out_done, out_sync, T, K, NM, r.chunks, r.rows_per_chunk, ws);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
-    dc_reduce_final<<<(unsigned)((K + 255) / 256), 256, 0, stream>>>(ws, T, K, NM, r.chunks, stats, baseline);
+    dc_reduce_final<<<(unsigned)((K + 31) / 32), kRedWarps * 32, 0, stream>>>(ws, T, K, NM, r.chunks, stats, baseline);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     return DC_OK;
 }
@@ -1081,7 +1272,7 @@ int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M, 
     if (T <= 0 || N <= 0 || M <= 0 || K <= 0 || chunk_trials <= 0) return DC_ERR_SHAPE;
     if (K > DC_MAX_K || N > INT32_MAX || M > INT32_MAX || N * M > (int64_t)INT32_MAX || T > (int64_t)INT32_MAX)
         return DC_ERR_RANGE;
-    if (rule != DC_RULE_FINISH_BEFORE_TAU) return DC_ERR_UNSUPPORTED;
+    if (rule != DC_RULE_FINISH_BEFORE_TAU && rule != DC_RULE_START_BEFORE_TAU) return DC_ERR_UNSUPPORTED;
     if (objective != DC_STAT_S_EFF && objective != DC_STAT_THR && objective != DC_STAT_THR_MEAN) return DC_ERR_UNSUPPORTED;
     if (chunk_trials > T) chunk_trials = T;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023) ||
@@ -1194,7 +1385,7 @@ int dc_simulate_launches(void) { return g_last_simulate_launches; }
 int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
 int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
 
-const char *dc_kernel_version(void) { return "sweep-tiled-5"; }
+const char *dc_kernel_version(void) { return "sweep-tiled-6"; }
 
 const char *dc_status_string(int status)
 {

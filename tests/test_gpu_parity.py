@@ -310,3 +310,46 @@ def test_results_do_not_depend_on_tuning_or_timing(api):
         api.dc_tune(api.TUNE_STAGES, 0)
         api.dc_tune(api.TUNE_LANE_COPIES, 0)
     api.dc_device_status()
+
+
+# ---- the start-before-tau rule (timeout looked at between accumulations) ---------------------------
+
+@pytest.mark.parametrize("T,N,M,K", EDGE_SHAPES)
+def test_start_before_tau_rule_matches_oracle(api, T, N, M, K):
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=300 + T + N + M, shift=0.01, mean=0.02).numpy()
+    taus = grid_for(lat, K, seed=K + 1)
+    t_comm = 0.0625 + 0.001
+    ref = oracle.sweep(lat, taus, t_comm, rule=1)
+    res = run_gpu(api, torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda(), t_comm, rule=1)
+    compare_sweep(res, ref, f"rule 1 {(T, N, M, K)}")
+    compare_stats(res, ref, N, M, what=f"rule 1 {(T, N, M, K)}")
+    api.dc_device_status()
+
+
+def test_start_before_tau_rule_special_grids(api):
+    T, N, M = 6, 37, 24
+    lat = W.iid_latencies("dyadic", T, N, M, seed=16, hi=8).numpy()
+    lat[:, ::3, ::2] = 0.0
+    for taus in (np.arange(40, dtype=np.float32) / 16.0, [-1.0, 0.0], [0.0], [INF], [-INF, INF], [1e30, INF, INF],
+                 [0.5] * 7, [-2.0, -1.0, 0.0, 0.125, 0.125, 3.0, INF]):
+        taus = np.array(taus, np.float32)
+        ref = oracle.sweep(lat, taus, 0.25, rule=1)
+        res = run_gpu(api, torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda(), 0.25, rule=1)
+        compare_sweep(res, ref, f"rule 1 {taus[:4]}")
+
+
+@pytest.mark.parametrize("name,trials", [("tiny", 1024), ("paper_scale", 2048), ("extrapolation", 256),
+                                         ("correlated", 48), ("bandwidth_stress", 48)])
+def test_start_before_tau_rule_on_workloads(api, name, trials):
+    w = W.WORKLOADS[name].with_trials(trials)
+    lat_d = W.fill_latencies(w, "cuda")
+    taus = W.make_taus(w)
+    res = run_gpu(api, lat_d, torch.from_numpy(taus).cuda(), w.t_comm, rule=1)
+    ref = oracle.sweep(lat_d.cpu().numpy(), taus, w.t_comm, rule=1)
+    compare_sweep(res, ref, f"rule 1 {name}")
+    compare_stats(res, ref, w.N, w.M, what=f"rule 1 {name}")
+    # the two rules are tied together: a worker starts at most one micro-batch more than it finishes in time
+    res0 = run_gpu(api, lat_d, torch.from_numpy(taus).cuda(), w.t_comm, rule=0)
+    assert bool((res.out_done >= res0.out_done).all()) and bool((res.out_done <= res0.out_done + w.N).all())
+    assert bool((res.out_step >= res0.out_step).all())
+    api.dc_device_status()

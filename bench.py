@@ -32,6 +32,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+from paper_2306_10598_b200 import sharding  # noqa: E402
 from paper_2306_10598_b200 import workloads as W  # noqa: E402
 
 METRIC = "latency samples/s (tau-sweep: dc_simulate + dc_reduce_trials + dc_argmax_tau)"
@@ -223,7 +224,7 @@ def run_ours(args, w: W.Workload):
         dist.init_process_group("nccl", device_id=dev)
 
     # every rank sweeps its own tensor of the same shape (independent trials: weak scaling)
-    wr = W.Workload(w.name, w.T, w.N, w.M, w.K, w.tau_lo, w.tau_hi, w.tau_unit, w.t_comm, w.law, seed=w.seed + rank)
+    wr = sharding.rank_workload(w, rank)
     lat = W.fill_latencies(wr, dev)
     taus_np = W.make_taus(wr)
     taus = torch.from_numpy(taus_np).to(dev)
@@ -279,10 +280,7 @@ def run_ours(args, w: W.Workload):
     step_ms = [e[0].elapsed_time(e[2]) for e in events]
     sim_ms = [e[0].elapsed_time(e[1]) for e in events]
     total_ms = sum(step_ms)
-    if dist:
-        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = sharding.max_over_ranks(total_ms, dev)
     clocks = sampler.stop(t_mark0, t_mark1) if rank == 0 else None
     api.dc_device_status()
 
@@ -344,10 +342,7 @@ def run_ours(args, w: W.Workload):
         for _ in range(n_e2e):
             hs = api.dc_sweep_host(host, taus_h, wr.t_comm, wsv, chunk, stats_out=stats_h, baseline_out=base_h)
         e2e_s = time.perf_counter() - t0   # dc_sweep_host is synchronous: results are in host memory on return
-        if dist:
-            tt = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_s = float(tt.item())
+        e2e_s = sharding.max_over_ranks(e2e_s, dev)
         e2e = {"value": world * n_e2e * Te * N * M / e2e_s, "unit": UNIT,
                "h2d_bytes_per_step": 4 * Te * N * M + 4 * K, "d2h_bytes_per_step": 8 * api.NSTATS * K + 16 + 8,
                "steps": n_e2e, "trials_per_step": Te, "chunk_trials": chunk, "ms_per_step": 1e3 * e2e_s / n_e2e,

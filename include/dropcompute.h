@@ -106,6 +106,17 @@ int dc_simulate_ex(const float *latencies, int64_t T, int64_t N, int64_t M,
                    int32_t rule, void *stream);
 
 /*
+ * dc_simulate_tc — dc_simulate_ex with the communication time given per trial, as Algorithm 2 has it
+ * ("communication time for each iteration T_i^c"):
+ *   t_comm_trials  DEVICE, [T] fp32; trial t uses t_comm_trials[t] wherever dc_simulate_ex uses t_comm.
+ * Everything else as dc_simulate_ex.  dc_reduce_trials needs no change: it works from out_step and out_sync.
+ */
+int dc_simulate_tc(const float *latencies, int64_t T, int64_t N, int64_t M,
+                   const float *taus, int32_t K, const float *t_comm_trials,
+                   float *out_step, int32_t *out_done, float *out_sync,
+                   int32_t rule, void *stream);
+
+/*
  * dc_reduce_trials — statistics over trials in fp64 (Algorithm 2: S_i(tau) and S_eff(tau); Eq. 6;
  * Sec. 4.4 throughput).  Sums run over trials in a fixed order that depends only on (T, K), so the
  * result is reproducible bit for bit.

@@ -67,7 +67,7 @@ def _bind(lib):
     p = ctypes.c_void_p
     for name in ("dco_sweep_literal", "dco_sweep_rows"):
         fn = getattr(lib, name)
-        fn.argtypes = [p, i64, i64, i64, p, i64, f32, i32, p, p, p]
+        fn.argtypes = [p, i64, i64, i64, p, i64, f32, p, i32, p, p, p]
         fn.restype = i32
     lib.dco_reduce_trials.argtypes = [p, p, p, i64, i64, i64, i64, p, p]
     lib.dco_reduce_trials.restype = i32
@@ -122,7 +122,8 @@ def sweep(lat, taus, t_comm: float, rule: int = 0, order: str = "rows", lib=None
     """Per-(iteration, tau) step time and completed count.
 
     ``order='literal'`` runs Algorithm 2's loop nest as printed (tau outermost);
-    ``order='rows'`` reads every sample once (same predicate, same integers)."""
+    ``order='rows'`` reads every sample once (same predicate, same integers).
+    ``t_comm`` is one number, or an array of T numbers (Algorithm 2's per-iteration T_i^c)."""
     lib = lib or load()
     lat = _f32c(lat, 3)
     taus = _f32c(taus, 1)
@@ -132,7 +133,12 @@ def sweep(lat, taus, t_comm: float, rule: int = 0, order: str = "rows", lib=None
     done = np.empty((T, K), np.int32)
     sync = np.empty((T,), np.float32)
     fn = {"literal": lib.dco_sweep_literal, "rows": lib.dco_sweep_rows}[order]
-    rc = fn(lat.ctypes.data, T, N, M, taus.ctypes.data, K, np.float32(t_comm), rule,
+    tc_vec = None
+    if np.ndim(t_comm) > 0:
+        tc_vec = np.ascontiguousarray(t_comm, dtype=np.float32)
+        assert tc_vec.shape == (T,)
+    rc = fn(lat.ctypes.data, T, N, M, taus.ctypes.data, K, np.float32(0.0 if tc_vec is not None else t_comm),
+            None if tc_vec is None else tc_vec.ctypes.data, rule,
             step.ctypes.data, done.ctypes.data, sync.ctypes.data)
     if rc != 0:
         raise ValueError(f"oracle sweep failed with status {rc}")

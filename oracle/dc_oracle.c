@@ -20,7 +20,7 @@
  *   - M~ is kept as the integer number of completed micro-batches summed over
  *     workers (Algorithm 2 adds 1/N per hit; the integer count divided once at
  *     the end is the same number in exact arithmetic);
- *   - T^c is one scalar for all iterations;
+ *   - T^c is given per iteration as in Algorithm 2, or as one scalar used for all iterations;
  *   - statistics over iterations are binary64;
  *   - argmax takes the first maximum and never selects a NaN.
  *
@@ -54,9 +54,11 @@
  *   out_step [T,K]  min(tau, T_i) + T^c            (rule 0)
  *   out_done [T,K]  N * M~_i(tau) as an integer
  *   out_sync [T]    T_i + T^c   (the tau = infinity step time)
+ *   t_comm_per_iter [T] or NULL: Algorithm 2 takes the communication time T_i^c per iteration; when this is
+ *                   NULL the one scalar t_comm is used for every iteration.
  * ------------------------------------------------------------------------- */
 int dco_sweep_literal(const float *lat, int64_t T, int64_t N, int64_t M,
-                      const float *taus, int64_t K, float t_comm, int rule,
+                      const float *taus, int64_t K, float t_comm, const float *t_comm_per_iter, int rule,
                       float *out_step, int32_t *out_done, float *out_sync)
 {
     if (!lat || !taus || !out_step || !out_done || !out_sync) return 1;
@@ -65,6 +67,7 @@ int dco_sweep_literal(const float *lat, int64_t T, int64_t N, int64_t M,
     for (int64_t k = 0; k < K; ++k) {
         const float tau = taus[k];
         for (int64_t i = 0; i < T; ++i) {
+            const float tc = t_comm_per_iter ? t_comm_per_iter[i] : t_comm;  /* T_i^c of Algorithm 2 */
             int64_t done = 0;      /* N * M~_i(tau) */
             float Ti = 0.0f;       /* slowest worker's full compute time */
             float Wi = 0.0f;       /* slowest worker's time under the threshold (rule 1) */
@@ -89,11 +92,11 @@ int dco_sweep_literal(const float *lat, int64_t T, int64_t N, int64_t M,
                 Wi = fmaxf(Wi, Win);
             }
             if (rule == 0)
-                out_step[i * K + k] = fminf(tau, Ti) + t_comm;
+                out_step[i * K + k] = fminf(tau, Ti) + tc;
             else
-                out_step[i * K + k] = Wi + t_comm;
+                out_step[i * K + k] = Wi + tc;
             out_done[i * K + k] = (int32_t)done;
-            out_sync[i] = Ti + t_comm;
+            out_sync[i] = Ti + tc;
         }
     }
     return 0;
@@ -107,7 +110,7 @@ int dco_sweep_literal(const float *lat, int64_t T, int64_t N, int64_t M,
  * Iterations are independent and are spread over OpenMP threads.
  * ------------------------------------------------------------------------- */
 int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
-                   const float *taus, int64_t K, float t_comm, int rule,
+                   const float *taus, int64_t K, float t_comm, const float *t_comm_per_iter, int rule,
                    float *out_step, int32_t *out_done, float *out_sync)
 {
     if (!lat || !taus || !out_step || !out_done || !out_sync) return 1;
@@ -125,6 +128,7 @@ int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
 #pragma omp for schedule(dynamic, 1)
         for (int64_t i = 0; i < T; ++i) {
             if (!cnt || !wmax) continue;
+            const float tc = t_comm_per_iter ? t_comm_per_iter[i] : t_comm;  /* T_i^c of Algorithm 2 */
             float Ti = 0.0f;
             for (int64_t k = 0; k < K; ++k) { cnt[k] = 0; wmax[k] = 0.0f; }
             for (int64_t n = 0; n < N; ++n) {
@@ -147,9 +151,9 @@ int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
                 }
                 Ti = fmaxf(Ti, Tin);
             }
-            out_sync[i] = Ti + t_comm;
+            out_sync[i] = Ti + tc;
             for (int64_t k = 0; k < K; ++k) {
-                out_step[i * K + k] = (rule == 0) ? (fminf(taus[k], Ti) + t_comm) : (wmax[k] + t_comm);
+                out_step[i * K + k] = (rule == 0) ? (fminf(taus[k], Ti) + tc) : (wmax[k] + tc);
                 out_done[i * K + k] = (int32_t)cnt[k];
             }
         }

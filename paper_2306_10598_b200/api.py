@@ -24,7 +24,7 @@ NSTATS = 5
 STAT_NAMES = ("mean_step", "done_frac", "thr", "thr_mean", "s_eff")
 
 EXPORTS = (
-    "dc_simulate", "dc_simulate_ex", "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_reduce_trials_static",
+    "dc_simulate", "dc_simulate_ex", "dc_simulate_tc", "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_reduce_trials_static",
     "dc_argmax_tau",
     "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan",
     "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string", "dc_tune",
@@ -48,6 +48,8 @@ _lib = ctypes.CDLL(LIB_PATH)
 _p, _i64, _i32, _f32, _sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_float, ctypes.c_size_t
 _lib.dc_simulate.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _p, _p, _p]
 _lib.dc_simulate_ex.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _p, _p, _p, _i32, _p]
+_lib.dc_simulate_tc.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _p, _p, _p, _p, _i32, _p]
+_lib.dc_simulate_tc.restype = ctypes.c_int
 _lib.dc_reduce_workspace_bytes.argtypes = [_i64, _i32]
 _lib.dc_reduce_workspace_bytes.restype = _sz
 _lib.dc_reduce_trials.argtypes = [_p, _p, _p, _i64, _i32, _i64, _i64, _p, _p, _p, _sz, _p]
@@ -124,6 +126,21 @@ def dc_simulate_ex(latencies: torch.Tensor, taus: torch.Tensor, t_comm: float, o
                                    _dev(out_done, torch.int32, "out_done"),
                                    None if out_sync is None else _dev(out_sync, torch.float32, "out_sync"),
                                    int(rule), _stream(latencies)), "dc_simulate_ex")
+
+
+def dc_simulate_tc(latencies: torch.Tensor, taus: torch.Tensor, t_comm_trials: torch.Tensor, out_step: torch.Tensor,
+                   out_done: torch.Tensor, out_sync: Optional[torch.Tensor], rule: int = RULE_FINISH_BEFORE_TAU) -> None:
+    """``dc_simulate_tc``: like dc_simulate_ex with one communication time per trial (t_comm_trials [T] fp32)."""
+    T, N, M = latencies.shape
+    K = taus.shape[0]
+    assert tuple(out_step.shape) == (T, K) and tuple(out_done.shape) == (T, K) and tuple(t_comm_trials.shape) == (T,)
+    assert out_sync is None or tuple(out_sync.shape) == (T,)
+    with torch.cuda.device(latencies.device):
+        _check(_lib.dc_simulate_tc(_dev(latencies, torch.float32, "latencies"), T, N, M, _dev(taus, torch.float32, "taus"),
+                                   K, _dev(t_comm_trials, torch.float32, "t_comm_trials"),
+                                   _dev(out_step, torch.float32, "out_step"), _dev(out_done, torch.int32, "out_done"),
+                                   None if out_sync is None else _dev(out_sync, torch.float32, "out_sync"),
+                                   int(rule), _stream(latencies)), "dc_simulate_tc")
 
 
 def dc_reduce_workspace_bytes(T: int, K: int) -> int:

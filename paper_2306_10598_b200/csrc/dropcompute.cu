@@ -63,6 +63,7 @@ struct SweepParams {
     long long T;
     int N, M, K;
     float t_comm;
+    const float *t_comm_vec;  // per-trial T^c, or null: t_comm for every trial
     int passes;        // passes over a trial's workers
     int rows;          // workers per pass (box height for the tiled kernel, blockDim.x for the plain one)
     int chunks;        // column chunks per row
@@ -249,6 +250,7 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
     const int K = p.K, H = p.hist_copies, HS = p.hist_stride;
     const int A = p.aux_copies, AS = K + 2;
     const bool rule1 = p.rule == DC_RULE_START_BEFORE_TAU;
+    const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
     rowmax = warp_max(rowmax);
     if (lane == 0) smax[warp] = rowmax;
     named_barrier(barrier_id, nthr);  // all histogram updates and smax[] visible
@@ -293,7 +295,7 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
         run += h;
         done_row[b] = run;
         if (!rule1) {
-            step_row[b] = __fadd_rn(fminf(tau_s[b], Tmax), p.t_comm);
+            step_row[b] = __fadd_rn(fminf(tau_s[b], Tmax), t_comm);
         } else {
             float w = 0.0f;
             for (int c = 0; c < A; ++c) {
@@ -302,14 +304,14 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
                 tail[c * AS + b] = 0.0f;
                 wmax[c * AS + b] = 0.0f;
             }
-            step_row[b] = __fadd_rn(fmaxf(w, tail_run), p.t_comm);
+            step_row[b] = __fadd_rn(fmaxf(w, tail_run), t_comm);
         }
     }
     for (int c = tid; c < H; c += nthr) {  // the bins of samples at or above the last threshold
         hist[c * HS + K] = 0;
         if (HS > K + 1) hist[c * HS + K + 1] = 0;
     }
-    if (tid == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, p.t_comm);
+    if (tid == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
     named_barrier(barrier_id, nthr);  // histograms cleared, smax/wtot free again
 }
 
@@ -957,8 +959,9 @@ int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t
 }
 
 int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
-                  float *out_step, int32_t *out_done, float *out_sync, int32_t rule, void *stream_v)
+                  const float *t_comm_vec, float *out_step, int32_t *out_done, float *out_sync, int32_t rule, void *stream_v)
 {
+    if (t_comm_vec && (reinterpret_cast<uintptr_t>(t_comm_vec) & 3)) return DC_ERR_ALIGN;
     const int rc = validate_simulate(lat, T, N, M, taus, K, out_step, out_done, rule);
     if (rc != DC_OK) return rc;
     if (out_sync && (reinterpret_cast<uintptr_t>(out_sync) & 3)) return DC_ERR_ALIGN;
@@ -978,6 +981,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.M = (int)M;
     p.K = K;
     p.t_comm = t_comm;
+    p.t_comm_vec = t_comm_vec;
     p.passes = (int)((N + kMaxRowsPerPass - 1) / kMaxRowsPerPass);
     p.rows = (int)((N + p.passes - 1) / p.passes);
     const int row_threads = ((p.rows + 31) / 32) * 32;
@@ -1116,13 +1120,20 @@ extern "C" {
 int dc_simulate(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
                 float *out_step, int32_t *out_done, void *stream)
 {
-    return simulate_impl(latencies, T, N, M, taus, K, t_comm, out_step, out_done, nullptr, DC_RULE_FINISH_BEFORE_TAU, stream);
+    return simulate_impl(latencies, T, N, M, taus, K, t_comm, nullptr, out_step, out_done, nullptr, DC_RULE_FINISH_BEFORE_TAU, stream);
 }
 
 int dc_simulate_ex(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
                    float *out_step, int32_t *out_done, float *out_sync, int32_t rule, void *stream)
 {
-    return simulate_impl(latencies, T, N, M, taus, K, t_comm, out_step, out_done, out_sync, rule, stream);
+    return simulate_impl(latencies, T, N, M, taus, K, t_comm, nullptr, out_step, out_done, out_sync, rule, stream);
+}
+
+int dc_simulate_tc(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K,
+                   const float *t_comm_trials, float *out_step, int32_t *out_done, float *out_sync, int32_t rule, void *stream)
+{
+    if (!t_comm_trials) return DC_ERR_NULL;
+    return simulate_impl(latencies, T, N, M, taus, K, 0.0f, t_comm_trials, out_step, out_done, out_sync, rule, stream);
 }
 
 int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K)
@@ -1331,7 +1342,7 @@ int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M, 
         DC_TRY(cudaEventRecord(ready[b], copy_stream));
         DC_TRY(cudaStreamWaitEvent(stream, ready[b], 0));
         if (!cuda_fail) {
-            rc = simulate_impl(buf[b], tn, N, M, d_taus, K, t_comm, d_step + (size_t)t0 * K, d_done + (size_t)t0 * K,
+            rc = simulate_impl(buf[b], tn, N, M, d_taus, K, t_comm, nullptr, d_step + (size_t)t0 * K, d_done + (size_t)t0 * K,
                                d_sync + t0, rule, stream);
             launches += 1;
         }

@@ -197,6 +197,33 @@ def pin_hand_example(lib, order="rows"):
             assert np.allclose(s_eff, st.stats[4], rtol=1e-14) and k_star == want["k_star"]
 
 
+def pin_per_iteration_comm(lib, order="rows"):
+    """Algorithm 2 takes the communication time per iteration (T_i^c).  A vector of equal values is the
+    scalar case bit for bit; with different values the hand-worked example changes only through
+    min(tau, T_i) + T_i^c and (T_i + T_i^c) / (...), recomputed here in rational arithmetic."""
+    with open(os.path.join(GOLDEN, "alg2_hand_example.json")) as f:
+        g = json.load(f)
+    lat = np.array([[[_fr(x) for x in row] for row in it] for it in g["latencies"]], np.float32)
+    taus_q = [Fraction(x) for x in g["taus"]]
+    taus = np.array([float(x) for x in taus_q], np.float32)
+    T, N, M = lat.shape
+    same = oracle.sweep(lat, taus, np.full(T, 0.25, np.float32), order=order, lib=lib)
+    scal = oracle.sweep(lat, taus, 0.25, order=order, lib=lib)
+    assert np.array_equal(same.step, scal.step) and np.array_equal(same.sync, scal.sync) and np.array_equal(same.done, scal.done)
+    tc = [Fraction(1, 8), Fraction(1, 2), Fraction(1, 4)]
+    tmax = [Fraction(x) - Fraction(g["t_comm"]) for x in g["sync"]]          # the example's T_i
+    sw = oracle.sweep(lat, taus, np.array([float(x) for x in tc], np.float32), order=order, lib=lib)
+    st = oracle.reduce_trials(sw.step, sw.done, sw.sync, N, M, lib=lib)
+    done = g["rule0"]["done"]
+    want_step = [[min(tau, tmax[i]) + tc[i] for tau in taus_q] for i in range(T)]
+    assert np.array_equal(sw.step, np.array([[float(x) for x in r] for r in want_step], np.float32))
+    assert np.array_equal(sw.sync, np.array([float(tmax[i] + tc[i]) for i in range(T)], np.float32))
+    assert np.array_equal(sw.done, np.array(done, np.int32))
+    for k in range(len(taus_q)):
+        s_eff = sum((tmax[i] + tc[i]) / want_step[i][k] * Fraction(done[i][k], N * M) for i in range(T)) / T
+        assert abs(st.stats[4, k] - float(s_eff)) <= 1e-14
+
+
 def pin_fp32_left_to_right(lib, order="rows"):
     """The running sum is binary32 with one rounding per addition, taken m = 1..M in order
     (Algorithm 2's inner loop; the precision is this build's reading)."""
@@ -327,9 +354,9 @@ def pin_independence_and_bailey(lib, order="rows"):
 
 ALL_PINS = (
     pin_exp_max_harmonic, pin_normal_max_quadrature, pin_done_frac_normal_eq5, pin_done_frac_erlang,
-    pin_enumeration, pin_hand_example, pin_fp32_left_to_right, pin_m1_sort, pin_invariants, pin_argmax,
+    pin_enumeration, pin_hand_example, pin_per_iteration_comm, pin_fp32_left_to_right, pin_m1_sort, pin_invariants, pin_argmax,
     pin_literal_equals_rows, pin_independence_and_bailey,
 )
 # a quick subset that still kills every planted mistake (used by the mutation test)
-FAST_PINS = (pin_hand_example, pin_enumeration, pin_fp32_left_to_right, pin_m1_sort, pin_argmax, pin_invariants,
+FAST_PINS = (pin_hand_example, pin_per_iteration_comm, pin_enumeration, pin_fp32_left_to_right, pin_m1_sort, pin_argmax, pin_invariants,
              pin_exp_max_harmonic)

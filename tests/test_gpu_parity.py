@@ -353,3 +353,29 @@ def test_start_before_tau_rule_on_workloads(api, name, trials):
     assert bool((res.out_done >= res0.out_done).all()) and bool((res.out_done <= res0.out_done + w.N).all())
     assert bool((res.out_step >= res0.out_step).all())
     api.dc_device_status()
+
+
+@pytest.mark.parametrize("rule", [0, 1])
+@pytest.mark.parametrize("T,N,M,K", [(9, 8, 4, 16), (5, 300, 36, 40), (4, 33, 129, 17), (40, 200, 12, 64)])
+def test_per_trial_communication_time(api, T, N, M, K, rule):
+    """Algorithm 2's T_i^c: one communication time per trial."""
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=400 + T, shift=0.01, mean=0.02).numpy()
+    taus = grid_for(lat, K, seed=K + 2)
+    tc = np.random.default_rng(T).uniform(0.01, 0.3, T).astype(np.float32)
+    ref = oracle.sweep(lat, taus, tc, rule=rule)
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    step = torch.empty((T, K), dtype=torch.float32, device="cuda")
+    done = torch.empty((T, K), dtype=torch.int32, device="cuda")
+    sync = torch.empty((T,), dtype=torch.float32, device="cuda")
+    api.dc_simulate_tc(lat_d, taus_d, torch.from_numpy(tc).cuda(), step, done, sync, rule)
+    stats = torch.empty((api.NSTATS, K), dtype=torch.float64, device="cuda")
+    base = torch.empty(2, dtype=torch.float64, device="cuda")
+    ws = torch.empty(api.dc_reduce_workspace_bytes(T, K), dtype=torch.uint8, device="cuda")
+    api.dc_reduce_trials(step, done, sync, N, M, stats, base, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(done.cpu().numpy(), ref.done)
+    assert np.array_equal(step.cpu().numpy().view(np.uint32), ref.step.view(np.uint32))
+    assert np.array_equal(sync.cpu().numpy().view(np.uint32), ref.sync.view(np.uint32))
+    st = oracle.reduce_trials(ref.step, ref.done, ref.sync, N, M)
+    assert np.allclose(stats.cpu().numpy(), st.stats, rtol=RTOL_STATS, atol=0)
+    assert np.allclose(base.cpu().numpy(), st.baseline, rtol=RTOL_STATS, atol=0)

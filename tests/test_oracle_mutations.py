@@ -16,11 +16,11 @@ MUTANTS = [
                             ("cnt[k] += (Tin < taus[k]) ? 1 : 0;", "cnt[k] += (Tin <= taus[k]) ? 1 : 0;", 1)]),
     ("last_worker_not_max", [("Ti = fmaxf(Ti, Tin);", "Ti = Tin;", 3)]),
     ("double_accumulator", [("float Tin = 0.0f;", "double Tin = 0.0;", 3)]),
-    ("no_min_with_tau", [("out_step[i * K + k] = fminf(tau, Ti) + t_comm;", "out_step[i * K + k] = tau + t_comm;", 1),
-                         ("(fminf(taus[k], Ti) + t_comm)", "(taus[k] + t_comm)", 1)]),
-    ("sync_without_comm", [("out_sync[i] = Ti + t_comm;", "out_sync[i] = Ti;", 2)]),
-    ("step_without_comm", [("out_step[i * K + k] = fminf(tau, Ti) + t_comm;", "out_step[i * K + k] = fminf(tau, Ti);", 1),
-                           ("(fminf(taus[k], Ti) + t_comm)", "(fminf(taus[k], Ti))", 1)]),
+    ("no_min_with_tau", [("out_step[i * K + k] = fminf(tau, Ti) + tc;", "out_step[i * K + k] = tau + tc;", 1),
+                         ("(fminf(taus[k], Ti) + tc)", "(taus[k] + tc)", 1)]),
+    ("sync_without_comm", [("out_sync[i] = Ti + tc;", "out_sync[i] = Ti;", 2)]),
+    ("step_without_comm", [("out_step[i * K + k] = fminf(tau, Ti) + tc;", "out_step[i * K + k] = fminf(tau, Ti);", 1),
+                           ("(fminf(taus[k], Ti) + tc)", "(fminf(taus[k], Ti))", 1)]),
     ("transposed_layout", [("const float *t = lat + (i * N + n) * M;", "const float *t = lat + (i * M + n) * N;", 2)]),
     ("skips_first_microbatch", [("for (int64_t m = 0; m < M; ++m) {\n                    if (rule == 0) {",
                                  "for (int64_t m = 1; m < M; ++m) {\n                    if (rule == 0) {", 2)]),
@@ -32,6 +32,7 @@ MUTANTS = [
     ("speedup_inverted_ratio", [("((double)sync[i] / st)", "(st / (double)sync[i])", 1)]),
     ("thr_mean_is_ratio_of_means", [("sum_ratio / (double)T", "((double)sum_done / sum_step)", 1)]),
     ("argmax_takes_last", [("v > objective[best]", "v >= objective[best]", 1)]),
+    ("comm_time_of_wrong_iteration", [("t_comm_per_iter ? t_comm_per_iter[i] : t_comm", "t_comm_per_iter ? t_comm_per_iter[0] : t_comm", 2)]),
     ("rule1_inclusive", [("if (before < taus[k]) {", "if (Tin < taus[k]) {", 1),
                          ("if (Tin < tau) {\n                            done += 1;", "if (Tin + t[m] < tau) {\n                            done += 1;", 1)]),
 ]

@@ -177,6 +177,21 @@ int dc_argmax_tau(const double *stats, const float *taus, int32_t K, int32_t obj
                   int32_t *out_k, float *out_tau, double *out_value, void *stream);
 
 /*
+ * dc_closed_form — the paper's analytical estimates (App. C.2) on a threshold grid, from the mean `mu` and
+ * standard deviation `sigma` of ONE micro-batch latency, for comparison with the simulation (Fig. 3):
+ *   out[0][k] = E[M~(tau_k)] / M        = (1/M) sum_{m=1..M} Phi((tau_k - m mu) / sqrt(m sigma^2))     (Eq. 5 / 10)
+ *   out[1][k] = min(tau_k, E[T]) + t_comm
+ *   out[2][k] = E[S_eff(tau_k)]         = out[0][k] (E[T] + t_comm) / out[1][k]                        (Eq. 11; numerator as in Eq. 6)
+ *   scalars[0] = E[T] = sqrt(M sigma^2) ((1-g) Phi^-1(1 - 1/N) + g Phi^-1(1 - 1/(e N))) + M mu         (Eq. 4 / 12,
+ *                g = Euler-Mascheroni; T does not contain t_comm), or mean_T itself when mean_T >= 0 (the
+ *                'analytical given E[T]' variant: pass the simulated mean_sync - t_comm).
+ * The analytic tau* is dc_argmax_tau over row 2 (pass `out` as stats with objective 2 — row 2 of a [3][K] matrix).
+ *   taus  DEVICE [K] fp32      out  DEVICE [3][K] fp64      scalars  DEVICE [1] fp64      M >= 1, N >= 2, sigma > 0
+ */
+int dc_closed_form(double mu, double sigma, int64_t M, int64_t N, double t_comm, double mean_T,
+                   const float *taus, int32_t K, double *out, double *scalars, void *stream);
+
+/*
  * dc_sweep_host — the whole path for a caller whose samples live in HOST memory: copies the
  * latencies to the device in chunks of whole trials (overlapped with the kernels), runs
  * dc_simulate_ex, dc_reduce_trials and dc_argmax_tau, copies the results back and waits for them.

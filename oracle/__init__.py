@@ -75,6 +75,11 @@ def _bind(lib):
     lib.dco_argmax.restype = i64
     lib.dco_algorithm2.argtypes = [p, i64, i64, i64, p, i64, f32, p, p]
     lib.dco_algorithm2.restype = i32
+    f64 = ctypes.c_double
+    lib.dco_closed_form.argtypes = [f64, f64, i64, i64, f64, f64, p, i64, p, p]
+    lib.dco_closed_form.restype = i32
+    lib.dco_bailey_mean_max.argtypes = [f64, f64, i64, i64]
+    lib.dco_bailey_mean_max.restype = f64
     return lib
 
 
@@ -181,3 +186,30 @@ def algorithm2(lat, taus, t_comm: float, lib=None):
     if rc != 0:
         raise ValueError(f"oracle algorithm2 failed with status {rc}")
     return s_eff, int(k_star.value)
+
+
+class ClosedForm(NamedTuple):
+    done_frac: np.ndarray  # [K] E[M~]/M                      (Eq. 5)
+    step: np.ndarray       # [K] min(tau, E[T]) + T^c
+    s_eff: np.ndarray      # [K] E[S_eff]                      (Eq. 11)
+    mean_T: float          # E[T] used (Eq. 4/12, or the value passed in)
+    k_star: int
+    tau_star: float
+
+
+def closed_form(mu: float, sigma: float, M: int, N: int, t_comm: float, taus, mean_T: float = -1.0, lib=None) -> ClosedForm:
+    """App. C.2's closed forms on a threshold grid; ``mean_T >= 0`` plugs in a measured E[T]."""
+    lib = lib or load()
+    taus = _f32c(taus, 1)
+    K = taus.shape[0]
+    out = np.empty((3, K), np.float64)
+    sc = np.empty((3,), np.float64)
+    rc = lib.dco_closed_form(mu, sigma, M, N, t_comm, mean_T, taus.ctypes.data, K, out.ctypes.data, sc.ctypes.data)
+    if rc != 0:
+        raise ValueError(f"oracle closed_form failed with status {rc}")
+    return ClosedForm(out[0], out[1], out[2], float(sc[0]), int(sc[1]), float(sc[2]))
+
+
+def bailey_mean_max(mu: float, sigma: float, M: int, N: int, lib=None) -> float:
+    lib = lib or load()
+    return float(lib.dco_bailey_mean_max(mu, sigma, M, N))

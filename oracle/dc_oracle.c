@@ -251,3 +251,62 @@ int dco_algorithm2(const float *lat, int64_t T, int64_t N, int64_t M,
     *k_star = dco_argmax(s_eff, K);
     return 0;
 }
+
+/* ===========================================================================
+ * Closed-form companion (App. C.2): what the paper derives from the mean mu and
+ * variance sigma^2 of one micro-batch latency alone.
+ *
+ *   Phi        standard normal CDF, here 0.5 erfc(-x / sqrt 2)
+ *   Phi^-1     its inverse; libm has none, so it is found by bisection on Phi
+ *   Eq. 4 / 12 E[T] ~ sqrt(M sigma^2) ((1-g) Phi^-1(1 - 1/N) + g Phi^-1(1 - 1/(e N))) + M mu,
+ *              g the Euler-Mascheroni constant.  Eq. 12 as printed also adds T^c; in this build T
+ *              never contains T^c (the paper adds it separately in Eq. 6, Eq. 11 and Algorithm 2).
+ *   Eq. 5 / 10 E[M~(tau)] ~ sum_{m=1..M} Phi((tau - m mu) / sqrt(m sigma^2))
+ *   Eq. 11     E[S_eff(tau)] ~ (E[M~]/M) (E[T] + T^c) / (min(tau, E[T]) + T^c)     (numerator as in Eq. 6)
+ *   tau*       arg max over the grid of Eq. 11 (first maximum)
+ * mean_T >= 0 replaces Eq. 12 by a measured E[T] (the paper's 'analytical given E[T]' curve).
+ * out[0][k] = E[M~]/M, out[1][k] = min(tau_k, E[T]) + T^c, out[2][k] = E[S_eff];  scalars = E[T], k*, tau*.
+ * =========================================================================== */
+static double dco_phi(double x) { return 0.5 * erfc(-x / sqrt(2.0)); }
+
+static double dco_phi_inv(double p)
+{
+    if (!(p > 0.0)) return -INFINITY;
+    if (!(p < 1.0)) return INFINITY;
+    double lo = -40.0, hi = 40.0;
+    for (int it = 0; it < 200; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (dco_phi(mid) < p) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+double dco_bailey_mean_max(double mu, double sigma, int64_t M, int64_t N)
+{
+    const double g = 0.57721566490153286061;
+    const double z = (1.0 - g) * dco_phi_inv(1.0 - 1.0 / (double)N) + g * dco_phi_inv(1.0 - 1.0 / (exp(1.0) * (double)N));
+    return sqrt((double)M * sigma * sigma) * z + (double)M * mu;
+}
+
+int dco_closed_form(double mu, double sigma, int64_t M, int64_t N, double t_comm, double mean_T,
+                    const float *taus, int64_t K, double *out, double *scalars)
+{
+    if (!taus || !out || !scalars) return 1;
+    if (M <= 0 || N < 2 || K <= 0) return 2;
+    if (!(sigma > 0.0)) return 4;
+    const double ET = (mean_T >= 0.0) ? mean_T : dco_bailey_mean_max(mu, sigma, M, N);
+    for (int64_t k = 0; k < K; ++k) {
+        const double tau = (double)taus[k];
+        double em = 0.0;
+        for (int64_t m = 1; m <= M; ++m) em += dco_phi((tau - (double)m * mu) / sqrt((double)m * sigma * sigma));
+        const double step = fmin(tau, ET) + t_comm;
+        out[0 * K + k] = em / (double)M;
+        out[1 * K + k] = step;
+        out[2 * K + k] = (em / (double)M) * (ET + t_comm) / step;
+    }
+    const int64_t ks = dco_argmax(out + 2 * K, K);
+    scalars[0] = ET;
+    scalars[1] = (double)ks;
+    scalars[2] = ks >= 0 ? (double)taus[ks] : NAN;
+    return 0;
+}

@@ -26,7 +26,7 @@ STAT_NAMES = ("mean_step", "done_frac", "thr", "thr_mean", "s_eff")
 EXPORTS = (
     "dc_simulate", "dc_simulate_ex", "dc_simulate_tc", "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_reduce_trials_static",
     "dc_argmax_tau",
-    "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan",
+    "dc_closed_form", "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan",
     "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string", "dc_tune",
     "dc_kernel_version",
 )
@@ -59,6 +59,8 @@ _lib.dc_argmax_tau.argtypes = [_p, _p, _i32, _i32, _p, _p, _p, _p]
 _lib.dc_sweep_host_workspace_bytes.argtypes = [_i64, _i64, _i64, _i32, _i64]
 _lib.dc_sweep_host_workspace_bytes.restype = _sz
 _lib.dc_sweep_host.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _i32, _i32, _i64, _p, _p, _p, _p, _p, _sz, _p]
+_lib.dc_closed_form.argtypes = [ctypes.c_double, ctypes.c_double, _i64, _i64, ctypes.c_double, ctypes.c_double, _p, _i32, _p, _p, _p]
+_lib.dc_closed_form.restype = ctypes.c_int
 _lib.dc_check_inputs.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _p, _p, _p]
 _lib.dc_device_status.argtypes = [_p]
 _lib.dc_simulate_plan.argtypes = [_p, _i64, _i64, _i64, _i32]
@@ -189,6 +191,18 @@ def dc_argmax_tau(stats: torch.Tensor, taus: torch.Tensor, objective: int, out_k
         _check(_lib.dc_argmax_tau(_dev(stats, torch.float64, "stats"), _dev(taus, torch.float32, "taus"), K, int(objective),
                                   _dev(out_k, torch.int32, "out_k"), _dev(out_tau, torch.float32, "out_tau"),
                                   _dev(out_value, torch.float64, "out_value"), _stream(stats)), "dc_argmax_tau")
+
+
+def dc_closed_form(mu: float, sigma: float, M: int, N: int, t_comm: float, taus: torch.Tensor, out: torch.Tensor,
+                   scalars: torch.Tensor, mean_T: float = -1.0) -> None:
+    """``dc_closed_form``: App. C.2's estimates on the grid.  out [3,K] fp64 (E[M~]/M, step, E[S_eff]),
+    scalars [1] fp64 (E[T]); mean_T >= 0 plugs in a measured E[T]."""
+    K = taus.shape[0]
+    assert tuple(out.shape) == (3, K) and scalars.numel() >= 1
+    with torch.cuda.device(taus.device):
+        _check(_lib.dc_closed_form(float(mu), float(sigma), int(M), int(N), float(t_comm), float(mean_T),
+                                   _dev(taus, torch.float32, "taus"), K, _dev(out, torch.float64, "out"),
+                                   _dev(scalars, torch.float64, "scalars"), _stream(taus)), "dc_closed_form")
 
 
 def dc_check_inputs(latencies: torch.Tensor, taus: torch.Tensor) -> None:

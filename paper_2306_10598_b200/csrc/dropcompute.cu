@@ -846,6 +846,33 @@ dc_argmax_kernel(const double *__restrict__ obj, const float *__restrict__ taus,
     }
 }
 
+// Closed-form companion (App. C.2), one thread per threshold, fp64:
+//   Eq. 5/10  E[M~(tau)]/M = (1/M) sum_m Phi((tau - m mu) / sqrt(m sigma^2))
+//   Eq. 4/12  E[T] = sqrt(M sigma^2) ((1-g) Phi^-1(1 - 1/N) + g Phi^-1(1 - 1/(e N))) + M mu   (T without T^c)
+//   Eq. 11    E[S_eff(tau)] = (E[M~]/M) (E[T] + T^c) / (min(tau, E[T]) + T^c)
+// out[0][k], out[1][k], out[2][k] = E[M~]/M, min(tau_k, E[T]) + T^c, E[S_eff]; scalars[0] = E[T].
+__global__ void __launch_bounds__(128)
+dc_closed_form_kernel(double mu, double sigma, long long M, long long N, double t_comm, double mean_T,
+                      const float *__restrict__ taus, int K, double *out, double *scalars)
+{
+    const double g = 0.57721566490153286061;
+    double ET = mean_T;
+    if (!(mean_T >= 0.0)) {
+        const double z = (1.0 - g) * normcdfinv(1.0 - 1.0 / (double)N) + g * normcdfinv(1.0 - 1.0 / (exp(1.0) * (double)N));
+        ET = sqrt((double)M * sigma * sigma) * z + (double)M * mu;
+    }
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k == 0) scalars[0] = ET;
+    if (k >= K) return;
+    const double tau = (double)taus[k];
+    double em = 0.0;
+    for (long long m = 1; m <= M; ++m) em += normcdf((tau - (double)m * mu) / sqrt((double)m * sigma * sigma));
+    const double step = fmin(tau, ET) + t_comm;
+    out[0 * (size_t)K + k] = em / (double)M;
+    out[1 * (size_t)K + k] = step;
+    out[2 * (size_t)K + k] = (em / (double)M) * (ET + t_comm) / step;
+}
+
 // Data precondition check: counts latencies that are negative, NaN or infinite, and thresholds
 // that are NaN or smaller than their predecessor.
 __global__ void __launch_bounds__(256)
@@ -1221,6 +1248,20 @@ int dc_argmax_tau(const double *stats, const float *taus, int32_t K, int32_t obj
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     g_last_argmax_launches = 1;
     return DC_OK;
+}
+
+int dc_closed_form(double mu, double sigma, int64_t M, int64_t N, double t_comm, double mean_T, const float *taus,
+                   int32_t K, double *out, double *scalars, void *stream_v)
+{
+    if (!taus || !out || !scalars) return DC_ERR_NULL;
+    if (M <= 0 || N < 2 || K <= 0) return DC_ERR_SHAPE;
+    if (K > DC_MAX_K || !(sigma > 0.0) || !(sigma < 1e300) || !(mu == mu) || !(t_comm == t_comm)) return DC_ERR_RANGE;
+    if ((reinterpret_cast<uintptr_t>(out) & 7) || (reinterpret_cast<uintptr_t>(scalars) & 7) ||
+        (reinterpret_cast<uintptr_t>(taus) & 3))
+        return DC_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    dc_closed_form_kernel<<<(unsigned)((K + 127) / 128), 128, 0, stream>>>(mu, sigma, M, N, t_comm, mean_T, taus, K, out, scalars);
+    return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
 
 int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, int64_t *counters,

@@ -133,6 +133,71 @@ _LAWS: Dict[str, Callable[[torch.Tensor, torch.Generator], None]] = {
     "shifted_gamma2": _fill_shifted_gamma2,
 }
 
+# --- the paper's own synthetic settings (App. B.1 and C.3) -------------------------------------------
+# App. C.3 simulates 12 accumulations of 0.45 s + eps with eps drawn from one of the laws of its two tables
+# (all with mean 0.225; variance 0.05 unless stated).  App. B.1 adds to a base latency mu the bounded
+# log-normal delay  mu * min(Z / alpha, beta),  Z ~ LogNormal(4, 1), alpha = 2 exp(4.5), beta = 5.5.
+C3_BASE = 0.45
+C3_M = 12
+C3_NOISE = {
+    # name: (kind, parameters as printed in the tables)
+    "lognormal_0.05": ("lognormal", -1.84, 0.83),
+    "normal_0.05": ("normal", 0.23, 0.22),
+    "bernoulli_0.05": ("bernoulli", 0.45, 0.5),
+    "exponential_0.05": ("exponential", 4.47),
+    "gamma_0.05": ("gamma1", 4.5),
+    "lognormal_0.10": ("lognormal", -2.04, 1.04),
+    "lognormal_0.15": ("lognormal", -2.18, 1.17),
+    "lognormal_0.20": ("lognormal", -2.29, 1.26),
+    "lognormal_0.25": ("lognormal", -2.38, 1.33),
+    "lognormal_0.30": ("lognormal", -2.46, 1.39),
+}
+B1_ALPHA = 2.0 * math.exp(4.5)
+B1_BETA = 5.5
+
+
+def _fill_c3(out: torch.Tensor, g: torch.Generator, name: str) -> None:
+    spec = C3_NOISE[name]
+    kind = spec[0]
+    if kind == "lognormal":
+        out.log_normal_(spec[1], spec[2], generator=g)
+    elif kind == "normal":
+        out.normal_(spec[1], spec[2], generator=g)
+        out.clamp_(min=-C3_BASE)          # a latency cannot be negative (a -3.1 sigma draw)
+    elif kind == "bernoulli":
+        out.uniform_(0.0, 1.0, generator=g)
+        out.copy_(torch.where(out < spec[2], torch.full_like(out, spec[1]), torch.zeros_like(out)))
+    elif kind == "exponential":
+        out.exponential_(spec[1], generator=g)
+    elif kind == "gamma1":                # Gamma(shape 1, rate 4.5) is Exponential(rate 4.5)
+        out.exponential_(spec[1], generator=g)
+    else:
+        raise ValueError(kind)
+    out.add_(C3_BASE)
+
+
+def _fill_b1(out: torch.Tensor, g: torch.Generator, mu: float) -> None:
+    # base latency mu plus the bounded log-normal delay of App. B.1
+    out.log_normal_(4.0, 1.0, generator=g)
+    out.div_(B1_ALPHA)
+    out.clamp_(max=B1_BETA)
+    out.mul_(mu)
+    out.add_(mu)
+
+
+def c3_workload(name: str, N: int, T: int = 256, K: int = 64, t_comm: float = 0.5, seed: int = 0) -> Workload:
+    """App. C.3: 12 accumulations of 0.45 s + eps, eps from the table row `name`; grid over [0.6, 2.0] x the
+    mean worker time 12 * 0.675 s."""
+    if name not in C3_NOISE:
+        raise ValueError(name)
+    return Workload(f"c3_{name}", T, N, C3_M, K, 0.6, 2.0, C3_M * (C3_BASE + 0.225), t_comm, f"c3:{name}", seed)
+
+
+def b1_workload(N: int, mu: float = 0.45, M: int = 12, T: int = 256, K: int = 64, t_comm: float = 0.5, seed: int = 0) -> Workload:
+    """App. B.1: every accumulation takes mu * (1 + min(Z / alpha, beta)); the delay has mean about 0.5 mu."""
+    return Workload("b1_delay", T, N, M, K, 0.6, 2.5, M * mu * 1.5, t_comm, f"b1:{mu!r}", seed)
+
+
 _CHUNK_FLOATS = 1 << 26  # 256 MB of fp32 per chunk of whole trials
 
 
@@ -153,7 +218,12 @@ def fill_latencies(w: Workload, device, out: Optional[torch.Tensor] = None,
         out = torch.empty((t1 - t0, w.N, w.M), dtype=torch.float32, device=device)
     assert out.shape == (t1 - t0, w.N, w.M) and out.dtype == torch.float32 and out.is_contiguous()
     ct = chunk_trials(w)
-    law = _LAWS[w.law]
+    if w.law.startswith("c3:"):
+        law = lambda o, g, _n=w.law[3:]: _fill_c3(o, g, _n)
+    elif w.law.startswith("b1:"):
+        law = lambda o, g, _m=float(w.law[3:]): _fill_b1(o, g, _m)
+    else:
+        law = _LAWS[w.law]
     c = t0 // ct
     while c * ct < t1:
         lo, hi = c * ct, min((c + 1) * ct, w.T)

@@ -352,11 +352,49 @@ def pin_independence_and_bailey(lib, order="rows"):
     assert abs(st.baseline[0] - bailey) <= 0.03 * bailey
 
 
+def pin_closed_form(lib, order="rows"):
+    """App. C.2: Phi and Phi^-1 against scipy, Eq. 4/12, Eq. 5/10, Eq. 11 and the analytic tau*; then the
+    closed forms against the simulator itself where they are exact (normal micro-batches: Eq. 5) or good
+    to a few percent (Bailey's E[max])."""
+    g = 0.5772156649015329
+    for mu, sd, M, N in ((1.0, 0.1, 16, 400), (0.675, math.sqrt(0.05), 12, 1000), (0.03, 0.004, 64, 2)):
+        z = (1 - g) * scipy.stats.norm.ppf(1 - 1 / N) + g * scipy.stats.norm.ppf(1 - 1 / (math.e * N))
+        want = math.sqrt(M) * sd * z + M * mu
+        assert abs(oracle.bailey_mean_max(mu, sd, M, N, lib=lib) - want) <= 1e-12 * want
+        taus = np.linspace(0.4 * M * mu, 1.4 * M * mu, 41).astype(np.float32)
+        tc = 0.3 * mu
+        cf = oracle.closed_form(mu, sd, M, N, tc, taus, lib=lib)
+        assert abs(cf.mean_T - want) <= 1e-12 * want
+        t64 = taus.astype(np.float64)
+        em = sum(scipy.stats.norm.cdf((t64 - m * mu) / (sd * math.sqrt(m))) for m in range(1, M + 1)) / M
+        assert np.allclose(cf.done_frac, em, rtol=1e-12, atol=1e-15)
+        assert np.allclose(cf.step, np.minimum(t64, want) + tc, rtol=1e-14)
+        assert np.allclose(cf.s_eff, em * (want + tc) / (np.minimum(t64, want) + tc), rtol=1e-12)
+        assert cf.k_star == int(np.argmax(cf.s_eff)) and cf.tau_star == float(taus[cf.k_star])
+        # a threshold far above everything: nothing dropped, no speedup
+        far = oracle.closed_form(mu, sd, M, N, tc, np.array([100 * M * mu], np.float32), lib=lib)
+        assert abs(far.s_eff[0] - 1.0) < 1e-12 and abs(far.done_frac[0] - 1.0) < 1e-12
+        # a measured E[T] replaces Eq. 12
+        given = oracle.closed_form(mu, sd, M, N, tc, taus, mean_T=1.1 * want, lib=lib)
+        assert given.mean_T == 1.1 * want and np.allclose(given.done_frac, cf.done_frac, rtol=0, atol=0)
+        assert np.allclose(given.s_eff, em * (1.1 * want + tc) / (np.minimum(t64, 1.1 * want) + tc), rtol=1e-12)
+    # against the simulator: normal micro-batches, many workers
+    mu, sd, N, M, T = 0.025, 0.004, 300, 16, 500
+    lat = W.iid_latencies("normal", T, N, M, 21, mu=mu, sd=sd)
+    taus = np.linspace(0.8 * M * mu, 1.3 * M * mu, 11).astype(np.float32)
+    sw, st = _stats(lib, lat, taus, 0.05, order=order)
+    cf = oracle.closed_form(mu, sd, M, N, 0.05, taus, lib=lib)
+    assert np.allclose(st.stats[1], cf.done_frac, rtol=0, atol=2e-3)                    # Eq. 5 is exact here
+    assert abs(st.baseline[0] - 0.05 - cf.mean_T) <= 0.03 * cf.mean_T                   # Bailey: a few percent
+    given = oracle.closed_form(mu, sd, M, N, 0.05, taus, mean_T=st.baseline[0] - 0.05, lib=lib)
+    assert np.allclose(st.stats[4], given.s_eff, rtol=0.02)                             # Eq. 11 with measured E[T]
+
+
 ALL_PINS = (
     pin_exp_max_harmonic, pin_normal_max_quadrature, pin_done_frac_normal_eq5, pin_done_frac_erlang,
     pin_enumeration, pin_hand_example, pin_per_iteration_comm, pin_fp32_left_to_right, pin_m1_sort, pin_invariants, pin_argmax,
-    pin_literal_equals_rows, pin_independence_and_bailey,
+    pin_literal_equals_rows, pin_independence_and_bailey, pin_closed_form,
 )
 # a quick subset that still kills every planted mistake (used by the mutation test)
-FAST_PINS = (pin_hand_example, pin_per_iteration_comm, pin_enumeration, pin_fp32_left_to_right, pin_m1_sort, pin_argmax, pin_invariants,
-             pin_exp_max_harmonic)
+FAST_PINS = (pin_hand_example, pin_per_iteration_comm, pin_enumeration, pin_fp32_left_to_right, pin_m1_sort, pin_argmax,
+             pin_closed_form, pin_invariants, pin_exp_max_harmonic)

@@ -379,3 +379,48 @@ def test_per_trial_communication_time(api, T, N, M, K, rule):
     st = oracle.reduce_trials(ref.step, ref.done, ref.sync, N, M)
     assert np.allclose(stats.cpu().numpy(), st.stats, rtol=RTOL_STATS, atol=0)
     assert np.allclose(base.cpu().numpy(), st.baseline, rtol=RTOL_STATS, atol=0)
+
+
+def test_closed_form_matches_oracle(api):
+    """App. C.2's estimates (Eq. 4/12, 5/10, 11) on the GPU against the oracle's, and the analytic tau*."""
+    import math
+    for mu, sd, M, N, tc in ((1.0, 0.1, 16, 400, 0.3), (0.675, math.sqrt(0.05), 12, 1000, 0.5), (0.03, 0.004, 64, 2, 0.0),
+                             (0.007, 0.0014, 128, 2048, 0.1)):
+        taus = np.linspace(0.4 * M * mu, 1.4 * M * mu, 257).astype(np.float32)
+        taus_d = torch.from_numpy(taus).cuda()
+        out = torch.empty((3, taus.size), dtype=torch.float64, device="cuda")
+        sc = torch.empty(1, dtype=torch.float64, device="cuda")
+        for mean_T in (-1.0, 1.07 * M * mu):
+            ref = oracle.closed_form(mu, sd, M, N, tc, taus, mean_T=mean_T)
+            api.dc_closed_form(mu, sd, M, N, tc, taus_d, out, sc, mean_T=mean_T)
+            k = torch.empty((), dtype=torch.int32, device="cuda")
+            tau_s = torch.empty((), dtype=torch.float32, device="cuda")
+            val = torch.empty((), dtype=torch.float64, device="cuda")
+            api.dc_argmax_tau(out, taus_d, 2, k, tau_s, val)           # row 2 of the [3,K] matrix
+            torch.cuda.synchronize()
+            got = out.cpu().numpy()
+            assert np.allclose(got[0], ref.done_frac, rtol=1e-9, atol=1e-300)
+            assert np.allclose(got[1], ref.step, rtol=1e-12)
+            assert np.allclose(got[2], ref.s_eff, rtol=1e-9, atol=1e-300)
+            assert abs(float(sc.item()) - ref.mean_T) <= 1e-10 * abs(ref.mean_T)
+            assert int(k.item()) == ref.k_star and float(tau_s.item()) == ref.tau_star
+
+
+def test_appendix_c3_workload_and_scale_row(api):
+    """The paper's own synthetic setting (12 accumulations of 0.45 s + eps): parity with the oracle, and the
+    scale-graph helper.  The printed E[T]/E[T_i] values are only a plausibility band (the worker count
+    behind them is not printed), so the check on them is loose on purpose."""
+    from paper_2306_10598_b200 import scale_graph
+    w = W.c3_workload("exponential_0.05", N=768, T=96, K=64)
+    lat_d = W.fill_latencies(w, "cuda")
+    taus = W.make_taus(w)
+    res = run_gpu(api, lat_d, torch.from_numpy(taus).cuda(), w.t_comm)
+    ref = oracle.sweep(lat_d.cpu().numpy(), taus, w.t_comm)
+    compare_sweep(res, ref, "c3 exponential")
+    compare_stats(res, ref, w.N, w.M, what="c3 exponential")
+    row = scale_graph.scale_row("exponential_0.05", 768, 256, 64, 0.5)
+    assert 1.25 < row["E[T]/E[T_i]"] < 1.55                   # paper prints 1.386 for this law
+    small = scale_graph.scale_row("exponential_0.05", 8, 256, 64, 0.5)
+    assert small["E[T]/E[T_i]"] < row["E[T]/E[T_i]"]           # grows with the number of workers (Sec. 4.2)
+    assert row["s_eff"] >= 1.0 and 0.0 <= row["drop_rate"] < 0.5
+    assert abs(row["s_eff_closed_form_given_E[T]"] - row["s_eff"]) < 0.1 * row["s_eff"]

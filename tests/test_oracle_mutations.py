@@ -33,6 +33,9 @@ MUTANTS = [
     ("thr_mean_is_ratio_of_means", [("sum_ratio / (double)T", "((double)sum_done / sum_step)", 1)]),
     ("argmax_takes_last", [("v > objective[best]", "v >= objective[best]", 1)]),
     ("comm_time_of_wrong_iteration", [("t_comm_per_iter ? t_comm_per_iter[i] : t_comm", "t_comm_per_iter ? t_comm_per_iter[0] : t_comm", 2)]),
+    ("bailey_weights_swapped", [("(1.0 - g) * dco_phi_inv(1.0 - 1.0 / (double)N) + g * dco_phi_inv(", "g * dco_phi_inv(1.0 - 1.0 / (double)N) + (1.0 - g) * dco_phi_inv(", 1)]),
+    ("eq5_variance_not_scaled_by_m", [("sqrt((double)m * sigma * sigma)", "sqrt(sigma * sigma)", 1)]),
+    ("eq11_numerator_without_comm", [("* (ET + t_comm) / step", "* ET / step", 1)]),
     ("rule1_inclusive", [("if (before < taus[k]) {", "if (Tin < taus[k]) {", 1),
                          ("if (Tin < tau) {\n                            done += 1;", "if (Tin + t[m] < tau) {\n                            done += 1;", 1)]),
 ]

@@ -80,6 +80,7 @@ struct SweepParams {
     int lut_cells;     // tiled kernel: cells of the bin lookup table (the table has lut_cells + 1 entries)
     int rule;          // DC_RULE_*
     int aux_copies;    // rule 1: copies of the per-threshold worker-time maxima (0 for rule 0)
+    int nbuf;          // histogram / maxima buffers: 2 in the tiled kernel (filled and drained in turn), 1 in the plain one
     int one;           // always 1; a value the compiler cannot see, used to tie a stage release to a warp vote
 };
 
@@ -332,14 +333,14 @@ __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepP
     SmemTail s;
     s.tau_s = reinterpret_cast<float *>(base);
     s.hist = reinterpret_cast<int *>(s.tau_s + (p.K + 1));
-    s.smax = reinterpret_cast<float *>(s.hist + p.hist_copies * p.hist_stride);
+    s.smax = reinterpret_cast<float *>(s.hist + p.nbuf * p.hist_copies * p.hist_stride);
     s.wtot = reinterpret_cast<int *>(s.smax + 32);
     s.meta = s.wtot + 32;
     s.lut = reinterpret_cast<unsigned short *>(s.meta + 8);
     s.wmx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(s.lut) +
                                       (((size_t)(p.lut_cells + 1) * sizeof(unsigned short) + 3) & ~(size_t)3));
     s.wmax = s.wmx + 32;
-    s.tail = s.wmax + p.aux_copies * (p.K + 2);
+    s.tail = s.wmax + p.nbuf * p.aux_copies * (p.K + 2);
     return s;
 }
 __host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride, int lut_cells, int aux_copies)
@@ -353,8 +354,8 @@ __device__ __forceinline__ void load_thresholds(const SweepParams &p, const Smem
 {
     for (int k = tid; k < p.K; k += nthr) s.tau_s[k] = p.taus[k];
     if (tid == 0) s.tau_s[p.K] = __int_as_float(0x7f800000);  // +inf sentinel
-    for (int i = tid; i < p.hist_copies * p.hist_stride; i += nthr) s.hist[i] = 0;
-    for (int i = tid; i < 2 * p.aux_copies * (p.K + 2); i += nthr) s.wmax[i] = 0.0f;  // wmax and tail are adjacent
+    for (int i = tid; i < p.nbuf * p.hist_copies * p.hist_stride; i += nthr) s.hist[i] = 0;
+    for (int i = tid; i < 2 * p.nbuf * p.aux_copies * (p.K + 2); i += nthr) s.wmax[i] = 0.0f;  // wmax and tail are adjacent
 }
 
 // ------------------------------------------------------------------------------------------
@@ -450,15 +451,121 @@ __device__ __forceinline__ void start_rule_sample(float P, unsigned &prev, float
 }
 
 // ------------------------------------------------------------------------------------------
-// Tiled kernel: TMA-staged rows, one producer warp + consumer warps, persistent over trials.
+// Tiled kernel: TMA-staged rows, persistent over trials.  Warp roles inside a block:
+//   warps 0 .. ncw-1   consumers: thread r owns row (pass*rows + r) of the current trial
+//   warp  ncw          producer: one thread streams the block's tiles through the ring of stages
+//   warp  ncw+1        epilogue: turns a finished trial's histograms into out_done / out_step / out_sync
+// The histograms (and the per-warp maxima) are double-buffered: consumers fill buffer j&1 for their j-th
+// trial and go straight on to the next trial while the epilogue warp sums, scans, writes and clears the
+// buffer.  Named barriers hand the buffers over: kBarReady+b (consumers arrive, epilogue waits) and
+// kBarFree+b (epilogue arrives, consumers wait before reusing the buffer two trials later).
 // NQ = 16-byte quads of a row per chunk held in registers (box width = 4*NQ floats at most).
-// A consumer thread adds its row's samples in order, eight at a time.  If after a group every
-// lane of the warp is still below the first threshold the eight samples are bin 0 (one register
-// add); if before the group every lane is at or above the last threshold they are in the bin
-// nobody reads; otherwise each running sum is binned through the lookup table.
+// A consumer thread adds its row's samples in order; per group of eight, if every lane of the warp is
+// still below the first threshold the samples are bin 0 (one register add); if every lane is at or
+// above the last threshold they are in the bin nobody reads; otherwise each running sum is binned
+// through the lookup table.
 // ------------------------------------------------------------------------------------------
+constexpr int kBarReady = 2;  // +0, +1
+constexpr int kBarFree = 4;   // +0, +1
+
+// Barrier numbers are compile-time immediates (a run-time number would make the compiler reserve all 16
+// hardware barriers for every block); b selects between the two buffers' barriers.
+template <int ID>
+__device__ __forceinline__ void bar_sync_imm(int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"n"(ID), "r"(threads) : "memory");
+}
+template <int ID>
+__device__ __forceinline__ void bar_arrive_imm(int threads)
+{
+    asm volatile("bar.arrive %0, %1;" ::"n"(ID), "r"(threads) : "memory");
+}
+template <int BASE>
+__device__ __forceinline__ void buffer_barrier_sync(int b, int threads)
+{
+    if (b == 0) bar_sync_imm<BASE>(threads);
+    else bar_sync_imm<BASE + 1>(threads);
+}
+template <int BASE>
+__device__ __forceinline__ void buffer_barrier_arrive(int b, int threads)
+{
+    if (b == 0) bar_arrive_imm<BASE>(threads);
+    else bar_arrive_imm<BASE + 1>(threads);
+}
+
+// The epilogue warp's loop (all 32 lanes).  Bins are taken 32 at a time: lane l sums bin k0+l over the
+// copies (and clears it), a warp scan gives the prefix, a carry links the blocks of 32.
+template <int RULE>
+__device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTail &s, int lane, int ncw)
+{
+    const int K = p.K, H = p.hist_copies, HS = p.hist_stride, A = p.aux_copies, AS = K + 2;
+    const int bar_threads = ncw * 32 + 32;
+    int j = 0;
+    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
+        const int b = j & 1;
+        buffer_barrier_sync<kBarReady>(b, bar_threads);  // every consumer has finished trial t
+        int *hist = s.hist + b * H * HS;
+        float *wmax = s.wmax + b * A * AS;
+        float *tail = s.tail + b * A * AS;
+        const float Tmax = warp_max(lane < ncw ? s.smax[32 * b + lane] : 0.0f);
+        const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
+        float *step_row = p.out_step + t * K;
+        int32_t *done_row = p.out_done + t * K;
+        int carry = 0;
+        float tail_carry = 0.0f;
+        for (int k0 = 0; k0 < K; k0 += 32) {
+            const int k = k0 + lane;
+            int h = 0;
+            float tl = 0.0f, w = 0.0f;
+            if (k < K) {
+                for (int c = 0; c < H; ++c) {
+                    h += hist[c * HS + k];
+                    hist[c * HS + k] = 0;
+                }
+                if (RULE == 1) {
+                    for (int c = 0; c < A; ++c) {
+                        tl = fmaxf(tl, tail[c * AS + k]);
+                        w = fmaxf(w, wmax[c * AS + k]);
+                        tail[c * AS + k] = 0.0f;
+                        wmax[c * AS + k] = 0.0f;
+                    }
+                }
+            }
+            const int incl = warp_inclusive_scan(h, lane);
+            float step;
+            if (RULE == 0) {
+                step = __fadd_rn(fminf(k < K ? s.tau_s[k] : 0.0f, Tmax), t_comm);
+            } else {
+                // max_n W_n(k) = max(wmax[k], max_{j <= k} tail[j])
+                const float tl_incl = warp_inclusive_max_scan(tl, lane);
+                step = __fadd_rn(fmaxf(w, fmaxf(tail_carry, tl_incl)), t_comm);
+                tail_carry = fmaxf(tail_carry, __shfl_sync(0xffffffffu, tl_incl, 31));
+            }
+            if (k < K) {
+                done_row[k] = carry + incl;
+                step_row[k] = step;
+            }
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        for (int c = lane; c < H; c += 32) {  // the two bins past the last threshold
+            hist[c * HS + K] = 0;
+            hist[c * HS + K + 1] = 0;
+        }
+        if (RULE == 1) {
+            for (int c = lane; c < A; c += 32) {
+                tail[c * AS + K] = 0.0f;
+                tail[c * AS + K + 1] = 0.0f;
+                wmax[c * AS + K] = 0.0f;
+                wmax[c * AS + K + 1] = 0.0f;
+            }
+        }
+        if (lane == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
+        buffer_barrier_arrive<kBarFree>(b, bar_threads);  // buffer b is clear again
+    }
+}
+
 template <int NQ, int RULE>
-__global__ void __launch_bounds__(kMaxRowsPerPass + 32, 2)
+__global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2)
 dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 {
     extern __shared__ unsigned char smem_raw[];
@@ -471,7 +578,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     const SmemTail s = carve_tail(reinterpret_cast<unsigned char *>(empty + kMaxStages), p);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int ncw = (blockDim.x >> 5) - 1;  // consumer warps; the last warp is the producer
+    const int ncw = (blockDim.x >> 5) - 2;  // consumer warps; then the producer warp, then the epilogue warp
     const int S = p.stages;
 
     if (tid == 0) {
@@ -487,57 +594,78 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     build_lut(p, s, tid, blockDim.x);
 
     if (warp == ncw) {
-        // ---------------- producer: one thread streams this block's tiles through the ring
+        // ---------------- producer
         if (lane == 0) {
-            uint32_t i = 0;
+            int st = 0;
+            uint32_t ph = 0;       // parity of the current use of stage st
+            bool first = true;     // the first S tiles find their stage empty
             for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
                 for (int pass = 0; pass < p.passes; ++pass) {
-                    for (int c = 0; c < p.chunks; ++c, ++i) {
-                        const int st = i % S;
-                        const uint32_t use = i / S;
-                        if (use > 0) mbar_wait(&empty[st], (use & 1u) ^ 1u, kErrStageNeverFreed);
+                    for (int c = 0; c < p.chunks; ++c) {
+                        if (!first) mbar_wait(&empty[st], ph ^ 1u, kErrStageNeverFreed);
                         mbar_arrive_expect_tx(&full[st], (uint32_t)(p.rows * p.pitch));
                         tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, c * p.bw, pass * p.rows, (int)t, &full[st]);
+                        if (++st == S) {
+                            st = 0;
+                            ph ^= 1u;
+                            first = false;
+                        }
                     }
                 }
             }
         }
         return;
     }
+    if (warp == ncw + 1) {
+        epilogue_warp<RULE>(p, s, lane, ncw);
+        return;
+    }
 
-    // ---------------- consumers: thread r owns row (pass*rows + r) of the current trial
+    // ---------------- consumers
     constexpr int GQ = NQ >= 2 ? 2 : 1;  // quads per group
-    const int nthr = ncw * 32;
+    const int bar_threads = ncw * 32 + 32;
     const int K = p.K;
-    int *myhist = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
-    unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
+    const int hist_buf_ints = p.hist_copies * p.hist_stride;
+    const int aux_buf_floats = p.aux_copies * (K + 2);
+    int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
     const unsigned char *tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
     const unsigned K4 = 4u * (unsigned)K;
     const bool one = s.meta[0] != 0;
     const float lut_lo = __int_as_float(s.meta[1]), lut_scale = __int_as_float(s.meta[2]);
     const unsigned C = (unsigned)p.lut_cells;
     const float tau_first = s.tau_s[0], tau_last = s.tau_s[K - 1];
-    // rule 1 only: this thread's copies of the worker-time maxima, and the bin of a running time of 0
-    unsigned char *wmax_b = reinterpret_cast<unsigned char *>(s.wmax + (p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0));
-    float *mytail = s.tail + (p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0);
+    // rule 1 only: this thread's copy of the worker-time maxima, and the bin of a running time of 0
+    const int aux_off = p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0;
     unsigned off_zero = 0;
     if (RULE == 1) off_zero = bin_offset<false>(0.0f, lut_lo, lut_scale, C, s.lut, tau_b, K4);
     // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
     // (threads past the last row of the box read the last row instead: always inside the stage)
     const uint32_t row_off = (uint32_t)min(tid, p.rows - 1) * (uint32_t)p.pitch;
     const uint32_t swz = ((row_off >> 7) & (uint32_t)p.swz_mask) << 4;
-    uint32_t i = 0;
-    for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
+    int st = 0;
+    uint32_t ph = 0;
+    int j = 0;
+    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
+        const int b = j & 1;
+        if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
+        int *myhist = myhist0 + b * hist_buf_ints;
+        unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
+        unsigned char *wmax_b = reinterpret_cast<unsigned char *>(s.wmax + b * aux_buf_floats + aux_off);
+        float *mytail = s.tail + b * aux_buf_floats + aux_off;
         float rowmax = 0.0f;
         int cnt0 = 0;
         for (int pass = 0; pass < p.passes; ++pass) {
             const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
             float P = 0.0f;
             unsigned prev = off_zero;  // rule 1: bin (byte offset) of the running time before the next micro-batch
-            for (int c = 0; c < p.chunks; ++c, ++i) {
-                const int st = i % S;
-                mbar_wait(&full[st], (i / S) & 1u, kErrLoadNeverArrived);
+            for (int c = 0; c < p.chunks; ++c) {
+                mbar_wait(&full[st], ph, kErrLoadNeverArrived);
                 const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes + row_off;
+                uint64_t *empty_bar = &empty[st];
+                if (++st == S) {
+                    st = 0;
+                    ph ^= 1u;
+                }
                 const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
                 float4 v[NQ];
 #pragma unroll
@@ -559,7 +687,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                 // the stage is released only after it, and the count operand of the arrive depends on the vote
                 // (p.one is 1), so the release cannot move ahead of the reads.
                 const bool chunk_low = __all_sync(0xffffffffu, !valid || P < tau_first);
-                if (lane == 0) mbar_arrive_count(&empty[st], chunk_low ? 1u : (uint32_t)p.one);
+                if (lane == 0) mbar_arrive_count(empty_bar, chunk_low ? 1u : (uint32_t)p.one);
                 if (chunk_low) {
                     if (valid) cnt0 += 4 * nq;
                     continue;
@@ -629,7 +757,9 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
             }
         }
         if (cnt0 > 0) atomicAdd(myhist, cnt0);
-        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot, s.wmax, s.tail, s.wmx);
+        rowmax = warp_max(rowmax);
+        if (lane == 0) s.smax[32 * b + warp] = rowmax;
+        buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
     }
 }
 
@@ -1018,6 +1148,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.warp_groups = 1;
     p.lut_cells = 0;
     p.one = 1;
+    p.nbuf = 1;
     p.rule = rule;
     p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? 1 : 0;
 
@@ -1040,28 +1171,37 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         // Shared memory per block: aim at two resident blocks per SM.  Histogram copies: lane l of warp w
         // adds into copy (w % warp_groups) * lane_copies + (l % lane_copies); copies used by one warp start
         // 32 / lane_copies banks apart so that equal bins of different lanes do not collide.
+        p.nbuf = 2;
         const int ncw = row_threads / 32;
         const size_t budget = (size_t)di.smem_per_sm / 2 - 1024 - 256;
         size_t smem = 0;
         bool fits = false;
+        // candidates from the preferred configuration down to the smallest one; the first that leaves room
+        // for two blocks per SM wins, and the smallest one is taken even if only one block fits
         const int lc_first = g_tune_lane_copies > 0 ? g_tune_lane_copies : 4;
+        const int wg_first = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
         for (int lc = lc_first; lc >= 1 && !fits; lc >>= 1) {
-            p.lane_copies = lc;
-            p.warp_groups = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
-            p.hist_copies = p.warp_groups * lc;
-            if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = p.warp_groups;
-            const int want = lc > 1 ? 32 / lc : 1;
-            p.hist_stride = K + 2;
-            while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
-            const size_t fixed = 1024 + 2 * kMaxStages * sizeof(uint64_t) + tail_bytes(K, p.hist_copies, p.hist_stride, p.lut_cells, p.aux_copies);
-            const int s_max = g_tune_stages > 0 ? g_tune_stages : min(kMaxStages, max(2, kStageBudgetBytes / p.stage_bytes));
-            for (int st = s_max; st >= 2; --st) {
-                smem = fixed + (size_t)st * p.stage_bytes;
-                if (smem <= budget || (lc == 1 && st == 2) || g_tune_stages > 0) {
-                    p.stages = st;
-                    fits = true;
-                    break;
+            for (int wg = wg_first; wg >= 1 && !fits; wg >>= 1) {
+                p.lane_copies = lc;
+                p.warp_groups = wg;
+                p.hist_copies = wg * lc;
+                if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = wg;
+                const int want = lc > 1 ? 32 / lc : 1;
+                p.hist_stride = K + 2;
+                while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
+                const size_t fixed = 1024 + 2 * kMaxStages * sizeof(uint64_t) +
+                                     tail_bytes(K, p.nbuf * p.hist_copies, p.hist_stride, p.lut_cells, p.nbuf * p.aux_copies);
+                const int s_max = g_tune_stages > 0 ? g_tune_stages : min(kMaxStages, max(2, kStageBudgetBytes / p.stage_bytes));
+                const bool last = (lc == 1 && wg == 1);
+                for (int st = s_max; st >= 2; --st) {
+                    smem = fixed + (size_t)st * p.stage_bytes;
+                    if (smem <= budget || (last && st == 2) || g_tune_stages > 0) {
+                        p.stages = st;
+                        fits = true;
+                        break;
+                    }
                 }
+                if (g_tune_warp_groups > 0) break;
             }
             if (g_tune_lane_copies > 0) break;
         }
@@ -1078,7 +1218,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
             return DC_ERR_CUDA;
 
         if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
-        const int block = row_threads + 32;
+        const int block = row_threads + 64;
         const int nq = p.bw / 4;
         int lrc;
         if (rule == DC_RULE_FINISH_BEFORE_TAU) {
@@ -1437,7 +1577,7 @@ int dc_simulate_launches(void) { return g_last_simulate_launches; }
 int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
 int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
 
-const char *dc_kernel_version(void) { return "sweep-tiled-6"; }
+const char *dc_kernel_version(void) { return "sweep-tiled-7"; }
 
 const char *dc_status_string(int status)
 {

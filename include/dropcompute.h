@@ -242,6 +242,8 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  *   DC_TUNE_STAGES       depth of the shared-memory ring the tiled kernel streams rows through (2..8)
  *   DC_TUNE_LANE_COPIES  histogram copies a warp spreads its lanes over in the tiled kernel (1, 2, 4 or 8)
  *   DC_TUNE_WARP_GROUPS  groups of warps with histogram copies of their own (1..8)
+ *   DC_TUNE_BATCH_LOOKUPS 1 = bin each running sum and update the histogram at once, 2 = look up the bins of a
+ *                        whole group of eight first (lower latency, better for trials that fit one tile)
  *   DC_TUNE_BOX_FLOATS   floats of a row fetched per tile (16 or 32; 16 needs M to be a multiple of 16)
  * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
  */
@@ -249,6 +251,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
 #define DC_TUNE_LANE_COPIES 2
 #define DC_TUNE_WARP_GROUPS 3
 #define DC_TUNE_BOX_FLOATS 4
+#define DC_TUNE_BATCH_LOOKUPS 5
 int dc_tune(int32_t key, int32_t value);
 
 /* Number of kernel launches the last successful call of each entry point enqueues (for accounting). */

@@ -80,6 +80,7 @@ struct SweepParams {
     int lut_cells;     // tiled kernel: cells of the bin lookup table (the table has lut_cells + 1 entries)
     int rule;          // DC_RULE_*
     int aux_copies;    // rule 1: copies of the per-threshold worker-time maxima (0 for rule 0)
+    int batch_lookups; // tiled kernel: 1 = look up a whole group's bins before updating the histogram
     int nbuf;          // histogram / maxima buffers: 2 in the tiled kernel (filled and drained in turn), 1 in the plain one
     int one;           // always 1; a value the compiler cannot see, used to tie a stage release to a warp vote
 };
@@ -564,7 +565,7 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
     }
 }
 
-template <int NQ, int RULE>
+template <int NQ, int RULE, bool BATCH>
 __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2)
 dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 {
@@ -721,12 +722,29 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                         } else if (!__all_sync(0xffffffffu, !valid || v[g].x >= tau_last)) {
                             if (valid) {
                                 if (one && gq == GQ) {  // the common case, no per-sample predicates
+                                    // all table and threshold reads of the group first (independent chains the
+                                    // hardware can overlap), then the histogram updates
+                                    if (BATCH) {
+                                        // all table and threshold reads of the group first (independent chains
+                                        // that overlap), then the histogram updates: lower latency per group
+                                        unsigned off[4 * GQ];
 #pragma unroll
-                                    for (int q = 0; q < GQ; ++q) {
-                                        bin_sample<true>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                        bin_sample<true>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                        bin_sample<true>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                        bin_sample<true>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                        for (int q = 0; q < GQ; ++q) {
+                                            off[4 * q + 0] = bin_offset<true>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4);
+                                            off[4 * q + 1] = bin_offset<true>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4);
+                                            off[4 * q + 2] = bin_offset<true>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4);
+                                            off[4 * q + 3] = bin_offset<true>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4);
+                                        }
+#pragma unroll
+                                        for (int e = 0; e < 4 * GQ; ++e) atomicAdd(reinterpret_cast<int *>(hist_b + off[e]), 1);
+                                    } else {
+#pragma unroll
+                                        for (int q = 0; q < GQ; ++q) {
+                                            bin_sample<true>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                            bin_sample<true>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                            bin_sample<true>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                            bin_sample<true>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
+                                        }
                                     }
                                 } else {
 #pragma unroll
@@ -1082,6 +1100,7 @@ int g_tune_stages = 0;       // 0 = automatic
 int g_tune_lane_copies = 0;  // 0 = automatic
 int g_tune_warp_groups = 0;  // 0 = automatic
 int g_tune_box_floats = 0;   // 0 = automatic
+int g_tune_batch = 0;        // 0 = automatic, 1 = off, 2 = on
 int g_last_simulate_launches = 0;
 int g_last_reduce_launches = 0;
 int g_last_argmax_launches = 0;
@@ -1102,17 +1121,26 @@ int validate_simulate(const float *lat, int64_t T, int64_t N, int64_t M, const f
 
 bool tiled_ok(const float *lat, int64_t M) { return (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0); }
 
-template <int NQ, int RULE>
-int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
-                 cudaStream_t stream)
+template <int NQ, int RULE, bool BATCH>
+int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
+                   cudaStream_t stream)
 {
-    auto kernel = dc_sweep_tiled<NQ, RULE>;
+    auto kernel = dc_sweep_tiled<NQ, RULE, BATCH>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
     const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
     kernel<<<(unsigned)grid, block, smem, stream>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+template <int NQ, int RULE>
+int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
+                 cudaStream_t stream)
+{
+    // rule 1 has one binning path only
+    if (RULE == 0 && p.batch_lookups) return launch_tiled_b<NQ, RULE, true>(map, p, block, smem, T, di, stream);
+    return launch_tiled_b<NQ, RULE, false>(map, p, block, smem, T, di, stream);
 }
 
 int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
@@ -1149,6 +1177,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.lut_cells = 0;
     p.one = 1;
     p.nbuf = 1;
+    p.batch_lookups = 0;
     p.rule = rule;
     p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? 1 : 0;
 
@@ -1168,6 +1197,9 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         else if (p.pitch == 32) { swz = CU_TENSOR_MAP_SWIZZLE_32B; p.swz_mask = 1; }
         p.stage_bytes = ((p.rows * p.pitch + 1023) / 1024) * 1024;
         p.lut_cells = min(kLutCellsMax, 4 * K);
+        // Rows that fit one tile gain from looking up a whole group's bins before touching the histogram (the
+        // chains overlap); longer rows measured faster with lookups and updates interleaved.
+        p.batch_lookups = g_tune_batch > 0 ? g_tune_batch - 1 : (p.chunks == 1 ? 1 : 0);
         // Shared memory per block: aim at two resident blocks per SM.  Histogram copies: lane l of warp w
         // adds into copy (w % warp_groups) * lane_copies + (l % lane_copies); copies used by one warp start
         // 32 / lane_copies banks apart so that equal bins of different lanes do not collide.
@@ -1176,34 +1208,34 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         const size_t budget = (size_t)di.smem_per_sm / 2 - 1024 - 256;
         size_t smem = 0;
         bool fits = false;
-        // candidates from the preferred configuration down to the smallest one; the first that leaves room
-        // for two blocks per SM wins, and the smallest one is taken even if only one block fits
+        // Candidates: ring depth first (bytes in flight matter most), then histogram copies, from the
+        // preferred configuration down to the smallest one.  The first that leaves room for two blocks per
+        // SM wins; the smallest one is taken even if only one block fits.
+        // (a ring deeper than three tiles measured slower on every workload, whatever the tile size)
+        const int s_max = g_tune_stages > 0 ? g_tune_stages : min(3, max(2, kStageBudgetBytes / p.stage_bytes));
+        const int s_min = g_tune_stages > 0 ? g_tune_stages : 2;
         const int lc_first = g_tune_lane_copies > 0 ? g_tune_lane_copies : 4;
+        const int lc_last = g_tune_lane_copies > 0 ? g_tune_lane_copies : 1;
         const int wg_first = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
-        for (int lc = lc_first; lc >= 1 && !fits; lc >>= 1) {
-            for (int wg = wg_first; wg >= 1 && !fits; wg >>= 1) {
-                p.lane_copies = lc;
-                p.warp_groups = wg;
-                p.hist_copies = wg * lc;
-                if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = wg;
-                const int want = lc > 1 ? 32 / lc : 1;
-                p.hist_stride = K + 2;
-                while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
-                const size_t fixed = 1024 + 2 * kMaxStages * sizeof(uint64_t) +
-                                     tail_bytes(K, p.nbuf * p.hist_copies, p.hist_stride, p.lut_cells, p.nbuf * p.aux_copies);
-                const int s_max = g_tune_stages > 0 ? g_tune_stages : min(kMaxStages, max(2, kStageBudgetBytes / p.stage_bytes));
-                const bool last = (lc == 1 && wg == 1);
-                for (int st = s_max; st >= 2; --st) {
-                    smem = fixed + (size_t)st * p.stage_bytes;
-                    if (smem <= budget || (last && st == 2) || g_tune_stages > 0) {
-                        p.stages = st;
-                        fits = true;
-                        break;
-                    }
+        const int wg_last = g_tune_warp_groups > 0 ? wg_first : 1;
+        const bool forced = g_tune_stages > 0 && g_tune_lane_copies > 0 && g_tune_warp_groups > 0;
+        for (int st = s_max; st >= s_min && !fits; --st) {
+            for (int lc = lc_first; lc >= lc_last && !fits; lc >>= 1) {
+                for (int wg = wg_first; wg >= wg_last && !fits; wg >>= 1) {
+                    p.stages = st;
+                    p.lane_copies = lc;
+                    p.warp_groups = wg;
+                    p.hist_copies = wg * lc;
+                    if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = wg;
+                    const int want = lc > 1 ? 32 / lc : 1;
+                    p.hist_stride = K + 2;
+                    while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
+                    smem = 1024 + 2 * kMaxStages * sizeof(uint64_t) + (size_t)st * p.stage_bytes +
+                           tail_bytes(K, p.nbuf * p.hist_copies, p.hist_stride, p.lut_cells, p.nbuf * p.aux_copies);
+                    const bool smallest = (st == s_min && lc == lc_last && wg == wg_last);
+                    if (smem <= budget || smallest || forced) fits = true;
                 }
-                if (g_tune_warp_groups > 0) break;
             }
-            if (g_tune_lane_copies > 0) break;
         }
         if (!fits) return DC_ERR_RANGE;
 
@@ -1566,6 +1598,10 @@ int dc_tune(int32_t key, int32_t value)
         g_tune_warp_groups = value;
         return DC_OK;
     }
+    if (key == DC_TUNE_BATCH_LOOKUPS && value >= 0 && value <= 2) {
+        g_tune_batch = value;
+        return DC_OK;
+    }
     if (key == DC_TUNE_BOX_FLOATS && (value == 0 || value == 16 || value == 32)) {
         g_tune_box_floats = value;
         return DC_OK;
@@ -1577,7 +1613,7 @@ int dc_simulate_launches(void) { return g_last_simulate_launches; }
 int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
 int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
 
-const char *dc_kernel_version(void) { return "sweep-tiled-7"; }
+const char *dc_kernel_version(void) { return "sweep-tiled-8"; }
 
 const char *dc_status_string(int status)
 {

@@ -76,7 +76,9 @@ typedef enum {
  *   out_done[t][k] = #{ (n,m) : P_{t,n,m} < taus[k] }          (= N * M~_t(tau_k); strict '<', fp32)
  *   out_step[t][k] = fl32( fminf(taus[k], max_n P_{t,n,M-1}) + t_comm )   (= min{tau,T} + T^c)
  *
- *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; 16-byte aligned; finite and >= 0
+ *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; finite and >= 0.  16-byte aligned with M a
+ *              multiple of 4 takes the fast (tiled) kernel; any 4-byte aligned pointer and any M are
+ *              accepted and take the plain-load kernel (see dc_simulate_plan)
  *   T, N, M    > 0, N*M <= INT32_MAX
  *   taus       DEVICE, [K] fp32, non-decreasing, no NaN; +infinity is allowed (gives the
  *              synchronous baseline); 4-byte aligned.  1 <= K <= DC_MAX_K

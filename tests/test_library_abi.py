@@ -64,6 +64,20 @@ def test_argument_errors_need_no_gpu(lib):
     assert lib.dc_simulate_plan(A, 4, 8, 13, 3) == 1
     assert lib.dc_simulate_plan(A + 4, 4, 8, 12, 3) == 1
     assert lib.dc_simulate_plan(A, 4, 8, 12, 5000) == -4
+    # the later entry points
+    assert lib.dc_simulate_tc(A, 1, 1, 1, A, 1, None, A, A, None, 0, None) == 1          # per-trial times missing
+    assert lib.dc_simulate_tc(A, 1, 1, 1, A, 1, A + 2, A, A, None, 0, None) == 3
+    assert lib.dc_reduce_trials_static(A, A, A, 4, 1025, 1, 1, A, A, None) == 4           # beyond the built-in scratch
+    assert lib.dc_reduce_trials_static(A, A, A, 0, 4, 1, 1, A, A, None) == 2
+    d = ctypes.c_double
+    assert lib.dc_closed_form(d(1.0), d(0.1), 4, 1, d(0.1), d(-1.0), A, 4, A, A, None) == 2   # needs N >= 2
+    assert lib.dc_closed_form(d(1.0), d(0.0), 4, 8, d(0.1), d(-1.0), A, 4, A, A, None) == 4   # sigma must be > 0
+    assert lib.dc_closed_form(d(1.0), d(0.1), 4, 8, d(0.1), d(-1.0), None, 4, A, A, None) == 1
+    # tuning knobs: unknown keys and values are refused, 0 always restores the default
+    assert lib.dc_tune(1, 9) == 7 and lib.dc_tune(2, 3) == 7 and lib.dc_tune(99, 0) == 7
+    for key in (1, 2, 3, 4, 5):
+        assert lib.dc_tune(key, 0) == 0
+    assert lib.dc_kernel_version().startswith(b"sweep-")
 
 
 def test_workspace_sizes(lib):

@@ -247,7 +247,7 @@ def run_ours(args, w: W.Workload):
             flush.zero_()
         if ev:
             ev[0].record()
-        api.dc_simulate_ex(lat, taus, wr.t_comm, out_step, out_done, out_sync)
+        api.dc_simulate_ex(lat, taus, wr.t_comm, out_step, out_done, out_sync, args.rule)
         if ev:
             ev[1].record()
         api.dc_reduce_trials(out_step, out_done, out_sync, N, M, stats, baseline, ws)
@@ -299,7 +299,7 @@ def run_ours(args, w: W.Workload):
         "config": {"workload": w.name, "T": T, "N": N, "M": M, "K": K, "t_comm": wr.t_comm,
                    "latency_bytes": wr.latency_bytes,
                    "l2": "inputs larger than L2" if flush is None else "256 MiB buffer written between steps",
-                   "parallelism": f"{world} x independent trials"},
+                   "parallelism": f"{world} x independent trials", "rule": args.rule},
         "hbm_gbs": achieved,
         "sweep_ms": sim_avg_s * 1e3,
         "sweep_ms_best": min(sim_ms),
@@ -369,6 +369,8 @@ def main():
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--workload", default="bandwidth_stress", choices=sorted(W.WORKLOADS))
     ap.add_argument("--trials", type=int, default=0, help="override the number of trials (profiling small cases)")
+    ap.add_argument("--rule", type=int, default=0, choices=(0, 1),
+                    help="completion rule: 0 = Algorithm 2 (finish before tau, the benchmark), 1 = start before tau")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -176,11 +176,26 @@ struct RowWalk {
     }
 };
 
-// Non-negative floats order like their bit patterns, so an integer atomicMax is an exact float max.  The
-// plain read first makes the atomic rare: a maximum over thousands of workers changes only a few times.
-__device__ __forceinline__ void float_max_nonneg(float *slot, float v)
+// Start-before-tau rule: the per-threshold maximum over workers of W_n(k), kept as an "envelope" env[k].
+// For one worker W_n(k) is a non-decreasing step function of k, so the maximum over workers is non-decreasing
+// too.  A worker raises env over a range [a, b) to the value V it has there by walking k upward and stopping
+// at the first k where env[k] >= V already: from there on some other worker q holds a value W_q(k) >= V, and
+// since W_q is non-decreasing and q itself walks on to every later k, everything to the right ends >= V as
+// well (entries only ever grow).  In the common case this is ONE read per range.  Non-negative floats order
+// like their bit patterns, so the integer atomicMax is an exact float max.
+// The thresholds a worker never reaches (k >= its last bin j) all get its total T_n.  Instead of walking that
+// range, the worker records T_n once in tail[j]; the epilogue takes max(env[k], max_{j <= k} tail[j]).  The
+// stopping argument above still holds with "q walks on or q's tail entry covers the rest".
+__device__ __forceinline__ void record_tail(float *tail, int j, float V)
 {
-    if (v > *reinterpret_cast<volatile float *>(slot)) atomicMax(reinterpret_cast<int *>(slot), __float_as_int(v));
+    if (V > *reinterpret_cast<volatile float *>(tail + j)) atomicMax(reinterpret_cast<int *>(tail + j), __float_as_int(V));
+}
+__device__ __forceinline__ void raise_envelope(float *env, int a, int b, float V)
+{
+    for (int k = a; k < b; ++k) {
+        if (*reinterpret_cast<volatile float *>(env + k) >= V) break;
+        atomicMax(reinterpret_cast<int *>(env + k), __float_as_int(V));
+    }
 }
 
 // Start-before-tau rule, one worker's row with a forward cursor (plain-load kernel).  Micro-batch m is run iff
@@ -195,18 +210,18 @@ struct RowWalkStart {
         cur = 0;
         while (cur < K && 0.0f >= tau_s[cur]) ++cur;
     }
-    __device__ __forceinline__ void step(float x, const float *tau_s, int *hist, float *wmax, int K)
+    __device__ __forceinline__ void step(float x, const float *tau_s, int *hist, float *env, int K)
     {
         atomicAdd(&hist[cur], 1);  // P_{m-1} is in bin cur
         P = __fadd_rn(P, x);
-        while (cur < K && P >= tau_s[cur]) {  // thresholds first reached by this micro-batch
-            float_max_nonneg(&wmax[cur], P);
-            ++cur;
-        }
+        int nc = cur;
+        while (nc < K && P >= tau_s[nc]) ++nc;  // thresholds cur .. nc-1 are first reached by this micro-batch
+        raise_envelope(env, cur, nc, P);
+        cur = nc;
     }
-    __device__ __forceinline__ void finish(float *tail, int K)
+    __device__ __forceinline__ void finish(float *tail)
     {
-        if (cur < K) float_max_nonneg(&tail[cur], P);  // thresholds cur.. were never reached: W = row total
+        record_tail(tail, cur, P);  // thresholds cur.. were never reached: W = row total (tail has K + 2 entries)
     }
 };
 
@@ -241,9 +256,8 @@ __device__ __forceinline__ int warp_inclusive_scan(int v, int lane)
 // T = max_n T_n, writes step[t][k] = min(tau_k, T) + T^c and sync[t] = T + T^c, and clears the
 // histograms for the next trial.
 // ------------------------------------------------------------------------------------------
-// Rule 1 (start-before-tau): step[t][k] = max_n W_n(k) + T^c with
-//   max_n W_n(k) = max( wmax[k], max_{j <= k} tail[j] )
-// (wmax[k]: largest first-reaching running sum; tail[j]: largest total among workers that stopped at bin j).
+// Rule 1 (start-before-tau): step[t][k] = max_n W_n(k) + T^c, the maximum being the envelope wmax[] (see
+// raise_envelope).
 __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t, float rowmax, int tid, int nthr,
                                                int barrier_id, const float *tau_s, int *hist, float *smax, int *wtot,
                                                float *wmax, float *tail, float *wmx)
@@ -303,8 +317,8 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
             for (int c = 0; c < A; ++c) {
                 tail_run = fmaxf(tail_run, tail[c * AS + b]);
                 w = fmaxf(w, wmax[c * AS + b]);
-                tail[c * AS + b] = 0.0f;
                 wmax[c * AS + b] = 0.0f;
+                tail[c * AS + b] = 0.0f;
             }
             step_row[b] = __fadd_rn(fmaxf(w, tail_run), t_comm);
         }
@@ -313,6 +327,11 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
         hist[c * HS + K] = 0;
         if (HS > K + 1) hist[c * HS + K + 1] = 0;
     }
+    if (rule1)
+        for (int c = tid; c < A; c += nthr) {
+            tail[c * AS + K] = 0.0f;
+            tail[c * AS + K + 1] = 0.0f;
+        }
     if (tid == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
     named_barrier(barrier_id, nthr);  // histograms cleared, smax/wtot free again
 }
@@ -325,9 +344,9 @@ struct SmemTail {
     int *wtot;
     int *meta;           // [0] lookup table has at most one finite threshold per cell, [1..2] lo, scale (as bits)
     unsigned short *lut; // lut_cells + 1 entries (tiled kernel only)
-    float *wmx;          // rule 1: warp totals of the tail max-scan
-    float *wmax;         // rule 1: [aux_copies][K + 2] largest first-reaching running sum per threshold
-    float *tail;         // rule 1: [aux_copies][K + 2] largest total among workers whose last bin is j
+    float *wmx;          // rule 1, plain kernel: warp totals of the tail max-scan
+    float *wmax;         // rule 1: [nbuf][aux_copies][K + 2] envelope of the workers' times per threshold
+    float *tail;         // rule 1: [nbuf][aux_copies][K + 2] largest total among workers whose last bin is j
 };
 __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepParams &p)
 {
@@ -446,8 +465,7 @@ __device__ __forceinline__ void start_rule_sample(float P, unsigned &prev, float
 {
     const unsigned off = bin_offset<ONE>(P, lo, scale, C, lut, tau_b, K4);
     atomicAdd(reinterpret_cast<int *>(hist_b + prev), 1);
-    const unsigned stop = min(off, K4);
-    for (unsigned o = prev; o < stop; o += 4u) float_max_nonneg(reinterpret_cast<float *>(wmax_b + o), P);
+    raise_envelope(reinterpret_cast<float *>(wmax_b), (int)(prev >> 2), (int)(min(off, K4) >> 2), P);
     prev = off;
 }
 
@@ -517,7 +535,7 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
         for (int k0 = 0; k0 < K; k0 += 32) {
             const int k = k0 + lane;
             int h = 0;
-            float tl = 0.0f, w = 0.0f;
+            float w = 0.0f, tl = 0.0f;
             if (k < K) {
                 for (int c = 0; c < H; ++c) {
                     h += hist[c * HS + k];
@@ -525,10 +543,10 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
                 }
                 if (RULE == 1) {
                     for (int c = 0; c < A; ++c) {
-                        tl = fmaxf(tl, tail[c * AS + k]);
                         w = fmaxf(w, wmax[c * AS + k]);
-                        tail[c * AS + k] = 0.0f;
+                        tl = fmaxf(tl, tail[c * AS + k]);
                         wmax[c * AS + k] = 0.0f;
+                        tail[c * AS + k] = 0.0f;
                     }
                 }
             }
@@ -537,7 +555,7 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
             if (RULE == 0) {
                 step = __fadd_rn(fminf(k < K ? s.tau_s[k] : 0.0f, Tmax), t_comm);
             } else {
-                // max_n W_n(k) = max(wmax[k], max_{j <= k} tail[j])
+                // max_n W_n(k) = max(envelope[k], max_{j <= k} tail[j])
                 const float tl_incl = warp_inclusive_max_scan(tl, lane);
                 step = __fadd_rn(fmaxf(w, fmaxf(tail_carry, tl_incl)), t_comm);
                 tail_carry = fmaxf(tail_carry, __shfl_sync(0xffffffffu, tl_incl, 31));
@@ -554,10 +572,10 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
         }
         if (RULE == 1) {
             for (int c = lane; c < A; c += 32) {
-                tail[c * AS + K] = 0.0f;
-                tail[c * AS + K + 1] = 0.0f;
                 wmax[c * AS + K] = 0.0f;
                 wmax[c * AS + K + 1] = 0.0f;
+                tail[c * AS + K] = 0.0f;
+                tail[c * AS + K + 1] = 0.0f;
             }
         }
         if (lane == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
@@ -771,7 +789,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
             }
             if (valid) {
                 rowmax = fmaxf(rowmax, P);
-                if (RULE == 1 && prev < K4) float_max_nonneg(mytail + (prev >> 2), P);  // thresholds never reached: W = total
+                if (RULE == 1) record_tail(mytail, (int)(prev >> 2), P);  // thresholds never reached: W = total
             }
         }
         if (cnt0 > 0) atomicAdd(myhist, cnt0);
@@ -810,7 +828,7 @@ __global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepPar
                     RowWalkStart w;
                     w.start(s.tau_s, p.K);
                     for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), s.tau_s, myhist, s.wmax, p.K);
-                    w.finish(s.tail, p.K);
+                    w.finish(s.tail);
                     rowmax = fmaxf(rowmax, w.P);
                 }
             }
@@ -1613,7 +1631,7 @@ int dc_simulate_launches(void) { return g_last_simulate_launches; }
 int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
 int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
 
-const char *dc_kernel_version(void) { return "sweep-tiled-8"; }
+const char *dc_kernel_version(void) { return "sweep-tiled-9"; }
 
 const char *dc_status_string(int status)
 {

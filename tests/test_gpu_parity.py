@@ -424,3 +424,49 @@ def test_appendix_c3_workload_and_scale_row(api):
     assert small["E[T]/E[T_i]"] < row["E[T]/E[T_i]"]           # grows with the number of workers (Sec. 4.2)
     assert row["s_eff"] >= 1.0 and 0.0 <= row["drop_rate"] < 0.5
     assert abs(row["s_eff_closed_form_given_E[T]"] - row["s_eff"]) < 0.1 * row["s_eff"]
+
+
+def test_random_shapes_and_grids(api):
+    """Seeded sweep over random shapes, latency laws, grids, both rules and both communication-time forms:
+    every tile geometry (16- to 128-byte rows, ragged last column chunk, several passes, plain-load kernel)
+    against the oracle, bit for bit."""
+    rng = np.random.default_rng(20260601)
+    laws = [("shifted_exp", dict(shift=0.01, mean=0.02)), ("uniform", dict(lo=0.0, hi=0.05)), ("dyadic", dict(hi=12)),
+            ("exp", dict(rate=30.0))]
+    for case in range(70):
+        T = int(rng.integers(1, 12))
+        N = int(rng.choice([1, 2, 7, 31, 32, 33, 100, 255, 256, 257, 600]))
+        M = int(rng.choice([1, 2, 3, 4, 8, 12, 16, 20, 24, 28, 32, 36, 44, 64, 68, 96, 100, 128, 132, 160]))
+        K = int(rng.choice([1, 2, 3, 16, 31, 32, 33, 64, 100, 257, 1000]))
+        law, prm = laws[int(rng.integers(len(laws)))]
+        lat = W.iid_latencies(law, T, N, M, seed=1000 + case, **prm).numpy()
+        kind = int(rng.integers(4))
+        if kind == 0:
+            taus = grid_for(lat, K, seed=case)
+        elif kind == 1:                                   # evenly spaced, like the workloads
+            tot = float(lat.sum(-1).mean())
+            taus = np.linspace(0.5 * tot, 1.5 * tot + 1e-3, K).astype(np.float32)
+        elif kind == 2:                                   # geometric: many thresholds share a table cell
+            tot = float(lat.sum(-1).max()) + 1e-3
+            taus = (tot * np.geomspace(1e-4, 2.0, K)).astype(np.float32)
+        else:                                             # few distinct values, heavy duplication
+            tot = float(lat.sum(-1).max()) + 1e-3
+            taus = np.sort(rng.choice(np.linspace(0, tot, 5), K)).astype(np.float32)
+        rule = int(rng.integers(2))
+        lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+        step = torch.empty((T, K), dtype=torch.float32, device="cuda")
+        done = torch.empty((T, K), dtype=torch.int32, device="cuda")
+        sync = torch.empty((T,), dtype=torch.float32, device="cuda")
+        if rng.integers(2):
+            tc = rng.uniform(0.0, 0.2, T).astype(np.float32)
+            api.dc_simulate_tc(lat_d, taus_d, torch.from_numpy(tc).cuda(), step, done, sync, rule)
+        else:
+            tc = float(np.float32(rng.uniform(0.0, 0.2)))
+            api.dc_simulate_ex(lat_d, taus_d, tc, step, done, sync, rule)
+        torch.cuda.synchronize()
+        ref = oracle.sweep(lat, taus, tc, rule=rule)
+        what = f"case {case}: T,N,M,K={T, N, M, K} law={law} grid={kind} rule={rule}"
+        assert np.array_equal(done.cpu().numpy(), ref.done), what
+        assert np.array_equal(step.cpu().numpy().view(np.uint32), ref.step.view(np.uint32)), what
+        assert np.array_equal(sync.cpu().numpy().view(np.uint32), ref.sync.view(np.uint32)), what
+    api.dc_device_status()

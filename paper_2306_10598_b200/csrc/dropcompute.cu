@@ -1144,9 +1144,29 @@ int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size
                    cudaStream_t stream)
 {
     auto kernel = dc_sweep_tiled<NQ, RULE, BATCH>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
+    // Per instantiation and device: the largest dynamic shared memory opted into so far, and the occupancy of
+    // the last (block, smem) asked for -- repeated calls with one shape then cost no runtime queries.
+    static std::mutex lock;
+    static size_t smem_opted[64] = {};
+    static struct { int block; size_t smem; int occ; } last[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return DC_ERR_CUDA;
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
+    {
+        std::lock_guard<std::mutex> guard(lock);
+        if (smem > smem_opted[dev]) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
+            smem_opted[dev] = smem;
+        }
+        if (last[dev].occ > 0 && last[dev].block == block && last[dev].smem == smem) {
+            occ = last[dev].occ;
+        } else {
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
+            last[dev].block = block;
+            last[dev].smem = smem;
+            last[dev].occ = occ;
+        }
+    }
     const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
     kernel<<<(unsigned)grid, block, smem, stream>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;

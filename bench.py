@@ -219,7 +219,7 @@ def run_ours(args, w: W.Workload):
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
-    if world > 1:
+    if world > 1 or ("RANK" in os.environ and "MASTER_ADDR" in os.environ):  # launched by torch.distributed.run
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 

@@ -470,6 +470,111 @@ __device__ __forceinline__ void start_rule_sample(float P, unsigned &prev, float
 }
 
 // ------------------------------------------------------------------------------------------
+// What a consumer thread does with one chunk of its row (up to 4*NQ samples held in registers), shared by
+// the tiled and the flat kernel.  `ns` samples of the chunk exist (the same number for all threads; missing
+// ones hold zeros, so the running sum stays put over them and they are never counted).
+// ------------------------------------------------------------------------------------------
+struct BinCtx {
+    float lut_lo, lut_scale;
+    unsigned C;
+    const unsigned short *lut;
+    const unsigned char *tau_b;
+    unsigned K4;
+    bool one;                 // the table guarantees at most one threshold to step over
+    float tau_first, tau_last;
+    uint32_t arrive_one;      // always 1, opaque to the compiler (ties a stage release to a warp vote)
+};
+
+template <int NQ>
+__device__ __forceinline__ float &sample_ref(float4 (&v)[NQ], int e)
+{
+    float4 &q = v[e >> 2];
+    switch (e & 3) {
+    case 0: return q.x;
+    case 1: return q.y;
+    case 2: return q.z;
+    default: return q.w;
+    }
+}
+
+template <int NQ, int RULE, bool BATCH>
+__device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool valid, int lane, const BinCtx &c,
+                                              unsigned char *hist_b, unsigned char *wmax_b, float &P, unsigned &prev,
+                                              int &cnt0, uint64_t *release_bar)
+{
+    constexpr int GS = NQ >= 2 ? 8 : 4;  // samples per group
+    // Running sums of the whole chunk, in place.
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        P = __fadd_rn(P, v[q].x); v[q].x = P;
+        P = __fadd_rn(P, v[q].y); v[q].y = P;
+        P = __fadd_rn(P, v[q].z); v[q].z = P;
+        P = __fadd_rn(P, v[q].w); v[q].w = P;
+    }
+    // Whole chunk still below the first threshold for every lane of the warp?  The vote needs every lane's last
+    // running sum, i.e. every shared-memory read of the stage by this warp has returned; the stage is released
+    // only after it, and the count operand of the arrive depends on the vote (arrive_one is 1), so the release
+    // cannot move ahead of the reads.
+    const bool chunk_low = __all_sync(0xffffffffu, !valid || P < c.tau_first);
+    if (release_bar != nullptr && lane == 0) mbar_arrive_count(release_bar, chunk_low ? 1u : c.arrive_one);
+    if (chunk_low) {
+        if (valid) cnt0 += ns;
+        return;
+    }
+#pragma unroll
+    for (int g = 0; g < 4 * NQ; g += GS) {
+        const int gs = min(GS, ns - g);  // samples of this group that exist (same for all threads)
+        if (gs > 0) {
+            const float pend = sample_ref(v, g + GS - 1);  // running sum after the group
+            if (__all_sync(0xffffffffu, !valid || pend < c.tau_first)) {
+                if (valid) cnt0 += gs;
+            } else if (RULE == 1) {
+                if (valid) {
+#pragma unroll
+                    for (int e = 0; e < GS; ++e) {
+                        if (e < gs) {
+                            if (c.one)
+                                start_rule_sample<true>(sample_ref(v, g + e), prev, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4, hist_b, wmax_b);
+                            else
+                                start_rule_sample<false>(sample_ref(v, g + e), prev, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4, hist_b, wmax_b);
+                        }
+                    }
+                }
+            } else if (!__all_sync(0xffffffffu, !valid || sample_ref(v, g) >= c.tau_last)) {
+                if (valid) {
+                    if (c.one && gs == GS) {  // the common case, no per-sample predicates
+                        if (BATCH) {
+                            // all table and threshold reads of the group first (independent chains that
+                            // overlap), then the histogram updates: lower latency per group
+                            unsigned off[GS];
+#pragma unroll
+                            for (int e = 0; e < GS; ++e)
+                                off[e] = bin_offset<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
+#pragma unroll
+                            for (int e = 0; e < GS; ++e) atomicAdd(reinterpret_cast<int *>(hist_b + off[e]), 1);
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < GS; ++e)
+                                bin_sample<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4, hist_b);
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < GS; ++e) {
+                            if (e < gs) {
+                                if (c.one)
+                                    bin_sample<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4, hist_b);
+                                else
+                                    bin_sample<false>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4, hist_b);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Tiled kernel: TMA-staged rows, persistent over trials.  Warp roles inside a block:
 //   warps 0 .. ncw-1   consumers: thread r owns row (pass*rows + r) of the current trial
 //   warp  ncw          producer: one thread streams the block's tiles through the ring of stages
@@ -641,7 +746,6 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     }
 
     // ---------------- consumers
-    constexpr int GQ = NQ >= 2 ? 2 : 1;  // quads per group
     const int bar_threads = ncw * 32 + 32;
     const int K = p.K;
     const int hist_buf_ints = p.hist_copies * p.hist_stride;
@@ -652,7 +756,17 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     const bool one = s.meta[0] != 0;
     const float lut_lo = __int_as_float(s.meta[1]), lut_scale = __int_as_float(s.meta[2]);
     const unsigned C = (unsigned)p.lut_cells;
-    const float tau_first = s.tau_s[0], tau_last = s.tau_s[K - 1];
+    BinCtx ctx;
+    ctx.lut_lo = lut_lo;
+    ctx.lut_scale = lut_scale;
+    ctx.C = C;
+    ctx.lut = s.lut;
+    ctx.tau_b = tau_b;
+    ctx.K4 = K4;
+    ctx.one = one;
+    ctx.tau_first = s.tau_s[0];
+    ctx.tau_last = s.tau_s[K - 1];
+    ctx.arrive_one = (uint32_t)p.one;
     // rule 1 only: this thread's copy of the worker-time maxima, and the bin of a running time of 0
     const int aux_off = p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0;
     unsigned off_zero = 0;
@@ -692,100 +806,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                     if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
                     else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 }
-                // Running sums of the whole chunk, in place (a missing quad holds zeros: P stays put and its
-                // entries are never binned).
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    P = __fadd_rn(P, v[q].x); v[q].x = P;
-                    P = __fadd_rn(P, v[q].y); v[q].y = P;
-                    P = __fadd_rn(P, v[q].z); v[q].z = P;
-                    P = __fadd_rn(P, v[q].w); v[q].w = P;
-                }
-                // Whole chunk still below the first threshold for every lane of the warp?  The vote needs every
-                // lane's last running sum, i.e. every shared-memory read of the stage by this warp has returned;
-                // the stage is released only after it, and the count operand of the arrive depends on the vote
-                // (p.one is 1), so the release cannot move ahead of the reads.
-                const bool chunk_low = __all_sync(0xffffffffu, !valid || P < tau_first);
-                if (lane == 0) mbar_arrive_count(empty_bar, chunk_low ? 1u : (uint32_t)p.one);
-                if (chunk_low) {
-                    if (valid) cnt0 += 4 * nq;
-                    continue;
-                }
-#pragma unroll
-                for (int g = 0; g < NQ; g += GQ) {
-                    const int gq = min(GQ, nq - g);  // quads of this group that exist (same for all threads)
-                    if (gq > 0) {
-                        const float pend = v[g + GQ - 1].w;  // running sum after the group
-                        if (__all_sync(0xffffffffu, !valid || pend < tau_first)) {
-                            if (valid) cnt0 += 4 * gq;
-                        } else if (RULE == 1) {
-                            if (valid) {
-#pragma unroll
-                                for (int q = 0; q < GQ; ++q) {
-                                    if (q < gq) {
-                                        if (one) {
-                                            start_rule_sample<true>(v[g + q].x, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
-                                            start_rule_sample<true>(v[g + q].y, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
-                                            start_rule_sample<true>(v[g + q].z, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
-                                            start_rule_sample<true>(v[g + q].w, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
-                                        } else {
-                                            start_rule_sample<false>(v[g + q].x, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
-                                            start_rule_sample<false>(v[g + q].y, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
-                                            start_rule_sample<false>(v[g + q].z, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
-                                            start_rule_sample<false>(v[g + q].w, prev, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b, wmax_b);
-                                        }
-                                    }
-                                }
-                            }
-                        } else if (!__all_sync(0xffffffffu, !valid || v[g].x >= tau_last)) {
-                            if (valid) {
-                                if (one && gq == GQ) {  // the common case, no per-sample predicates
-                                    // all table and threshold reads of the group first (independent chains the
-                                    // hardware can overlap), then the histogram updates
-                                    if (BATCH) {
-                                        // all table and threshold reads of the group first (independent chains
-                                        // that overlap), then the histogram updates: lower latency per group
-                                        unsigned off[4 * GQ];
-#pragma unroll
-                                        for (int q = 0; q < GQ; ++q) {
-                                            off[4 * q + 0] = bin_offset<true>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4);
-                                            off[4 * q + 1] = bin_offset<true>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4);
-                                            off[4 * q + 2] = bin_offset<true>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4);
-                                            off[4 * q + 3] = bin_offset<true>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4);
-                                        }
-#pragma unroll
-                                        for (int e = 0; e < 4 * GQ; ++e) atomicAdd(reinterpret_cast<int *>(hist_b + off[e]), 1);
-                                    } else {
-#pragma unroll
-                                        for (int q = 0; q < GQ; ++q) {
-                                            bin_sample<true>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                            bin_sample<true>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                            bin_sample<true>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                            bin_sample<true>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                        }
-                                    }
-                                } else {
-#pragma unroll
-                                    for (int q = 0; q < GQ; ++q) {
-                                        if (q < gq) {
-                                            if (one) {
-                                                bin_sample<true>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                                bin_sample<true>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                                bin_sample<true>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                                bin_sample<true>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                            } else {
-                                                bin_sample<false>(v[g + q].x, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                                bin_sample<false>(v[g + q].y, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                                bin_sample<false>(v[g + q].z, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                                bin_sample<false>(v[g + q].w, lut_lo, lut_scale, C, s.lut, tau_b, K4, hist_b);
-                                            }
-                                        }
-                                    }
-                                }
-                            }
-                        }
-                    }
-                }
+                consume_chunk<NQ, RULE, BATCH>(v, 4 * nq, valid, lane, ctx, hist_b, wmax_b, P, prev, cnt0, empty_bar);
             }
             if (valid) {
                 rowmax = fmaxf(rowmax, P);

@@ -77,8 +77,9 @@ typedef enum {
  *   out_step[t][k] = fl32( fminf(taus[k], max_n P_{t,n,M-1}) + t_comm )   (= min{tau,T} + T^c)
  *
  *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; finite and >= 0.  16-byte aligned with M a
- *              multiple of 4 takes the fast (tiled) kernel; any 4-byte aligned pointer and any M are
- *              accepted and take the plain-load kernel (see dc_simulate_plan)
+ *              multiple of 4 takes the fastest (tiled) kernel, 16-byte aligned with any other M <= 255 the
+ *              flat kernel; any 4-byte aligned pointer and any M are accepted (plain-load kernel, slow);
+ *              see dc_simulate_plan
  *   T, N, M    > 0, N*M <= INT32_MAX
  *   taus       DEVICE, [K] fp32, non-decreasing, no NaN; +infinity is allowed (gives the
  *              synchronous baseline); 4-byte aligned.  1 <= K <= DC_MAX_K
@@ -234,8 +235,9 @@ int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M,
  */
 int dc_device_status(uint32_t *flags_host);
 
-/* Which kernel dc_simulate_ex would use for a shape: 0 = tiled bulk-copy kernel, 1 = plain-load
- * kernel (M not a multiple of 4, or a pointer only 4-byte aligned), negative = -dc_status. */
+/* Which kernel dc_simulate_ex would use for a shape: 0 = tiled kernel (M a multiple of 4, 16-byte aligned
+ * pointer), 2 = flat kernel (any other M up to 255, 16-byte aligned pointer), 1 = plain-load kernel (longer
+ * such rows, or a pointer only 4-byte aligned), negative = -dc_status. */
 int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K);
 
 /*

@@ -47,6 +47,7 @@ constexpr int kHistBudgetBytes = 32 * 1024;   // shared memory spent on per-warp
 constexpr uint32_t kWaitLimit = 1u << 22;     // polls of one mbarrier wait before giving up (roughly a second)
 constexpr int kReduceChunksMax = 64;          // partial sums per threshold in dc_reduce_trials
 constexpr int kConsumerBarrier = 1;           // named barrier used by the consumer warps
+constexpr int kFlatMaxM = 255;                // longest row the flat kernel takes (32 rows of it fill a stage)
 constexpr int kLutCellsMax = 4096;            // cells of the bin lookup table (4 per threshold up to this)
 
 constexpr uint32_t kErrLoadNeverArrived = 1u;
@@ -821,6 +822,155 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 }
 
 // ------------------------------------------------------------------------------------------
+// Flat kernel: rows whose length is not a multiple of 4 (so a tensor map cannot describe them), up to
+// kFlatMaxM samples, base pointer 16-byte aligned.  A pass's rows are one contiguous span of the tensor; the
+// producer brings the 16-byte aligned span that covers them into a stage with ONE plain bulk copy
+// (cp.async.bulk, no tensor map) and thread r reads its row from float offset delta + r*M with 4-byte
+// shared loads, 32 samples at a time.  Everything after the loads is the tiled kernel's code (consume_chunk,
+// epilogue warp, double-buffered histograms).  The few floats past the last multiple of 4 of the whole
+// tensor cannot be bulk-copied in bounds; the producer moves them with ordinary loads.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+
+template <int RULE, bool BATCH>
+__global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const SweepParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+    unsigned char *stage0 = smem;
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)p.stages * p.stage_bytes);
+    uint64_t *empty = full + kMaxStages;
+    const SmemTail s = carve_tail(reinterpret_cast<unsigned char *>(empty + kMaxStages), p);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int ncw = (blockDim.x >> 5) - 2;
+    const int S = p.stages;
+    const unsigned long long NM = (unsigned long long)p.N * (unsigned long long)p.M;
+    const unsigned long long total = (unsigned long long)p.T * NM;
+    const unsigned long long total4 = total & ~3ull;
+
+    if (tid == 0) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(&full[i], 1);
+            mbar_init(&empty[i], ncw);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    load_thresholds(p, s, tid, blockDim.x);
+    __syncthreads();
+    build_lut(p, s, tid, blockDim.x);
+
+    if (warp == ncw) {
+        // ---------------- producer
+        if (lane == 0) {
+            int st = 0;
+            uint32_t ph = 0;
+            bool first = true;
+            for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
+                for (int pass = 0; pass < p.passes; ++pass) {
+                    const int row0 = pass * p.rows;
+                    const int nrows = min(p.rows, p.N - row0);
+                    const unsigned long long b0 = (unsigned long long)t * NM + (unsigned long long)row0 * p.M;
+                    const unsigned long long e0 = b0 + (unsigned long long)nrows * p.M;
+                    const unsigned long long b4 = b0 & ~3ull;                       // aligned start of the span
+                    unsigned long long e4 = (e0 + 3ull) & ~3ull;                      // aligned end, inside the tensor
+                    if (e4 > total4) e4 = total4;
+                    if (e4 < b4) e4 = b4;
+                    if (!first) mbar_wait(&empty[st], ph ^ 1u, kErrStageNeverFreed);
+                    float *dst = reinterpret_cast<float *>(stage0 + (size_t)st * p.stage_bytes);
+                    for (unsigned long long i = e4; i < e0; ++i) dst[i - b4] = p.lat[i];  // at most 3 floats, last tile only
+                    const uint32_t bytes = (uint32_t)((e4 - b4) * 4ull);
+                    mbar_arrive_expect_tx(&full[st], bytes);
+                    if (bytes != 0u) bulk_load_1d(dst, p.lat + b4, bytes, &full[st]);
+                    if (++st == S) {
+                        st = 0;
+                        ph ^= 1u;
+                        first = false;
+                    }
+                }
+            }
+        }
+        return;
+    }
+    if (warp == ncw + 1) {
+        epilogue_warp<RULE>(p, s, lane, ncw);
+        return;
+    }
+
+    // ---------------- consumers
+    const int bar_threads = ncw * 32 + 32;
+    const int K = p.K, M = p.M;
+    const int hist_buf_ints = p.hist_copies * p.hist_stride;
+    const int aux_buf_floats = p.aux_copies * (K + 2);
+    int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
+    BinCtx ctx;
+    ctx.lut_lo = __int_as_float(s.meta[1]);
+    ctx.lut_scale = __int_as_float(s.meta[2]);
+    ctx.C = (unsigned)p.lut_cells;
+    ctx.lut = s.lut;
+    ctx.tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
+    ctx.K4 = 4u * (unsigned)K;
+    ctx.one = s.meta[0] != 0;
+    ctx.tau_first = s.tau_s[0];
+    ctx.tau_last = s.tau_s[K - 1];
+    ctx.arrive_one = (uint32_t)p.one;
+    const int aux_off = p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0;
+    unsigned off_zero = 0;
+    if (RULE == 1) off_zero = bin_offset<false>(0.0f, ctx.lut_lo, ctx.lut_scale, ctx.C, ctx.lut, ctx.tau_b, ctx.K4);
+    const int myrow = min(tid, p.rows - 1);  // threads past the last row read the last row: always inside the stage
+    int st = 0;
+    uint32_t ph = 0;
+    int j = 0;
+    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
+        const int b = j & 1;
+        if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);
+        int *myhist = myhist0 + b * hist_buf_ints;
+        unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
+        unsigned char *wmax_b = reinterpret_cast<unsigned char *>(s.wmax + b * aux_buf_floats + aux_off);
+        float *mytail = s.tail + b * aux_buf_floats + aux_off;
+        float rowmax = 0.0f;
+        int cnt0 = 0;
+        for (int pass = 0; pass < p.passes; ++pass) {
+            const int row0 = pass * p.rows;
+            const bool valid = (tid < p.rows) && (row0 + tid < p.N);
+            const unsigned long long b0 = (unsigned long long)t * NM + (unsigned long long)row0 * M;
+            const int delta = (int)(b0 & 3ull);
+            float P = 0.0f;
+            unsigned prev = off_zero;
+            mbar_wait(&full[st], ph, kErrLoadNeverArrived);
+            const float *row = reinterpret_cast<const float *>(stage0 + (size_t)st * p.stage_bytes) + delta + myrow * M;
+            uint64_t *empty_bar = &empty[st];
+            if (++st == S) {
+                st = 0;
+                ph ^= 1u;
+            }
+            for (int m0 = 0; m0 < M; m0 += 32) {
+                const int ns = min(32, M - m0);
+                float4 v[8];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) sample_ref(v, e) = (e < ns) ? row[m0 + e] : 0.0f;
+                consume_chunk<8, RULE, BATCH>(v, ns, valid, lane, ctx, hist_b, wmax_b, P, prev, cnt0,
+                                              (m0 + 32 >= M) ? empty_bar : nullptr);
+            }
+            if (valid) {
+                rowmax = fmaxf(rowmax, P);
+                if (RULE == 1) record_tail(mytail, (int)(prev >> 2), P);
+            }
+        }
+        if (cnt0 > 0) atomicAdd(myhist, cnt0);
+        rowmax = warp_max(rowmax);
+        if (lane == 0) s.smax[32 * b + warp] = rowmax;
+        buffer_barrier_arrive<kBarReady>(b, bar_threads);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Plain-load kernel for shapes the tensor map cannot describe (M not a multiple of 4, or a base
 // pointer that is only 4-byte aligned).  Same walk and epilogue; each thread reads its row
 // straight from global memory.
@@ -1159,6 +1309,22 @@ int validate_simulate(const float *lat, int64_t T, int64_t N, int64_t M, const f
 }
 
 bool tiled_ok(const float *lat, int64_t M) { return (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0); }
+bool flat_ok(const float *lat, int64_t M)
+{
+    return !tiled_ok(lat, M) && M <= kFlatMaxM && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0);
+}
+
+template <int RULE, bool BATCH>
+int launch_flat(const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di, cudaStream_t stream)
+{
+    auto kernel = dc_sweep_flat<RULE, BATCH>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
+    const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
+    kernel<<<(unsigned)grid, block, smem, stream>>>(p);
+    return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
 
 template <int NQ, int RULE, bool BATCH>
 int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
@@ -1200,6 +1366,56 @@ int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t
     // rule 1 has one binning path only
     if (RULE == 0 && p.batch_lookups) return launch_tiled_b<NQ, RULE, true>(map, p, block, smem, T, di, stream);
     return launch_tiled_b<NQ, RULE, false>(map, p, block, smem, T, di, stream);
+}
+
+// Shared-memory layout of a block of the staged kernels (tiled and flat): ring depth, histogram copies, table
+// size.  Needs p.stage_bytes, p.chunks and the row-thread count; fills the rest and the dynamic shared bytes.
+int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const DeviceInfo &di, size_t *smem_out)
+{
+    p.lut_cells = min(kLutCellsMax, 4 * K);
+    // Rows that fit one tile gain from looking up a whole group's bins before touching the histogram (the
+    // chains overlap); longer rows measured faster with lookups and updates interleaved.
+    p.batch_lookups = g_tune_batch > 0 ? g_tune_batch - 1 : (p.chunks == 1 ? 1 : 0);
+    // Shared memory per block: aim at two resident blocks per SM.  Histogram copies: lane l of warp w
+    // adds into copy (w % warp_groups) * lane_copies + (l % lane_copies); copies used by one warp start
+    // 32 / lane_copies banks apart so that equal bins of different lanes do not collide.
+    p.nbuf = 2;
+    const int ncw = row_threads / 32;
+    const size_t budget = (size_t)di.smem_per_sm / 2 - 1024 - 256;
+    size_t smem = 0;
+    bool fits = false;
+    // Candidates: ring depth first (bytes in flight matter most), then histogram copies, from the
+    // preferred configuration down to the smallest one.  The first that leaves room for two blocks per
+    // SM wins; the smallest one is taken even if only one block fits.
+    // (a ring deeper than three tiles measured slower on every workload, whatever the tile size)
+    const int s_max = g_tune_stages > 0 ? g_tune_stages : min(3, max(2, kStageBudgetBytes / p.stage_bytes));
+    const int s_min = g_tune_stages > 0 ? g_tune_stages : 2;
+    const int lc_first = g_tune_lane_copies > 0 ? g_tune_lane_copies : 4;
+    const int lc_last = g_tune_lane_copies > 0 ? g_tune_lane_copies : 1;
+    const int wg_first = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
+    const int wg_last = g_tune_warp_groups > 0 ? wg_first : 1;
+    const bool forced = g_tune_stages > 0 && g_tune_lane_copies > 0 && g_tune_warp_groups > 0;
+    for (int st = s_max; st >= s_min && !fits; --st) {
+        for (int lc = lc_first; lc >= lc_last && !fits; lc >>= 1) {
+            for (int wg = wg_first; wg >= wg_last && !fits; wg >>= 1) {
+                p.stages = st;
+                p.lane_copies = lc;
+                p.warp_groups = wg;
+                p.hist_copies = wg * lc;
+                if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = wg;
+                const int want = lc > 1 ? 32 / lc : 1;
+                p.hist_stride = K + 2;
+                while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
+                smem = 1024 + 2 * kMaxStages * sizeof(uint64_t) + (size_t)st * p.stage_bytes +
+                       tail_bytes(K, p.nbuf * p.hist_copies, p.hist_stride, p.lut_cells, p.nbuf * p.aux_copies);
+                const bool smallest = (st == s_min && lc == lc_last && wg == wg_last);
+                if (smem <= budget || smallest || forced) fits = true;
+            }
+        }
+    }
+    if (!fits) return DC_ERR_RANGE;
+    *smem_out = smem;
+    return DC_OK;
 }
 
 int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
@@ -1255,48 +1471,11 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         else if (p.pitch == 64) { swz = CU_TENSOR_MAP_SWIZZLE_64B; p.swz_mask = 3; }
         else if (p.pitch == 32) { swz = CU_TENSOR_MAP_SWIZZLE_32B; p.swz_mask = 1; }
         p.stage_bytes = ((p.rows * p.pitch + 1023) / 1024) * 1024;
-        p.lut_cells = min(kLutCellsMax, 4 * K);
-        // Rows that fit one tile gain from looking up a whole group's bins before touching the histogram (the
-        // chains overlap); longer rows measured faster with lookups and updates interleaved.
-        p.batch_lookups = g_tune_batch > 0 ? g_tune_batch - 1 : (p.chunks == 1 ? 1 : 0);
-        // Shared memory per block: aim at two resident blocks per SM.  Histogram copies: lane l of warp w
-        // adds into copy (w % warp_groups) * lane_copies + (l % lane_copies); copies used by one warp start
-        // 32 / lane_copies banks apart so that equal bins of different lanes do not collide.
-        p.nbuf = 2;
-        const int ncw = row_threads / 32;
-        const size_t budget = (size_t)di.smem_per_sm / 2 - 1024 - 256;
         size_t smem = 0;
-        bool fits = false;
-        // Candidates: ring depth first (bytes in flight matter most), then histogram copies, from the
-        // preferred configuration down to the smallest one.  The first that leaves room for two blocks per
-        // SM wins; the smallest one is taken even if only one block fits.
-        // (a ring deeper than three tiles measured slower on every workload, whatever the tile size)
-        const int s_max = g_tune_stages > 0 ? g_tune_stages : min(3, max(2, kStageBudgetBytes / p.stage_bytes));
-        const int s_min = g_tune_stages > 0 ? g_tune_stages : 2;
-        const int lc_first = g_tune_lane_copies > 0 ? g_tune_lane_copies : 4;
-        const int lc_last = g_tune_lane_copies > 0 ? g_tune_lane_copies : 1;
-        const int wg_first = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
-        const int wg_last = g_tune_warp_groups > 0 ? wg_first : 1;
-        const bool forced = g_tune_stages > 0 && g_tune_lane_copies > 0 && g_tune_warp_groups > 0;
-        for (int st = s_max; st >= s_min && !fits; --st) {
-            for (int lc = lc_first; lc >= lc_last && !fits; lc >>= 1) {
-                for (int wg = wg_first; wg >= wg_last && !fits; wg >>= 1) {
-                    p.stages = st;
-                    p.lane_copies = lc;
-                    p.warp_groups = wg;
-                    p.hist_copies = wg * lc;
-                    if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = wg;
-                    const int want = lc > 1 ? 32 / lc : 1;
-                    p.hist_stride = K + 2;
-                    while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
-                    smem = 1024 + 2 * kMaxStages * sizeof(uint64_t) + (size_t)st * p.stage_bytes +
-                           tail_bytes(K, p.nbuf * p.hist_copies, p.hist_stride, p.lut_cells, p.nbuf * p.aux_copies);
-                    const bool smallest = (st == s_min && lc == lc_last && wg == wg_last);
-                    if (smem <= budget || smallest || forced) fits = true;
-                }
-            }
+        {
+            const int lrc0 = choose_block_layout(p, row_threads, K, rule, di, &smem);
+            if (lrc0 != DC_OK) return lrc0;
         }
-        if (!fits) return DC_ERR_RANGE;
 
         CUtensorMap map;
         const cuuint64_t gdim[3] = {(cuuint64_t)M, (cuuint64_t)N, (cuuint64_t)T};
@@ -1323,6 +1502,31 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
             else if (nq <= 4) lrc = launch_tiled<4, 1>(map, p, block, smem, T, di, stream);
             else lrc = launch_tiled<8, 1>(map, p, block, smem, T, di, stream);
         }
+        if (lrc == DC_OK) g_last_simulate_launches = 1;
+        return lrc;
+    }
+
+    if (flat_ok(lat, M)) {
+        // rows per pass: as many whole rows as fit a 32 KB stage (a multiple of 32, at most 256)
+        int cap = (int)((32768 - 64) / (4 * M));
+        cap = min(kMaxRowsPerPass, (cap / 32) * 32);
+        p.passes = (int)((N + cap - 1) / cap);
+        p.rows = (int)((N + p.passes - 1) / p.passes);
+        const int flat_threads = ((p.rows + 31) / 32) * 32;
+        p.bw = (int)M;
+        p.chunks = (int)((M + 31) / 32);
+        p.pitch = (int)M * 4;
+        p.stage_bytes = (int)((((size_t)p.rows * M * 4 + 32) + 1023) / 1024 * 1024);
+        size_t smem = 0;
+        const int lrc0 = choose_block_layout(p, flat_threads, K, rule, di, &smem);
+        if (lrc0 != DC_OK) return lrc0;
+        if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
+        const int block = flat_threads + 64;
+        int lrc;
+        if (rule == DC_RULE_FINISH_BEFORE_TAU)
+            lrc = p.batch_lookups ? launch_flat<0, true>(p, block, smem, T, di, stream) : launch_flat<0, false>(p, block, smem, T, di, stream);
+        else
+            lrc = launch_flat<1, false>(p, block, smem, T, di, stream);
         if (lrc == DC_OK) g_last_simulate_launches = 1;
         return lrc;
     }
@@ -1401,7 +1605,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
     if (K > DC_MAX_K || N > INT32_MAX || M > INT32_MAX || N * M > (int64_t)INT32_MAX || T > (int64_t)INT32_MAX)
         return -DC_ERR_RANGE;
     if (reinterpret_cast<uintptr_t>(latencies) & 3) return -DC_ERR_ALIGN;
-    return tiled_ok(latencies, M) ? 0 : 1;
+    return tiled_ok(latencies, M) ? 0 : (flat_ok(latencies, M) ? 2 : 1);
 }
 
 size_t dc_reduce_workspace_bytes(int64_t T, int32_t K)
@@ -1672,7 +1876,7 @@ int dc_simulate_launches(void) { return g_last_simulate_launches; }
 int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
 int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
 
-const char *dc_kernel_version(void) { return "sweep-tiled-9"; }
+const char *dc_kernel_version(void) { return "sweep-tiled-10"; }
 
 const char *dc_status_string(int status)
 {

@@ -470,3 +470,27 @@ def test_random_shapes_and_grids(api):
         assert np.array_equal(step.cpu().numpy().view(np.uint32), ref.step.view(np.uint32)), what
         assert np.array_equal(sync.cpu().numpy().view(np.uint32), ref.sync.view(np.uint32)), what
     api.dc_device_status()
+
+
+def test_flat_kernel_shapes(api):
+    """Rows whose length is not a multiple of 4 (flat kernel: one bulk copy per pass, 4-byte shared loads):
+    spans that start at every offset modulo 4, a tensor whose size is not a multiple of 4 (its last floats
+    are moved by ordinary loads), several passes, the longest supported row, both rules, and repeated runs
+    under different ring depths."""
+    cases = [(7, 3, 5, 9), (5, 1, 1, 3), (3, 257, 30, 64), (6, 513, 6, 33), (4, 100, 255, 40), (9, 64, 33, 100),
+             (11, 37, 10, 16), (2, 2048, 126, 256), (64, 200, 14, 64)]
+    try:
+        for (T, N, M, K) in cases:
+            lat = W.iid_latencies("shifted_exp", T, N, M, seed=900 + T + N + M, shift=0.01, mean=0.02).numpy()
+            taus = grid_for(lat, K, seed=K + 5)
+            lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+            assert api.dc_simulate_plan(lat_d, K) == 2
+            for rule in (0, 1):
+                ref = oracle.sweep(lat, taus, 0.07, rule=rule)
+                for stages in (0, 2, 3):
+                    api.dc_tune(api.TUNE_STAGES, stages)
+                    res = run_gpu(api, lat_d, taus_d, 0.07, rule=rule)
+                    compare_sweep(res, ref, f"flat {(T, N, M, K)} rule {rule} stages {stages}")
+    finally:
+        api.dc_tune(api.TUNE_STAGES, 0)
+    api.dc_device_status()

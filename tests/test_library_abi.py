@@ -61,7 +61,8 @@ def test_argument_errors_need_no_gpu(lib):
     assert lib.dc_argmax_tau(A, A, 4, 1, A, A, A, None) == 7      # done_frac is not an objective
     assert lib.dc_argmax_tau(A, A, 0, 4, A, A, A, None) == 2
     assert lib.dc_simulate_plan(A, 4, 8, 12, 3) == 0
-    assert lib.dc_simulate_plan(A, 4, 8, 13, 3) == 1
+    assert lib.dc_simulate_plan(A, 4, 8, 13, 3) == 2
+    assert lib.dc_simulate_plan(A, 4, 8, 301, 3) == 1
     assert lib.dc_simulate_plan(A + 4, 4, 8, 12, 3) == 1
     assert lib.dc_simulate_plan(A, 4, 8, 12, 5000) == -4
     # the later entry points

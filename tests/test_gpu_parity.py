@@ -494,3 +494,18 @@ def test_flat_kernel_shapes(api):
     finally:
         api.dc_tune(api.TUNE_STAGES, 0)
     api.dc_device_status()
+
+
+@pytest.mark.parametrize("T,N,M,K", [(3, 100000, 4, 40), (200000, 8, 4, 16), (2, 40, 4096, 64), (2, 70, 1030, 33),
+                                      (1, 300000, 1, 8), (50000, 1, 32, 5)])
+def test_extreme_aspect_ratios(api, T, N, M, K):
+    """Very many workers (hundreds of passes per trial), very many trials, very long rows (hundreds of column
+    chunks; 1030 is not a multiple of 4 and too long for the flat kernel, so it takes the plain-load one)."""
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=7000 + K, shift=0.001, mean=0.002).numpy()
+    taus = grid_for(lat, K, seed=K + 9)
+    for rule in (0, 1):
+        ref = oracle.sweep(lat, taus, 0.01, rule=rule)
+        res = run_gpu(api, torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda(), 0.01, rule=rule)
+        compare_sweep(res, ref, f"{(T, N, M, K)} rule {rule}")
+        compare_stats(res, ref, N, M, what=f"{(T, N, M, K)} rule {rule}")
+    api.dc_device_status()

@@ -117,7 +117,7 @@ def cpu_baseline(w: W.Workload, lat_dev, taus: np.ndarray, budget_s: float = 15.
     dt = max(time.perf_counter() - t, 1e-4)
     n = int(max(probe, min(w.T, budget_s / (dt / probe))))
     # keep the host copy of the sample modest
-    n = min(n, max(probe, (8 << 30) // (4 * w.N * w.M)))
+    n = min(n, max(probe, (16 << 30) // (4 * w.N * w.M)))
     lat = lat_dev[:n].cpu().numpy()
     t = time.perf_counter()
     sw = oracle.sweep(lat, taus, w.t_comm)

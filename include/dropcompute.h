@@ -120,6 +120,23 @@ int dc_simulate_tc(const float *latencies, int64_t T, int64_t N, int64_t M,
                    int32_t rule, void *stream);
 
 /*
+ * dc_simulate_split — dc_simulate_ex for FEW trials of MANY workers.  The sweep kernels give a whole trial to
+ * one thread block, so fewer trials than about twice the number of SMs leave most of the GPU idle.  This entry
+ * point sweeps every trial as G groups of N/G workers (G a divisor of N chosen by the library; no data is
+ * moved) and then merges the groups: counts add, step times and the synchronous time are maxima.  Results are
+ * bit-identical to dc_simulate_ex.  When nothing would be gained (enough trials, N < 128, or N has no suitable
+ * divisor) it simply calls dc_simulate_ex and needs no workspace.
+ *   workspace  DEVICE scratch, 256-byte aligned, at least dc_simulate_split_workspace_bytes(T, N, M, K) bytes
+ *              (0 when no split is used; sizes refer to the current device).  Contents unspecified afterwards.
+ * Other arguments as dc_simulate_ex.
+ */
+size_t dc_simulate_split_workspace_bytes(int64_t T, int64_t N, int64_t M, int32_t K);
+int dc_simulate_split(const float *latencies, int64_t T, int64_t N, int64_t M,
+                      const float *taus, int32_t K, float t_comm,
+                      float *out_step, int32_t *out_done, float *out_sync, int32_t rule,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * dc_reduce_trials — statistics over trials in fp64 (Algorithm 2: S_i(tau) and S_eff(tau); Eq. 6;
  * Sec. 4.4 throughput).  Sums run over trials in a fixed order that depends only on (T, K), so the
  * result is reproducible bit for bit.

@@ -1210,6 +1210,34 @@ dc_closed_form_kernel(double mu, double sigma, long long M, long long N, double 
     out[2 * (size_t)K + k] = (em / (double)M) * (ET + t_comm) / step;
 }
 
+// Few trials, many workers: dc_simulate_split sweeps every trial as G groups of N/G workers (the tensor is the
+// same bytes read as [T*G][N/G][M]) and this kernel puts the groups back together: completed counts add up,
+// step times and the synchronous time are maxima (rounding is monotone, so max_g fl(x_g + t_comm) equals
+// fl(max_g x_g + t_comm), and min(tau, .) commutes with the maximum).
+__global__ void __launch_bounds__(256)
+dc_combine_groups(const float *__restrict__ g_step, const int32_t *__restrict__ g_done, const float *__restrict__ g_sync,
+                  long long T, int G, int K, float *out_step, int32_t *out_done, float *out_sync)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;  // index into [T][K]
+    if (i < T * K) {
+        const long long t = i / K;
+        const int k = (int)(i - t * K);
+        int d = 0;
+        float st = g_step[(t * G) * K + k];
+        for (int g = 0; g < G; ++g) {
+            d += g_done[(t * G + g) * K + k];
+            st = fmaxf(st, g_step[(t * G + g) * K + k]);
+        }
+        out_done[i] = d;
+        out_step[i] = st;
+    }
+    if (out_sync != nullptr && i < T) {
+        float sy = g_sync[i * G];
+        for (int g = 1; g < G; ++g) sy = fmaxf(sy, g_sync[i * G + g]);
+        out_sync[i] = sy;
+    }
+}
+
 // Data precondition check: counts latencies that are negative, NaN or infinite, and thresholds
 // that are NaN or smaller than their predecessor.
 __global__ void __launch_bounds__(256)
@@ -1596,6 +1624,60 @@ int dc_simulate_tc(const float *latencies, int64_t T, int64_t N, int64_t M, cons
 {
     if (!t_comm_trials) return DC_ERR_NULL;
     return simulate_impl(latencies, T, N, M, taus, K, 0.0f, t_comm_trials, out_step, out_done, out_sync, rule, stream);
+}
+
+// Groups per trial for dc_simulate_split: the smallest divisor G of N that gives T*G >= two blocks per SM while
+// leaving at least 64 workers per group (else the largest divisor that leaves 64); 1 when nothing is gained.
+static int64_t split_groups(int64_t T, int64_t N, int sms)
+{
+    const int64_t want = 2 * (int64_t)sms;
+    if (T >= want || N < 128) return 1;
+    int64_t best = 1;
+    for (int64_t g = 2; g <= N / 64; ++g) {
+        if (N % g != 0) continue;
+        best = g;
+        if (T * g >= want) break;
+    }
+    return best;
+}
+
+size_t dc_simulate_split_workspace_bytes(int64_t T, int64_t N, int64_t M, int32_t K)
+{
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return 0;
+    DeviceInfo di;
+    if (!device_info(&di)) return 0;
+    const int64_t G = split_groups(T, N, di.sms);
+    if (G <= 1) return 0;
+    return align_up((size_t)T * G * K * 4, 256) * 2 + align_up((size_t)T * G * 4, 256);
+}
+
+int dc_simulate_split(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
+                      float *out_step, int32_t *out_done, float *out_sync, int32_t rule, void *workspace,
+                      size_t workspace_bytes, void *stream_v)
+{
+    const int rc = validate_simulate(latencies, T, N, M, taus, K, out_step, out_done, rule);
+    if (rc != DC_OK) return rc;
+    DeviceInfo di;
+    if (!device_info(&di)) return DC_ERR_CUDA;
+    const int64_t G = split_groups(T, N, di.sms);
+    if (G <= 1) return simulate_impl(latencies, T, N, M, taus, K, t_comm, nullptr, out_step, out_done, out_sync, rule, stream_v);
+    if (T * G > (int64_t)INT32_MAX) return DC_ERR_RANGE;
+    const size_t need = align_up((size_t)T * G * K * 4, 256) * 2 + align_up((size_t)T * G * 4, 256);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < need) return DC_ERR_WORKSPACE;
+    unsigned char *w = static_cast<unsigned char *>(workspace);
+    float *g_step = reinterpret_cast<float *>(w);
+    w += align_up((size_t)T * G * K * 4, 256);
+    int32_t *g_done = reinterpret_cast<int32_t *>(w);
+    w += align_up((size_t)T * G * K * 4, 256);
+    float *g_sync = reinterpret_cast<float *>(w);
+    const int src = simulate_impl(latencies, T * G, N / G, M, taus, K, t_comm, nullptr, g_step, g_done, g_sync, rule, stream_v);
+    if (src != DC_OK) return src;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const long long items = (long long)T * K > T ? (long long)T * K : T;
+    dc_combine_groups<<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(g_step, g_done, g_sync, T, (int)G, K, out_step, out_done, out_sync);
+    if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
+    g_last_simulate_launches = 2;
+    return DC_OK;
 }
 
 int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K)

@@ -509,3 +509,36 @@ def test_extreme_aspect_ratios(api, T, N, M, K):
         compare_sweep(res, ref, f"{(T, N, M, K)} rule {rule}")
         compare_stats(res, ref, N, M, what=f"{(T, N, M, K)} rule {rule}")
     api.dc_device_status()
+
+
+@pytest.mark.parametrize("T,N,M,K", [(3, 4096, 32, 64), (1, 20000, 16, 40), (7, 1000, 12, 33), (2, 2048, 126, 50),
+                                      (5, 1009, 8, 16), (400, 512, 8, 16), (4, 100, 8, 9)])
+def test_split_entry_point_matches(api, T, N, M, K):
+    """dc_simulate_split (few trials swept as groups of workers, then merged) gives the bits of dc_simulate_ex
+    and of the oracle; with a prime N, few workers or many trials it falls back to the plain call."""
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=8000 + N, shift=0.005, mean=0.01).numpy()
+    taus = grid_for(lat, K, seed=K + 11)
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    wbytes = api.dc_simulate_split_workspace_bytes(T, N, M, K)
+    if N == 1009 or N == 100 or T == 400:
+        assert wbytes == 0
+    else:
+        assert wbytes > 0
+    ws = torch.empty(wbytes + 256, dtype=torch.uint8, device="cuda") if wbytes else None
+    if ws is not None:
+        ws = ws[(-ws.data_ptr()) % 256:]
+    for rule in (0, 1):
+        ref = oracle.sweep(lat, taus, 0.02, rule=rule)
+        step = torch.empty((T, K), dtype=torch.float32, device="cuda")
+        done = torch.empty((T, K), dtype=torch.int32, device="cuda")
+        sync = torch.empty((T,), dtype=torch.float32, device="cuda")
+        api.dc_simulate_split(lat_d, taus_d, 0.02, step, done, sync, ws, rule)
+        torch.cuda.synchronize()
+        assert np.array_equal(done.cpu().numpy(), ref.done), (rule, "done")
+        assert np.array_equal(step.cpu().numpy().view(np.uint32), ref.step.view(np.uint32)), (rule, "step")
+        assert np.array_equal(sync.cpu().numpy().view(np.uint32), ref.sync.view(np.uint32)), (rule, "sync")
+    if wbytes:
+        with pytest.raises(api.DropComputeError) as e:
+            api.dc_simulate_split(lat_d, taus_d, 0.02, step, done, sync, None, 0)
+        assert e.value.status == 9
+    api.dc_device_status()

@@ -181,19 +181,23 @@ def test_check_inputs(api):
                         torch.empty(4, 4, dtype=torch.int32, device="cuda"))
 
 
-def test_sweep_host_matches_oracle(api):
-    T, N, M, K = 37, 64, 16, 20
+@pytest.mark.parametrize("M,rule,objective", [(16, 0, 4), (16, 1, 2), (10, 0, 3), (7, 1, 4)])
+def test_sweep_host_matches_oracle(api, M, rule, objective):
+    """The host-memory entry point (chunked copies overlapped with the kernels), for both rules, every
+    objective, and rows that take the tiled or the flat kernel; pageable host memory works too."""
+    T, N, K = 37, 64, 20
     lat = W.iid_latencies("shifted_exp", T, N, M, seed=9, shift=0.02, mean=0.01)
-    taus = np.linspace(0.3, 0.7, K).astype(np.float32)
-    ref = oracle.sweep(lat.numpy(), taus, 0.1)
+    taus = np.linspace(0.02 * M, 0.045 * M, K).astype(np.float32)
+    ref = oracle.sweep(lat.numpy(), taus, 0.1, rule=rule)
     st = oracle.reduce_trials(ref.step, ref.done, ref.sync, N, M)
-    for chunk in (5, 37, 100):
+    for chunk, pinned in ((5, True), (37, True), (100, False)):
         ws = torch.empty(api.dc_sweep_host_workspace_bytes(T, N, M, K, chunk) + 1024, dtype=torch.uint8, device="cuda")
         off = (-ws.data_ptr()) % 1024
-        hs = api.dc_sweep_host(lat.pin_memory(), torch.from_numpy(taus), 0.1, ws[off:], chunk)
+        hs = api.dc_sweep_host(lat.pin_memory() if pinned else lat, torch.from_numpy(taus), 0.1, ws[off:], chunk,
+                               rule=rule, objective=objective)
         assert np.allclose(hs.stats.numpy(), st.stats, rtol=RTOL_STATS, atol=0)
         assert np.allclose(hs.baseline.numpy(), st.baseline, rtol=RTOL_STATS, atol=0)
-        assert hs.k_star == oracle.argmax(st.stats[4]) and hs.tau_star == float(taus[hs.k_star])
+        assert hs.k_star == oracle.argmax(st.stats[objective]) and hs.tau_star == float(taus[hs.k_star])
 
 
 # ---- the five benchmark workloads ---------------------------------------------------------------

@@ -80,7 +80,7 @@ struct SweepParams {
     int warp_groups;   // tiled kernel: warp w uses the copies of group w % warp_groups
     int lut_cells;     // tiled kernel: cells of the bin lookup table (the table has lut_cells + 1 entries)
     int rule;          // DC_RULE_*
-    int aux_copies;    // rule 1: copies of the per-threshold worker-time maxima (0 for rule 0)
+    int aux_copies;    // rule 1: copies of the per-bin finish-time maxima, one per histogram copy (0 for rule 0)
     int batch_lookups; // tiled kernel: 1 = look up a whole group's bins before updating the histogram
     int nbuf;          // histogram / maxima buffers: 2 in the tiled kernel (filled and drained in turn), 1 in the plain one
     int one;           // always 1; a value the compiler cannot see, used to tie a stage release to a warp vote
@@ -177,31 +177,21 @@ struct RowWalk {
     }
 };
 
-// Start-before-tau rule: the per-threshold maximum over workers of W_n(k), kept as an "envelope" env[k].
-// For one worker W_n(k) is a non-decreasing step function of k, so the maximum over workers is non-decreasing
-// too.  A worker raises env over a range [a, b) to the value V it has there by walking k upward and stopping
-// at the first k where env[k] >= V already: from there on some other worker q holds a value W_q(k) >= V, and
-// since W_q is non-decreasing and q itself walks on to every later k, everything to the right ends >= V as
-// well (entries only ever grow).  In the common case this is ONE read per range.  Non-negative floats order
-// like their bit patterns, so the integer atomicMax is an exact float max.
-// The thresholds a worker never reaches (k >= its last bin j) all get its total T_n.  Instead of walking that
-// range, the worker records T_n once in tail[j]; the epilogue takes max(env[k], max_{j <= k} tail[j]).  The
-// stopping argument above still holds with "q walks on or q's tail entry covers the rest".
-__device__ __forceinline__ void record_tail(float *tail, int j, float V)
+// Start-before-tau rule.  Micro-batch m is run iff the time before it, P_{m-1}, is < tau_k, and a worker's time
+// W_n(k) is the finish time of the last micro-batch it ran (0 if it ran none).  Running sums never decrease, so
+// W_n(k) is also the LARGEST finish time among the micro-batches the worker ran, and the step's compute time is
+//     max_n W_n(k) = max { P_{n,m} : P_{n,m-1} < tau_k }            (all micro-batches any worker started).
+// With j(x) = #{k' : tau_k' <= x} (the bin of x), P_{m-1} < tau_k  <=>  j(P_{m-1}) <= k.  So each micro-batch
+// makes two POINT updates at the bin a = j(P_{m-1}) of the time before it,
+//     hist[a] += 1   and   fmax[a] = max(fmax[a], P_m),
+// and the epilogue turns them into done[t][k] (prefix sum of hist) and max_n W_n(k) (prefix maximum of fmax).
+// Non-negative floats order like their bit patterns, so the integer atomicMax is an exact float maximum.
+__device__ __forceinline__ void raise_max(float *slot, float V)
 {
-    if (V > *reinterpret_cast<volatile float *>(tail + j)) atomicMax(reinterpret_cast<int *>(tail + j), __float_as_int(V));
-}
-__device__ __forceinline__ void raise_envelope(float *env, int a, int b, float V)
-{
-    for (int k = a; k < b; ++k) {
-        if (*reinterpret_cast<volatile float *>(env + k) >= V) break;
-        atomicMax(reinterpret_cast<int *>(env + k), __float_as_int(V));
-    }
+    atomicMax(reinterpret_cast<int *>(slot), __float_as_int(V));
 }
 
-// Start-before-tau rule, one worker's row with a forward cursor (plain-load kernel).  Micro-batch m is run iff
-// the time before it, P_{m-1}, is < tau_k; the worker's time W(k) is the finish time of the last one it ran:
-// the first running sum that reaches tau_k, or the row total if none does, or 0 if tau_k <= 0.
+// Start-before-tau rule, one worker's row with a forward cursor (plain-load kernel).
 struct RowWalkStart {
     float P;
     int cur;  // #{k : tau_k <= P}
@@ -211,18 +201,12 @@ struct RowWalkStart {
         cur = 0;
         while (cur < K && 0.0f >= tau_s[cur]) ++cur;
     }
-    __device__ __forceinline__ void step(float x, const float *tau_s, int *hist, float *env, int K)
+    __device__ __forceinline__ void step(float x, const float *tau_s, int *hist, float *fmax, int K)
     {
         atomicAdd(&hist[cur], 1);  // P_{m-1} is in bin cur
         P = __fadd_rn(P, x);
-        int nc = cur;
-        while (nc < K && P >= tau_s[nc]) ++nc;  // thresholds cur .. nc-1 are first reached by this micro-batch
-        raise_envelope(env, cur, nc, P);
-        cur = nc;
-    }
-    __device__ __forceinline__ void finish(float *tail)
-    {
-        record_tail(tail, cur, P);  // thresholds cur.. were never reached: W = row total (tail has K + 2 entries)
+        raise_max(&fmax[cur], P);
+        while (cur < K && P >= tau_s[cur]) ++cur;
     }
 };
 
@@ -257,15 +241,13 @@ __device__ __forceinline__ int warp_inclusive_scan(int v, int lane)
 // T = max_n T_n, writes step[t][k] = min(tau_k, T) + T^c and sync[t] = T + T^c, and clears the
 // histograms for the next trial.
 // ------------------------------------------------------------------------------------------
-// Rule 1 (start-before-tau): step[t][k] = max_n W_n(k) + T^c, the maximum being the envelope wmax[] (see
-// raise_envelope).
+// Rule 1 (start-before-tau): step[t][k] = max_n W_n(k) + T^c = (prefix maximum of fmax[] up to bin k) + T^c.
 __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t, float rowmax, int tid, int nthr,
                                                int barrier_id, const float *tau_s, int *hist, float *smax, int *wtot,
-                                               float *wmax, float *tail, float *wmx)
+                                               float *fmax, float *wmx)
 {
     const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
     const int K = p.K, H = p.hist_copies, HS = p.hist_stride;
-    const int A = p.aux_copies, AS = K + 2;
     const bool rule1 = p.rule == DC_RULE_START_BEFORE_TAU;
     const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
     rowmax = warp_max(rowmax);
@@ -278,28 +260,29 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
     const int ipt = (K + nthr - 1) / nthr;  // bins per thread (consecutive)
     const int b0 = min(K, tid * ipt), b1 = min(K, b0 + ipt);
     int tot = 0;
-    float tl = 0.0f;
+    float fm = 0.0f;
     for (int b = b0; b < b1; ++b) {
-        for (int c = 0; c < H; ++c) tot += hist[c * HS + b];
-        if (rule1)
-            for (int c = 0; c < A; ++c) tl = fmaxf(tl, tail[c * AS + b]);
+        for (int c = 0; c < H; ++c) {
+            tot += hist[c * HS + b];
+            if (rule1) fm = fmaxf(fm, fmax[c * HS + b]);
+        }
     }
     const int incl = warp_inclusive_scan(tot, lane);
     if (lane == 31) wtot[warp] = incl;
-    float tl_incl = 0.0f;
+    float fm_incl = 0.0f;
     if (rule1) {
-        tl_incl = warp_inclusive_max_scan(tl, lane);
-        if (lane == 31) wmx[warp] = tl_incl;
+        fm_incl = warp_inclusive_max_scan(fm, lane);
+        if (lane == 31) wmx[warp] = fm_incl;
     }
     named_barrier(barrier_id, nthr);
 
     int run = incl - tot;
     for (int w = 0; w < warp; ++w) run += wtot[w];
-    float tail_run = 0.0f;  // max of tail[] over all bins before b0
+    float fm_run = 0.0f;  // maximum of fmax[] over all bins before b0
     if (rule1) {
-        const float up = __shfl_up_sync(0xffffffffu, tl_incl, 1);
-        if (lane > 0) tail_run = up;
-        for (int w = 0; w < warp; ++w) tail_run = fmaxf(tail_run, wmx[w]);
+        const float up = __shfl_up_sync(0xffffffffu, fm_incl, 1);
+        if (lane > 0) fm_run = up;
+        for (int w = 0; w < warp; ++w) fm_run = fmaxf(fm_run, wmx[w]);
     }
     float *step_row = p.out_step + t * K;
     int32_t *done_row = p.out_done + t * K;
@@ -308,31 +291,23 @@ __device__ __forceinline__ void trial_epilogue(const SweepParams &p, long long t
         for (int c = 0; c < H; ++c) {
             h += hist[c * HS + b];
             hist[c * HS + b] = 0;
+            if (rule1) {
+                fm_run = fmaxf(fm_run, fmax[c * HS + b]);
+                fmax[c * HS + b] = 0.0f;
+            }
         }
         run += h;
         done_row[b] = run;
-        if (!rule1) {
-            step_row[b] = __fadd_rn(fminf(tau_s[b], Tmax), t_comm);
-        } else {
-            float w = 0.0f;
-            for (int c = 0; c < A; ++c) {
-                tail_run = fmaxf(tail_run, tail[c * AS + b]);
-                w = fmaxf(w, wmax[c * AS + b]);
-                wmax[c * AS + b] = 0.0f;
-                tail[c * AS + b] = 0.0f;
-            }
-            step_row[b] = __fadd_rn(fmaxf(w, tail_run), t_comm);
-        }
+        step_row[b] = __fadd_rn(rule1 ? fm_run : fminf(tau_s[b], Tmax), t_comm);
     }
     for (int c = tid; c < H; c += nthr) {  // the bins of samples at or above the last threshold
         hist[c * HS + K] = 0;
         if (HS > K + 1) hist[c * HS + K + 1] = 0;
-    }
-    if (rule1)
-        for (int c = tid; c < A; c += nthr) {
-            tail[c * AS + K] = 0.0f;
-            tail[c * AS + K + 1] = 0.0f;
+        if (rule1) {
+            fmax[c * HS + K] = 0.0f;
+            if (HS > K + 1) fmax[c * HS + K + 1] = 0.0f;
         }
+    }
     if (tid == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
     named_barrier(barrier_id, nthr);  // histograms cleared, smax/wtot free again
 }
@@ -345,9 +320,9 @@ struct SmemTail {
     int *wtot;
     int *meta;           // [0] lookup table has at most one finite threshold per cell, [1..2] lo, scale (as bits)
     unsigned short *lut; // lut_cells + 1 entries (tiled kernel only)
-    float *wmx;          // rule 1, plain kernel: warp totals of the tail max-scan
-    float *wmax;         // rule 1: [nbuf][aux_copies][K + 2] envelope of the workers' times per threshold
-    float *tail;         // rule 1: [nbuf][aux_copies][K + 2] largest total among workers whose last bin is j
+    float *wmx;          // rule 1, plain kernel: warp totals of the prefix-maximum scan
+    float *fmax;         // rule 1: [nbuf][hist_copies][hist_stride], laid out like hist: largest finish time among
+                         // the micro-batches whose start time lies in the bin
 };
 __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepParams &p)
 {
@@ -360,15 +335,15 @@ __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepP
     s.lut = reinterpret_cast<unsigned short *>(s.meta + 8);
     s.wmx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(s.lut) +
                                       (((size_t)(p.lut_cells + 1) * sizeof(unsigned short) + 3) & ~(size_t)3));
-    s.wmax = s.wmx + 32;
-    s.tail = s.wmax + p.nbuf * p.aux_copies * (p.K + 2);
+    s.fmax = s.wmx + 32;
     return s;
 }
-__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride, int lut_cells, int aux_copies)
+// hist_copies and fmax_copies count all buffers (nbuf times the copies of one buffer)
+__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride, int lut_cells, int fmax_copies)
 {
     return sizeof(float) * (size_t)(K + 1) + sizeof(int) * (size_t)hist_copies * hist_stride + 72 * sizeof(int) +
            (((size_t)(lut_cells + 1) * sizeof(unsigned short) + 3) & ~(size_t)3) + 32 * sizeof(float) +
-           2 * sizeof(float) * (size_t)aux_copies * (K + 2);
+           sizeof(float) * (size_t)fmax_copies * hist_stride;
 }
 
 __device__ __forceinline__ void load_thresholds(const SweepParams &p, const SmemTail &s, int tid, int nthr)
@@ -376,7 +351,7 @@ __device__ __forceinline__ void load_thresholds(const SweepParams &p, const Smem
     for (int k = tid; k < p.K; k += nthr) s.tau_s[k] = p.taus[k];
     if (tid == 0) s.tau_s[p.K] = __int_as_float(0x7f800000);  // +inf sentinel
     for (int i = tid; i < p.nbuf * p.hist_copies * p.hist_stride; i += nthr) s.hist[i] = 0;
-    for (int i = tid; i < 2 * p.nbuf * p.aux_copies * (p.K + 2); i += nthr) s.wmax[i] = 0.0f;  // wmax and tail are adjacent
+    for (int i = tid; i < p.nbuf * p.aux_copies * p.hist_stride; i += nthr) s.fmax[i] = 0.0f;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -457,17 +432,12 @@ __device__ __forceinline__ void bin_sample(float P, float lo, float scale, unsig
     atomicAdd(reinterpret_cast<int *>(hist_b + bin_offset<ONE>(P, lo, scale, C, lut, tau_b, K4)), 1);
 }
 // Start-before-tau rule: micro-batch m with finish time P.  The time before it lies in bin `prev` (byte
-// offset), which is what the completion count is taken on; the thresholds in [prev, j(P)) are first reached by
-// this micro-batch, so P is a candidate for their worker-time maximum.
-template <bool ONE>
-__device__ __forceinline__ void start_rule_sample(float P, unsigned &prev, float lo, float scale, unsigned C,
-                                                  const unsigned short *lut, const unsigned char *tau_b, unsigned K4,
-                                                  unsigned char *hist_b, unsigned char *wmax_b)
+// offset): that bin's count goes up by one and its finish-time maximum is raised to P (see RowWalkStart);
+// fmax_delta is the byte distance from a histogram entry to the maximum of the same bin and copy.
+__device__ __forceinline__ void start_rule_update(float P, unsigned prev, unsigned char *hist_b, unsigned fmax_delta)
 {
-    const unsigned off = bin_offset<ONE>(P, lo, scale, C, lut, tau_b, K4);
     atomicAdd(reinterpret_cast<int *>(hist_b + prev), 1);
-    raise_envelope(reinterpret_cast<float *>(wmax_b), (int)(prev >> 2), (int)(min(off, K4) >> 2), P);
-    prev = off;
+    atomicMax(reinterpret_cast<int *>(hist_b + fmax_delta + prev), __float_as_int(P));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -498,10 +468,12 @@ __device__ __forceinline__ float &sample_ref(float4 (&v)[NQ], int e)
     }
 }
 
+// Rule 1 keeps, besides the count of bin-0 samples (cnt0), the largest finish time among them (fin0), and the bin
+// `prev` (byte offset) of the running time before the next micro-batch.
 template <int NQ, int RULE, bool BATCH>
 __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool valid, int lane, const BinCtx &c,
-                                              unsigned char *hist_b, unsigned char *wmax_b, float &P, unsigned &prev,
-                                              int &cnt0, uint64_t *release_bar)
+                                              unsigned char *hist_b, unsigned fmax_delta, float &P, unsigned &prev,
+                                              int &cnt0, float &fin0, uint64_t *release_bar)
 {
     constexpr int GS = NQ >= 2 ? 8 : 4;  // samples per group
     // Running sums of the whole chunk, in place.
@@ -519,7 +491,12 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
     const bool chunk_low = __all_sync(0xffffffffu, !valid || P < c.tau_first);
     if (release_bar != nullptr && lane == 0) mbar_arrive_count(release_bar, chunk_low ? 1u : c.arrive_one);
     if (chunk_low) {
-        if (valid) cnt0 += ns;
+        // (rule 1: the times before these micro-batches are below the first threshold too, and a positive first
+        // threshold puts them, like a time of 0, into bin 0)
+        if (valid) {
+            cnt0 += ns;
+            if (RULE == 1) fin0 = fmaxf(fin0, P);
+        }
         return;
     }
 #pragma unroll
@@ -528,16 +505,35 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
         if (gs > 0) {
             const float pend = sample_ref(v, g + GS - 1);  // running sum after the group
             if (__all_sync(0xffffffffu, !valid || pend < c.tau_first)) {
-                if (valid) cnt0 += gs;
-            } else if (RULE == 1) {
                 if (valid) {
+                    cnt0 += gs;
+                    if (RULE == 1) fin0 = fmaxf(fin0, pend);
+                }
+            } else if (RULE == 1) {
+                // Every lane already at or above the last threshold before the group: none of its micro-batches
+                // is started under any threshold.
+                if (!__all_sync(0xffffffffu, !valid || prev >= c.K4)) {
+                    if (valid) {
+                        if (c.one && gs == GS) {
+                            unsigned off[GS];
 #pragma unroll
-                    for (int e = 0; e < GS; ++e) {
-                        if (e < gs) {
-                            if (c.one)
-                                start_rule_sample<true>(sample_ref(v, g + e), prev, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4, hist_b, wmax_b);
-                            else
-                                start_rule_sample<false>(sample_ref(v, g + e), prev, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4, hist_b, wmax_b);
+                            for (int e = 0; e < GS; ++e)
+                                off[e] = bin_offset<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
+#pragma unroll
+                            for (int e = 0; e < GS; ++e) {
+                                start_rule_update(sample_ref(v, g + e), prev, hist_b, fmax_delta);
+                                prev = off[e];
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < GS; ++e) {
+                                if (e < gs) {
+                                    const float Pe = sample_ref(v, g + e);
+                                    start_rule_update(Pe, prev, hist_b, fmax_delta);
+                                    prev = c.one ? bin_offset<true>(Pe, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4)
+                                                 : bin_offset<false>(Pe, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
+                                }
+                            }
                         }
                     }
                 }
@@ -623,36 +619,33 @@ __device__ __forceinline__ void buffer_barrier_arrive(int b, int threads)
 template <int RULE>
 __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTail &s, int lane, int ncw)
 {
-    const int K = p.K, H = p.hist_copies, HS = p.hist_stride, A = p.aux_copies, AS = K + 2;
+    const int K = p.K, H = p.hist_copies, HS = p.hist_stride;
     const int bar_threads = ncw * 32 + 32;
     int j = 0;
     for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
         const int b = j & 1;
         buffer_barrier_sync<kBarReady>(b, bar_threads);  // every consumer has finished trial t
         int *hist = s.hist + b * H * HS;
-        float *wmax = s.wmax + b * A * AS;
-        float *tail = s.tail + b * A * AS;
+        float *fmax = s.fmax + b * H * HS;  // rule 1 only
         const float Tmax = warp_max(lane < ncw ? s.smax[32 * b + lane] : 0.0f);
         const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
         float *step_row = p.out_step + t * K;
         int32_t *done_row = p.out_done + t * K;
         int carry = 0;
-        float tail_carry = 0.0f;
+        float fm_carry = 0.0f;
         for (int k0 = 0; k0 < K; k0 += 32) {
             const int k = k0 + lane;
             int h = 0;
-            float w = 0.0f, tl = 0.0f;
+            float fm = 0.0f;
             if (k < K) {
                 for (int c = 0; c < H; ++c) {
                     h += hist[c * HS + k];
                     hist[c * HS + k] = 0;
                 }
                 if (RULE == 1) {
-                    for (int c = 0; c < A; ++c) {
-                        w = fmaxf(w, wmax[c * AS + k]);
-                        tl = fmaxf(tl, tail[c * AS + k]);
-                        wmax[c * AS + k] = 0.0f;
-                        tail[c * AS + k] = 0.0f;
+                    for (int c = 0; c < H; ++c) {
+                        fm = fmaxf(fm, fmax[c * HS + k]);
+                        fmax[c * HS + k] = 0.0f;
                     }
                 }
             }
@@ -661,10 +654,10 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
             if (RULE == 0) {
                 step = __fadd_rn(fminf(k < K ? s.tau_s[k] : 0.0f, Tmax), t_comm);
             } else {
-                // max_n W_n(k) = max(envelope[k], max_{j <= k} tail[j])
-                const float tl_incl = warp_inclusive_max_scan(tl, lane);
-                step = __fadd_rn(fmaxf(w, fmaxf(tail_carry, tl_incl)), t_comm);
-                tail_carry = fmaxf(tail_carry, __shfl_sync(0xffffffffu, tl_incl, 31));
+                // max_n W_n(k) = max_{j <= k} fmax[j]
+                const float fm_incl = warp_inclusive_max_scan(fm, lane);
+                step = __fadd_rn(fmaxf(fm_carry, fm_incl), t_comm);
+                fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fm_incl, 31));
             }
             if (k < K) {
                 done_row[k] = carry + incl;
@@ -677,11 +670,9 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
             hist[c * HS + K + 1] = 0;
         }
         if (RULE == 1) {
-            for (int c = lane; c < A; c += 32) {
-                wmax[c * AS + K] = 0.0f;
-                wmax[c * AS + K + 1] = 0.0f;
-                tail[c * AS + K] = 0.0f;
-                tail[c * AS + K + 1] = 0.0f;
+            for (int c = lane; c < H; c += 32) {
+                fmax[c * HS + K] = 0.0f;
+                fmax[c * HS + K + 1] = 0.0f;
             }
         }
         if (lane == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
@@ -750,8 +741,9 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     const int bar_threads = ncw * 32 + 32;
     const int K = p.K;
     const int hist_buf_ints = p.hist_copies * p.hist_stride;
-    const int aux_buf_floats = p.aux_copies * (K + 2);
     int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
+    // rule 1: byte distance from a histogram entry to the finish-time maximum of the same buffer, copy and bin
+    const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));
     const unsigned char *tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
     const unsigned K4 = 4u * (unsigned)K;
     const bool one = s.meta[0] != 0;
@@ -768,8 +760,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     ctx.tau_first = s.tau_s[0];
     ctx.tau_last = s.tau_s[K - 1];
     ctx.arrive_one = (uint32_t)p.one;
-    // rule 1 only: this thread's copy of the worker-time maxima, and the bin of a running time of 0
-    const int aux_off = p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0;
+    // rule 1 only: the bin of a running time of 0
     unsigned off_zero = 0;
     if (RULE == 1) off_zero = bin_offset<false>(0.0f, lut_lo, lut_scale, C, s.lut, tau_b, K4);
     // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
@@ -784,9 +775,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
         if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
         int *myhist = myhist0 + b * hist_buf_ints;
         unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
-        unsigned char *wmax_b = reinterpret_cast<unsigned char *>(s.wmax + b * aux_buf_floats + aux_off);
-        float *mytail = s.tail + b * aux_buf_floats + aux_off;
-        float rowmax = 0.0f;
+        float rowmax = 0.0f, fin0 = 0.0f;
         int cnt0 = 0;
         for (int pass = 0; pass < p.passes; ++pass) {
             const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
@@ -807,14 +796,14 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
                     if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
                     else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 }
-                consume_chunk<NQ, RULE, BATCH>(v, 4 * nq, valid, lane, ctx, hist_b, wmax_b, P, prev, cnt0, empty_bar);
+                consume_chunk<NQ, RULE, BATCH>(v, 4 * nq, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, empty_bar);
             }
-            if (valid) {
-                rowmax = fmaxf(rowmax, P);
-                if (RULE == 1) record_tail(mytail, (int)(prev >> 2), P);  // thresholds never reached: W = total
-            }
+            if (valid) rowmax = fmaxf(rowmax, P);
         }
-        if (cnt0 > 0) atomicAdd(myhist, cnt0);
+        if (cnt0 > 0) {
+            atomicAdd(myhist, cnt0);
+            if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
+        }
         rowmax = warp_max(rowmax);
         if (lane == 0) s.smax[32 * b + warp] = rowmax;
         buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
@@ -907,8 +896,8 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
     const int bar_threads = ncw * 32 + 32;
     const int K = p.K, M = p.M;
     const int hist_buf_ints = p.hist_copies * p.hist_stride;
-    const int aux_buf_floats = p.aux_copies * (K + 2);
     int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
+    const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));
     BinCtx ctx;
     ctx.lut_lo = __int_as_float(s.meta[1]);
     ctx.lut_scale = __int_as_float(s.meta[2]);
@@ -920,7 +909,6 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
     ctx.tau_first = s.tau_s[0];
     ctx.tau_last = s.tau_s[K - 1];
     ctx.arrive_one = (uint32_t)p.one;
-    const int aux_off = p.aux_copies ? (warp % p.aux_copies) * (K + 2) : 0;
     unsigned off_zero = 0;
     if (RULE == 1) off_zero = bin_offset<false>(0.0f, ctx.lut_lo, ctx.lut_scale, ctx.C, ctx.lut, ctx.tau_b, ctx.K4);
     const int myrow = min(tid, p.rows - 1);  // threads past the last row read the last row: always inside the stage
@@ -932,9 +920,7 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
         if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);
         int *myhist = myhist0 + b * hist_buf_ints;
         unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
-        unsigned char *wmax_b = reinterpret_cast<unsigned char *>(s.wmax + b * aux_buf_floats + aux_off);
-        float *mytail = s.tail + b * aux_buf_floats + aux_off;
-        float rowmax = 0.0f;
+        float rowmax = 0.0f, fin0 = 0.0f;
         int cnt0 = 0;
         for (int pass = 0; pass < p.passes; ++pass) {
             const int row0 = pass * p.rows;
@@ -955,15 +941,15 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
                 float4 v[8];
 #pragma unroll
                 for (int e = 0; e < 32; ++e) sample_ref(v, e) = (e < ns) ? row[m0 + e] : 0.0f;
-                consume_chunk<8, RULE, BATCH>(v, ns, valid, lane, ctx, hist_b, wmax_b, P, prev, cnt0,
+                consume_chunk<8, RULE, BATCH>(v, ns, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0,
                                               (m0 + 32 >= M) ? empty_bar : nullptr);
             }
-            if (valid) {
-                rowmax = fmaxf(rowmax, P);
-                if (RULE == 1) record_tail(mytail, (int)(prev >> 2), P);
-            }
+            if (valid) rowmax = fmaxf(rowmax, P);
         }
-        if (cnt0 > 0) atomicAdd(myhist, cnt0);
+        if (cnt0 > 0) {
+            atomicAdd(myhist, cnt0);
+            if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
+        }
         rowmax = warp_max(rowmax);
         if (lane == 0) s.smax[32 * b + warp] = rowmax;
         buffer_barrier_arrive<kBarReady>(b, bar_threads);
@@ -983,6 +969,7 @@ __global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepPar
     load_thresholds(p, s, tid, nthr);
     __syncthreads();
     int *myhist = s.hist + (warp & (p.hist_copies - 1)) * p.hist_stride;
+    float *myfmax = s.fmax + (warp & (p.hist_copies - 1)) * p.hist_stride;  // rule 1 only
     for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
         float rowmax = 0.0f;
         for (int pass = 0; pass < p.passes; ++pass) {
@@ -998,13 +985,12 @@ __global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepPar
                 } else {
                     RowWalkStart w;
                     w.start(s.tau_s, p.K);
-                    for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), s.tau_s, myhist, s.wmax, p.K);
-                    w.finish(s.tail);
+                    for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), s.tau_s, myhist, myfmax, p.K);
                     rowmax = fmaxf(rowmax, w.P);
                 }
             }
         }
-        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot, s.wmax, s.tail, s.wmx);
+        trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot, s.fmax, s.wmx);
     }
 }
 
@@ -1392,7 +1378,9 @@ int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t
                  cudaStream_t stream)
 {
     // rule 1 has one binning path only
-    if (RULE == 0 && p.batch_lookups) return launch_tiled_b<NQ, RULE, true>(map, p, block, smem, T, di, stream);
+    if constexpr (RULE == 0) {
+        if (p.batch_lookups) return launch_tiled_b<NQ, RULE, true>(map, p, block, smem, T, di, stream);
+    }
     return launch_tiled_b<NQ, RULE, false>(map, p, block, smem, T, di, stream);
 }
 
@@ -1430,7 +1418,7 @@ int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const 
                 p.lane_copies = lc;
                 p.warp_groups = wg;
                 p.hist_copies = wg * lc;
-                if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = wg;
+                if (rule == DC_RULE_START_BEFORE_TAU) p.aux_copies = p.hist_copies;
                 const int want = lc > 1 ? 32 / lc : 1;
                 p.hist_stride = K + 2;
                 while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
@@ -1482,7 +1470,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.nbuf = 1;
     p.batch_lookups = 0;
     p.rule = rule;
-    p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? 1 : 0;
+    p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? p.hist_copies : 0;
 
     if (tiled_ok(lat, M)) {
         EncodeTiledFn encode = get_encode_fn();

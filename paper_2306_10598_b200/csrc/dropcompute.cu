@@ -434,10 +434,19 @@ __device__ __forceinline__ void bin_sample(float P, float lo, float scale, unsig
 // Start-before-tau rule: micro-batch m with finish time P.  The time before it lies in bin `prev` (byte
 // offset): that bin's count goes up by one and its finish-time maximum is raised to P (see RowWalkStart);
 // fmax_delta is the byte distance from a histogram entry to the maximum of the same bin and copy.
-__device__ __forceinline__ void start_rule_update(float P, unsigned prev, unsigned char *hist_b, unsigned fmax_delta)
+// Bin 0 is kept in the thread's registers (cnt0, fin0) and added once per trial: when a straggler lane sends its
+// warp through this path the other lanes are typically all still in bin 0 and would pile up on one entry.  (The
+// same test in the finish-before-tau path measured slower there, so that path adds unconditionally.)
+__device__ __forceinline__ void start_rule_update(float P, unsigned prev, unsigned char *hist_b, unsigned fmax_delta,
+                                                  int &cnt0, float &fin0)
 {
-    atomicAdd(reinterpret_cast<int *>(hist_b + prev), 1);
-    atomicMax(reinterpret_cast<int *>(hist_b + fmax_delta + prev), __float_as_int(P));
+    if (prev != 0u) {
+        atomicAdd(reinterpret_cast<int *>(hist_b + prev), 1);
+        atomicMax(reinterpret_cast<int *>(hist_b + fmax_delta + prev), __float_as_int(P));
+    } else {
+        ++cnt0;
+        fin0 = fmaxf(fin0, P);
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -521,7 +530,7 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
                                 off[e] = bin_offset<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
 #pragma unroll
                             for (int e = 0; e < GS; ++e) {
-                                start_rule_update(sample_ref(v, g + e), prev, hist_b, fmax_delta);
+                                start_rule_update(sample_ref(v, g + e), prev, hist_b, fmax_delta, cnt0, fin0);
                                 prev = off[e];
                             }
                         } else {
@@ -529,7 +538,7 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
                             for (int e = 0; e < GS; ++e) {
                                 if (e < gs) {
                                     const float Pe = sample_ref(v, g + e);
-                                    start_rule_update(Pe, prev, hist_b, fmax_delta);
+                                    start_rule_update(Pe, prev, hist_b, fmax_delta, cnt0, fin0);
                                     prev = c.one ? bin_offset<true>(Pe, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4)
                                                  : bin_offset<false>(Pe, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
                                 }

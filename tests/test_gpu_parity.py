@@ -115,6 +115,31 @@ def test_unaligned_base_takes_plain_kernel(api):
     compare_sweep(res, oracle.sweep(lat, taus, 0.3))
 
 
+@pytest.mark.parametrize("rule", [0, 1])
+@pytest.mark.parametrize("T,N,M,K", [(5, 200, 32, 64), (3, 300, 36, 132), (4, 77, 10, 256)])
+def test_outputs_only_4_byte_aligned(api, T, N, M, K, rule):
+    # Output rows that start on 16-byte boundaries are written four thresholds at a time; outputs that are only
+    # 4-byte aligned (views one element into a buffer) take the one-threshold-per-lane path.  Both must give the
+    # oracle's bits.
+    lat = W.iid_latencies("uniform", T, N, M, seed=21 + K, lo=0.0, hi=0.05).numpy()
+    taus = grid_for(lat, K, 7)
+    ref = oracle.sweep(lat, taus, 0.2, rule=rule)
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    for shift in (0, 1):
+        step = torch.full((T * K + shift,), -1.0, dtype=torch.float32, device="cuda")
+        done = torch.full((T * K + shift,), -1, dtype=torch.int32, device="cuda")
+        sync = torch.empty(T, dtype=torch.float32, device="cuda")
+        api.dc_simulate_ex(lat_d, taus_d, 0.2, step[shift:].view(T, K), done[shift:].view(T, K), sync, rule)
+        torch.cuda.synchronize()
+        assert np.array_equal(done[shift:].view(T, K).cpu().numpy(), ref.done), f"out_done differs (shift {shift})"
+        assert np.array_equal(step[shift:].view(T, K).cpu().numpy().view(np.uint32), ref.step.view(np.uint32)), \
+            f"out_step differs (shift {shift})"
+        assert np.array_equal(sync.cpu().numpy().view(np.uint32), ref.sync.view(np.uint32))
+        if shift:
+            assert float(step[0]) == -1.0 and int(done[0]) == -1   # nothing written before the view
+    api.dc_device_status()
+
+
 def test_zero_and_tie_latencies(api):
     # dyadic values: many running sums coincide with thresholds exactly, zeros repeat a running sum
     T, N, M, K = 6, 37, 24, 40

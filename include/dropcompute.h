@@ -266,6 +266,8 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  *   DC_TUNE_BATCH_LOOKUPS 1 = bin each running sum and update the histogram at once, 2 = look up the bins of a
  *                        whole group of eight first (lower latency, better for trials that fit one tile)
  *   DC_TUNE_BOX_FLOATS   floats of a row fetched per tile (16 or 32; 16 needs M to be a multiple of 16)
+ *   DC_TUNE_DIRECT_BINS  1 = always bin through the lookup table, 2 = bin evenly spaced thresholds arithmetically
+ *                        (one multiply-add and one comparison per sample, no table read) in the tiled kernel
  * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
  */
 #define DC_TUNE_STAGES 1
@@ -273,6 +275,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
 #define DC_TUNE_WARP_GROUPS 3
 #define DC_TUNE_BOX_FLOATS 4
 #define DC_TUNE_BATCH_LOOKUPS 5
+#define DC_TUNE_DIRECT_BINS 6
 int dc_tune(int32_t key, int32_t value);
 
 /* Number of kernel launches the last successful call of each entry point enqueues (for accounting). */

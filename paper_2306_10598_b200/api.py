@@ -290,7 +290,7 @@ def dc_sweep_host(latencies_host: torch.Tensor, taus_host: torch.Tensor, t_comm:
     return HostSweep(stats, base, int(k_star.value), float(tau_star.value))
 
 
-TUNE_STAGES, TUNE_LANE_COPIES, TUNE_WARP_GROUPS, TUNE_BOX_FLOATS = 1, 2, 3, 4
+TUNE_STAGES, TUNE_LANE_COPIES, TUNE_WARP_GROUPS, TUNE_BOX_FLOATS, TUNE_BATCH_LOOKUPS, TUNE_DIRECT_BINS = 1, 2, 3, 4, 5, 6
 
 
 def dc_tune(key: int, value: int) -> None:

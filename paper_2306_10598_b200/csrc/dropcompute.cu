@@ -84,6 +84,7 @@ struct SweepParams {
     int batch_lookups; // tiled kernel: 1 = look up a whole group's bins before updating the histogram
     int nbuf;          // histogram / maxima buffers: 2 in the tiled kernel (filled and drained in turn), 1 in the plain one
     int one;           // always 1; a value the compiler cannot see, used to tie a stage release to a warp vote
+    int direct_bins;   // staged kernels: 1 = bin evenly spaced thresholds arithmetically instead of through the table
     int epi_vec;       // staged kernels: the epilogue warp may take four bins per lane with 16-byte accesses
                        // (K a multiple of 4, out_step / out_done 16-byte aligned, hist_stride a multiple of 4)
 };
@@ -320,7 +321,8 @@ struct SmemTail {
     int *hist;
     float *smax;
     int *wtot;
-    int *meta;           // [0] lookup table has at most one finite threshold per cell, [1..2] lo, scale (as bits)
+    int *meta;           // [0] lookup table has at most one finite threshold per cell, [1..2] lo, scale (as bits),
+                         // [3] the thresholds are evenly spaced enough for direct binning, [4..5] its scale, shift
     unsigned short *lut; // lut_cells + 1 entries (tiled kernel only)
     float *wmx;          // rule 1, plain kernel: warp totals of the prefix-maximum scan
     float *fmax;         // rule 1: [nbuf][hist_copies][hist_stride], laid out like hist: largest finish time among
@@ -370,6 +372,23 @@ __device__ __forceinline__ unsigned lut_cell(float x, float lo, float scale, uns
     return min(__float2uint_rz(__fmul_rn(__fsub_rn(x, lo), scale)), C);  // negative and NaN -> 0, huge -> C
 }
 
+// Direct binning for evenly spaced thresholds, without the table.  dcell(x) = min(uint(x * dscale + dshift), K) with
+// dscale = (K-1) / (tau_{K-1} - tau_0) and dshift = 0.5 - tau_0 * dscale puts tau_k in the middle of cell k.  It is
+// used only if dcell(tau_k) == k holds for EVERY k (checked below with the same instruction sequence).  dcell is
+// monotone (one fused multiply-add, one truncation, one minimum), hence for a sample P with c = dcell(P):
+// k < c gives dcell(tau_k) < dcell(P), so tau_k < P; k > c gives tau_k > P; and tau_c is compared directly:
+//     j(P) = c + [P >= tau_c]        (tau_K = +inf)
+__device__ __forceinline__ unsigned direct_cell(float x, float dscale, float dshift, unsigned K)
+{
+    return min(__float2uint_rz(__fmaf_rn(x, dscale, dshift)), K);  // negative and NaN -> 0, huge -> K
+}
+__device__ __forceinline__ unsigned direct_offset(float P, float dscale, float dshift, unsigned K, const unsigned char *tau_b)
+{
+    unsigned off = 4u * direct_cell(P, dscale, dshift, K);
+    off += (P >= *reinterpret_cast<const float *>(tau_b + off)) ? 4u : 0u;
+    return off;
+}
+
 // All threads of the block; tau_s[0..K] is loaded (tau_s[K] = +inf).  Ends with __syncthreads().
 __device__ __forceinline__ void build_lut(const SweepParams &p, const SmemTail &s, int tid, int nthr)
 {
@@ -390,6 +409,18 @@ __device__ __forceinline__ void build_lut(const SweepParams &p, const SmemTail &
         s.meta[0] = 1;
         s.meta[1] = __float_as_int(lo);
         s.meta[2] = __float_as_int(scale);
+        // direct binning: all thresholds finite, checked cell by cell after the barrier
+        float dscale = 0.0f;
+        const bool finite = (klo == 0 && khi == K - 1);
+        if (finite && K > 1) {
+            const float range = __fsub_rn(s.tau_s[K - 1], s.tau_s[0]);
+            if (range > 0.0f && range < pinf) dscale = __fdiv_rn((float)(K - 1), range);
+            if (!(dscale < pinf)) dscale = 0.0f;
+        }
+        const float dshift = finite ? __fmaf_rn(-s.tau_s[0], dscale, 0.5f) : 0.0f;
+        s.meta[3] = (finite && dshift == dshift && fabsf(dshift) < pinf) ? 1 : 0;
+        s.meta[4] = __float_as_int(dscale);
+        s.meta[5] = __float_as_int(dshift);
     }
     for (unsigned c = tid; c <= C; c += nthr) s.lut[c] = 0;
     __syncthreads();
@@ -408,6 +439,8 @@ __device__ __forceinline__ void build_lut(const SweepParams &p, const SmemTail &
         const int last = min(cur, (int)C);
         for (int c = prev + 1; c <= last; ++c) s.lut[c] = (unsigned short)(4 * k);  // byte offset of the smallest k with cx(k) >= c
         if (k > 0 && k < K && cur == prev && cur >= 0 && cur <= (int)C) s.meta[0] = 0;  // two finite thresholds share a cell
+        if (k < K && direct_cell(s.tau_s[k], __int_as_float(s.meta[4]), __int_as_float(s.meta[5]), (unsigned)K) != (unsigned)k)
+            s.meta[3] = 0;  // threshold k is not in cell k: no direct binning
     }
     __syncthreads();
 }
@@ -463,6 +496,8 @@ struct BinCtx {
     const unsigned char *tau_b;
     unsigned K4;
     bool one;                 // the table guarantees at most one threshold to step over
+    float dscale, dshift;     // direct binning (only used when the grid qualifies)
+    unsigned K;
     float tau_first, tau_last;
     uint32_t arrive_one;      // always 1, opaque to the compiler (ties a stage release to a warp vote)
 };
@@ -481,7 +516,8 @@ __device__ __forceinline__ float &sample_ref(float4 (&v)[NQ], int e)
 
 // Rule 1 keeps, besides the count of bin-0 samples (cnt0), the largest finish time among them (fin0), and the bin
 // `prev` (byte offset) of the running time before the next micro-batch.
-template <int NQ, int RULE, bool BATCH>
+// DIRECT = evenly spaced thresholds binned arithmetically (direct_offset) instead of through the table.
+template <int NQ, int RULE, bool BATCH, bool DIRECT>
 __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool valid, int lane, const BinCtx &c,
                                               unsigned char *hist_b, unsigned fmax_delta, float &P, unsigned &prev,
                                               int &cnt0, float &fin0, uint64_t *release_bar)
@@ -527,9 +563,14 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
                     if (valid) {
                         if (c.one && gs == GS) {
                             unsigned off[GS];
+                            if (DIRECT) {
 #pragma unroll
-                            for (int e = 0; e < GS; ++e)
-                                off[e] = bin_offset<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
+                                for (int e = 0; e < GS; ++e) off[e] = direct_offset(sample_ref(v, g + e), c.dscale, c.dshift, c.K, c.tau_b);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < GS; ++e)
+                                    off[e] = bin_offset<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
+                            }
 #pragma unroll
                             for (int e = 0; e < GS; ++e) {
                                 start_rule_update(sample_ref(v, g + e), prev, hist_b, fmax_delta, cnt0, fin0);
@@ -555,11 +596,20 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
                             // all table and threshold reads of the group first (independent chains that
                             // overlap), then the histogram updates: lower latency per group
                             unsigned off[GS];
+                            if (DIRECT) {
 #pragma unroll
-                            for (int e = 0; e < GS; ++e)
-                                off[e] = bin_offset<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
+                                for (int e = 0; e < GS; ++e) off[e] = direct_offset(sample_ref(v, g + e), c.dscale, c.dshift, c.K, c.tau_b);
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < GS; ++e)
+                                    off[e] = bin_offset<true>(sample_ref(v, g + e), c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
+                            }
 #pragma unroll
                             for (int e = 0; e < GS; ++e) atomicAdd(reinterpret_cast<int *>(hist_b + off[e]), 1);
+                        } else if (DIRECT) {
+#pragma unroll
+                            for (int e = 0; e < GS; ++e)
+                                atomicAdd(reinterpret_cast<int *>(hist_b + direct_offset(sample_ref(v, g + e), c.dscale, c.dshift, c.K, c.tau_b)), 1);
                         } else {
 #pragma unroll
                             for (int e = 0; e < GS; ++e)
@@ -735,6 +785,62 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
     }
 }
 
+// The consumer threads' loop over the block's trials (tiled kernel).
+template <int NQ, int RULE, bool BATCH, bool DIRECT>
+__device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTail &s, const BinCtx &ctx, unsigned char *stage0,
+                                             uint64_t *full, uint64_t *empty, int tid, int lane, int warp, int ncw,
+                                             int *myhist0, unsigned fmax_delta, unsigned off_zero)
+{
+    const int S = p.stages;
+    const int bar_threads = ncw * 32 + 32;
+    const int hist_buf_ints = p.hist_copies * p.hist_stride;
+    // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
+    // (threads past the last row of the box read the last row instead: always inside the stage)
+    const uint32_t row_off = (uint32_t)min(tid, p.rows - 1) * (uint32_t)p.pitch;
+    const uint32_t swz = ((row_off >> 7) & (uint32_t)p.swz_mask) << 4;
+    int st = 0;
+    uint32_t ph = 0;
+    int j = 0;
+    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
+        const int b = j & 1;
+        if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
+        int *myhist = myhist0 + b * hist_buf_ints;
+        unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
+        float rowmax = 0.0f, fin0 = 0.0f;
+        int cnt0 = 0;
+        for (int pass = 0; pass < p.passes; ++pass) {
+            const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
+            float P = 0.0f;
+            unsigned prev = off_zero;  // rule 1: bin (byte offset) of the running time before the next micro-batch
+            for (int c = 0; c < p.chunks; ++c) {
+                mbar_wait(&full[st], ph, kErrLoadNeverArrived);
+                const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes + row_off;
+                uint64_t *empty_bar = &empty[st];
+                if (++st == S) {
+                    st = 0;
+                    ph ^= 1u;
+                }
+                const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
+                float4 v[NQ];
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
+                    else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                }
+                consume_chunk<NQ, RULE, BATCH, DIRECT>(v, 4 * nq, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, empty_bar);
+            }
+            if (valid) rowmax = fmaxf(rowmax, P);
+        }
+        if (cnt0 > 0) {
+            atomicAdd(myhist, cnt0);
+            if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
+        }
+        rowmax = warp_max(rowmax);
+        if (lane == 0) s.smax[32 * b + warp] = rowmax;
+        buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
+    }
+}
+
 template <int NQ, int RULE, bool BATCH>
 __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2)
 dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
@@ -803,9 +909,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     }
 
     // ---------------- consumers
-    const int bar_threads = ncw * 32 + 32;
     const int K = p.K;
-    const int hist_buf_ints = p.hist_copies * p.hist_stride;
     int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
     // rule 1: byte distance from a histogram entry to the finish-time maximum of the same buffer, copy and bin
     const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));
@@ -822,57 +926,19 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     ctx.tau_b = tau_b;
     ctx.K4 = K4;
     ctx.one = one;
+    ctx.dscale = __int_as_float(s.meta[4]);
+    ctx.dshift = __int_as_float(s.meta[5]);
+    ctx.K = (unsigned)K;
     ctx.tau_first = s.tau_s[0];
     ctx.tau_last = s.tau_s[K - 1];
     ctx.arrive_one = (uint32_t)p.one;
     // rule 1 only: the bin of a running time of 0
     unsigned off_zero = 0;
     if (RULE == 1) off_zero = bin_offset<false>(0.0f, lut_lo, lut_scale, C, s.lut, tau_b, K4);
-    // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
-    // (threads past the last row of the box read the last row instead: always inside the stage)
-    const uint32_t row_off = (uint32_t)min(tid, p.rows - 1) * (uint32_t)p.pitch;
-    const uint32_t swz = ((row_off >> 7) & (uint32_t)p.swz_mask) << 4;
-    int st = 0;
-    uint32_t ph = 0;
-    int j = 0;
-    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
-        const int b = j & 1;
-        if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
-        int *myhist = myhist0 + b * hist_buf_ints;
-        unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
-        float rowmax = 0.0f, fin0 = 0.0f;
-        int cnt0 = 0;
-        for (int pass = 0; pass < p.passes; ++pass) {
-            const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
-            float P = 0.0f;
-            unsigned prev = off_zero;  // rule 1: bin (byte offset) of the running time before the next micro-batch
-            for (int c = 0; c < p.chunks; ++c) {
-                mbar_wait(&full[st], ph, kErrLoadNeverArrived);
-                const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes + row_off;
-                uint64_t *empty_bar = &empty[st];
-                if (++st == S) {
-                    st = 0;
-                    ph ^= 1u;
-                }
-                const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
-                float4 v[NQ];
-#pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
-                    else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                }
-                consume_chunk<NQ, RULE, BATCH>(v, 4 * nq, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, empty_bar);
-            }
-            if (valid) rowmax = fmaxf(rowmax, P);
-        }
-        if (cnt0 > 0) {
-            atomicAdd(myhist, cnt0);
-            if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
-        }
-        rowmax = warp_max(rowmax);
-        if (lane == 0) s.smax[32 * b + warp] = rowmax;
-        buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
-    }
+    if (s.meta[3] != 0 && one && p.direct_bins != 0)
+        tiled_trials<NQ, RULE, BATCH, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, myhist0, fmax_delta, off_zero);
+    else
+        tiled_trials<NQ, RULE, BATCH, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, myhist0, fmax_delta, off_zero);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -971,6 +1037,9 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
     ctx.tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
     ctx.K4 = 4u * (unsigned)K;
     ctx.one = s.meta[0] != 0;
+    ctx.dscale = __int_as_float(s.meta[4]);
+    ctx.dshift = __int_as_float(s.meta[5]);
+    ctx.K = (unsigned)K;
     ctx.tau_first = s.tau_s[0];
     ctx.tau_last = s.tau_s[K - 1];
     ctx.arrive_one = (uint32_t)p.one;
@@ -1006,7 +1075,7 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
                 float4 v[8];
 #pragma unroll
                 for (int e = 0; e < 32; ++e) sample_ref(v, e) = (e < ns) ? row[m0 + e] : 0.0f;
-                consume_chunk<8, RULE, BATCH>(v, ns, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0,
+                consume_chunk<8, RULE, BATCH, false>(v, ns, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0,
                                               (m0 + 32 >= M) ? empty_bar : nullptr);
             }
             if (valid) rowmax = fmaxf(rowmax, P);
@@ -1369,6 +1438,7 @@ int g_tune_lane_copies = 0;  // 0 = automatic
 int g_tune_warp_groups = 0;  // 0 = automatic
 int g_tune_box_floats = 0;   // 0 = automatic
 int g_tune_batch = 0;        // 0 = automatic, 1 = off, 2 = on
+int g_tune_direct = 0;       // 0 = automatic (on), 1 = off, 2 = on
 int g_last_simulate_launches = 0;
 int g_last_reduce_launches = 0;
 int g_last_argmax_launches = 0;
@@ -1457,6 +1527,9 @@ int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const 
     // Rows that fit one tile gain from looking up a whole group's bins before touching the histogram (the
     // chains overlap); longer rows measured faster with lookups and updates interleaved.
     p.batch_lookups = g_tune_batch > 0 ? g_tune_batch - 1 : (p.chunks == 1 ? 1 : 0);
+    // Arithmetic binning of evenly spaced thresholds measured faster wherever a group's bins are computed before
+    // its updates (rows of one tile, and the start-before-tau rule), slower for long rows under the paper's rule.
+    p.direct_bins = g_tune_direct > 0 ? g_tune_direct - 1 : ((rule == DC_RULE_START_BEFORE_TAU || p.chunks == 1) ? 1 : 0);
     // Shared memory per block: aim at two resident blocks per SM.  Histogram copies: lane l of warp w
     // adds into copy (w % warp_groups) * lane_copies + (l % lane_copies); copies used by one warp start
     // 32 / lane_copies banks apart so that equal bins of different lanes do not collide.
@@ -2000,6 +2073,10 @@ int dc_tune(int32_t key, int32_t value)
     }
     if (key == DC_TUNE_BATCH_LOOKUPS && value >= 0 && value <= 2) {
         g_tune_batch = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_DIRECT_BINS && value >= 0 && value <= 2) {
+        g_tune_direct = value;
         return DC_OK;
     }
     if (key == DC_TUNE_BOX_FLOATS && (value == 0 || value == 16 || value == 32)) {

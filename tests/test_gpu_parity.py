@@ -341,6 +341,39 @@ def test_results_do_not_depend_on_tuning_or_timing(api):
     api.dc_device_status()
 
 
+@pytest.mark.parametrize("rule", [0, 1])
+def test_direct_and_table_binning_agree_with_oracle(api, rule):
+    """Evenly spaced grids are binned arithmetically, every other grid through the lookup table; both must
+    give the oracle's bits.  Grids: exact dyadic steps with samples ON the thresholds, float32 linspace grids
+    of awkward ranges, a single threshold, a two-point grid, and a nearly even grid (falls back to the table)."""
+    rng = np.random.default_rng(11)
+    cases = []
+    lat = W.iid_latencies("dyadic", 5, 70, 24, seed=31, hi=8).numpy()
+    cases.append((lat, np.arange(48, dtype=np.float32) / 16.0))
+    lat = W.iid_latencies("uniform", 4, 300, 36, seed=32, lo=0.0, hi=0.05).numpy()
+    cases.append((lat, np.linspace(0.3, 1.1, 129).astype(np.float32)))
+    cases.append((lat, np.linspace(0.9, 0.9000305, 64).astype(np.float32)))   # steps of a few ulps
+    cases.append((lat, np.linspace(-0.2, 3.0, 7).astype(np.float32)))
+    cases.append((lat, np.array([0.7], np.float32)))
+    cases.append((lat, np.array([0.5, 0.9], np.float32)))
+    g = np.linspace(0.3, 1.1, 200)
+    g[1:-1] += rng.uniform(-0.4, 0.4, 198) * (g[1] - g[0])                      # uneven: table
+    cases.append((lat, np.sort(g).astype(np.float32)))
+    lat = W.iid_latencies("uniform", 3, 2048, 128, seed=33, lo=0.0, hi=0.014).numpy()
+    cases.append((lat, np.linspace(0.6 * 0.896, 1.4 * 0.896, 256).astype(np.float32)))
+    try:
+        for lat, taus in cases:
+            ref = oracle.sweep(lat, taus, 0.1, rule=rule)
+            lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+            for mode in (1, 2):
+                api.dc_tune(api.TUNE_DIRECT_BINS, mode)
+                res = run_gpu(api, lat_d, taus_d, 0.1, rule=rule)
+                compare_sweep(res, ref, f"(K={len(taus)}, direct bins {'on' if mode == 2 else 'off'})")
+    finally:
+        api.dc_tune(api.TUNE_DIRECT_BINS, 0)
+    api.dc_device_status()
+
+
 # ---- the start-before-tau rule (timeout looked at between accumulations) ---------------------------
 
 @pytest.mark.parametrize("T,N,M,K", EDGE_SHAPES)

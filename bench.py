@@ -284,6 +284,22 @@ def run_ours(args, w: W.Workload):
     clocks = sampler.stop(t_mark0, t_mark1) if rank == 0 else None
     api.dc_device_status()
 
+    # a plain read-only pass over the same latency bytes, under the same flush regime (context for the roofline
+    # fraction: short passes do not reach the bandwidth a long copy measures)
+    sink = torch.zeros((1,), dtype=torch.float32, device=dev)
+    probe_ms = []
+    for i in range(8):
+        if flush is not None:
+            flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        api.dc_read_probe(lat, sink)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            probe_ms.append(e0.elapsed_time(e1))
+    read_probe_ms = statistics.median(probe_ms)
+
     samples = T * N * M
     value_sps = world * args.steps * samples / (total_ms * 1e-3)
     sim_avg_s = (sum(sim_ms) / len(sim_ms)) * 1e-3
@@ -304,9 +320,11 @@ def run_ours(args, w: W.Workload):
         "sweep_ms": sim_avg_s * 1e3,
         "sweep_ms_best": min(sim_ms),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "kernel": "dc_sweep_tiled" if api.dc_simulate_plan(lat, K) == 0 else "dc_sweep_plain",
+                     "traffic": traffic, "kernel": ("dc_sweep_tiled", "dc_sweep_plain", "dc_sweep_flat")[api.dc_simulate_plan(lat, K)],
                      "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": alg_bytes,
-                     "frac_of_nominal_8TBs": achieved / 8000.0},
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "read_only_pass_ms": read_probe_ms, "read_only_pass_gbs": 4 * samples / (read_probe_ms * 1e-3) / 1e9,
+                     "sweep_over_read_only_pass": (sim_avg_s * 1e3) / read_probe_ms},
         "gpu_launches": args.steps * sum(api.launches().values()),
         "clocks": clocks,
     }

@@ -234,6 +234,15 @@ int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M,
                   void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * dc_read_probe — measurement aid with no counterpart in the paper: enqueues a kernel that reads
+ * data[0 .. count - count % 4) once with 16-byte loads and does nothing else.  Timed on a latency tensor it gives
+ * the duration of a plain read-only pass over those bytes, which benchmarks report beside the sweep's.
+ *   data   DEVICE, 16-byte aligned, count floats (all >= 0, as latencies are)
+ *   sink   DEVICE, one float; never written for such data
+ */
+int dc_read_probe(const float *data, int64_t count, float *sink, void *stream);
+
+/*
  * dc_check_inputs — SYNCHRONOUS check of the data preconditions of dc_simulate on `stream`:
  * returns DC_ERR_LATENCIES if any latency is negative, NaN or infinite, DC_ERR_TAUS if the grid is
  * not non-decreasing or holds a NaN, DC_OK otherwise.  report_host (HOST, [2] int64, may be NULL)

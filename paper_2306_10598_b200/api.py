@@ -27,7 +27,7 @@ EXPORTS = (
     "dc_simulate", "dc_simulate_ex", "dc_simulate_tc", "dc_simulate_split_workspace_bytes", "dc_simulate_split",
     "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_reduce_trials_static",
     "dc_argmax_tau",
-    "dc_closed_form", "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan",
+    "dc_closed_form", "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan", "dc_read_probe",
     "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string", "dc_tune",
     "dc_kernel_version",
 )
@@ -68,6 +68,7 @@ _lib.dc_closed_form.argtypes = [ctypes.c_double, ctypes.c_double, _i64, _i64, ct
 _lib.dc_closed_form.restype = ctypes.c_int
 _lib.dc_check_inputs.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _p, _p, _p]
 _lib.dc_device_status.argtypes = [_p]
+_lib.dc_read_probe.argtypes = [_p, _i64, _p, _p]
 _lib.dc_simulate_plan.argtypes = [_p, _i64, _i64, _i64, _i32]
 _lib.dc_tune.argtypes = [_i32, _i32]
 _lib.dc_tune.restype = ctypes.c_int
@@ -241,6 +242,13 @@ def dc_check_inputs(latencies: torch.Tensor, taus: torch.Tensor) -> None:
     with torch.cuda.device(latencies.device):
         _check(_lib.dc_check_inputs(_dev(latencies, torch.float32, "latencies"), T, N, M, _dev(taus, torch.float32, "taus"),
                                     taus.shape[0], counters.data_ptr(), None, _stream(latencies)), "dc_check_inputs")
+
+
+def dc_read_probe(data: torch.Tensor, sink: torch.Tensor) -> None:
+    """Enqueues a plain read-only pass over `data` (a measurement aid; see the header)."""
+    with torch.cuda.device(data.device):
+        _check(_lib.dc_read_probe(_dev(data, torch.float32, "data"), data.numel(), _dev(sink, torch.float32, "sink"),
+                                  _stream(data)), "dc_read_probe")
 
 
 def dc_device_status() -> int:

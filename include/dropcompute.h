@@ -277,6 +277,10 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  *   DC_TUNE_BOX_FLOATS   floats of a row fetched per tile (16 or 32; 16 needs M to be a multiple of 16)
  *   DC_TUNE_DIRECT_BINS  1 = always bin through the lookup table, 2 = bin evenly spaced thresholds arithmetically
  *                        (one multiply-add and one comparison per sample, no table read) in the tiled kernel
+ *   DC_TUNE_FLAT_TILE_WARPS, DC_TUNE_FLAT_GROUPS, DC_TUNE_FLAT_DEPTH  flat kernel (row length not a multiple
+ *                        of 4): warps per tile (tile = 32 x that many rows), groups of warps working on different
+ *                        tiles at once, ring stages per group; used only when all three are set, and a setting
+ *                        whose tiles or ring do not fit makes dc_simulate* return DC_ERR_RANGE
  * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
  */
 #define DC_TUNE_STAGES 1
@@ -285,6 +289,9 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
 #define DC_TUNE_BOX_FLOATS 4
 #define DC_TUNE_BATCH_LOOKUPS 5
 #define DC_TUNE_DIRECT_BINS 6
+#define DC_TUNE_FLAT_TILE_WARPS 7
+#define DC_TUNE_FLAT_GROUPS 8
+#define DC_TUNE_FLAT_DEPTH 9
 int dc_tune(int32_t key, int32_t value);
 
 /* Number of kernel launches the last successful call of each entry point enqueues (for accounting). */

@@ -84,6 +84,8 @@ struct SweepParams {
     int batch_lookups; // tiled kernel: 1 = look up a whole group's bins before updating the histogram
     int nbuf;          // histogram / maxima buffers: 2 in the tiled kernel (filled and drained in turn), 1 in the plain one
     int one;           // always 1; a value the compiler cannot see, used to tie a stage release to a warp vote
+    int flat_groups;   // flat kernel: groups of consumer warps working on different tiles at the same time
+    int tile_warps;    // flat kernel: warps per group (rows / 32)
     int direct_bins;   // staged kernels: 1 = bin evenly spaced thresholds arithmetically instead of through the table
     int epi_vec;       // staged kernels: the epilogue warp may take four bins per lane with 16-byte accesses
                        // (K a multiple of 4, out_step / out_done 16-byte aligned, hist_stride a multiple of 4)
@@ -943,12 +945,17 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 
 // ------------------------------------------------------------------------------------------
 // Flat kernel: rows whose length is not a multiple of 4 (so a tensor map cannot describe them), up to
-// kFlatMaxM samples, base pointer 16-byte aligned.  A pass's rows are one contiguous span of the tensor; the
-// producer brings the 16-byte aligned span that covers them into a stage with ONE plain bulk copy
-// (cp.async.bulk, no tensor map) and thread r reads its row from float offset delta + r*M with 4-byte
-// shared loads, 32 samples at a time.  Everything after the loads is the tiled kernel's code (consume_chunk,
-// epilogue warp, double-buffered histograms).  The few floats past the last multiple of 4 of the whole
-// tensor cannot be bulk-copied in bounds; the producer moves them with ordinary loads.
+// kFlatMaxM samples, base pointer 16-byte aligned.  Consecutive rows of a trial are one contiguous span of the
+// tensor.  A tile is `rows` consecutive rows (a multiple of 32, at most 32 KB); the producer brings the 16-byte
+// aligned span that covers it into a stage with ONE plain bulk copy (cp.async.bulk, no tensor map) and thread r
+// of the tile's warps reads its row from float offset delta + r*M with 4-byte shared loads, 32 samples at a time.
+// Whole rows have to be resident, so long rows mean few rows per tile: the consumer warps are therefore split
+// into G groups of rows/32 warps, tile i goes to group i mod G, and the groups work on different tiles at the
+// same time.  The ring has a multiple of G stages, so a stage is only ever used by one group and each group sees
+// its own stages in order, like a ring of its own (for short rows G = 1: the tiled kernel's schedule).  Everything
+// after the loads is the tiled kernel's code (consume_chunk, epilogue warp, double-buffered histograms).  The
+// few floats past the last multiple of 4 of the whole tensor cannot be bulk-copied in bounds; the producer
+// moves them with ordinary loads.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
 {
@@ -970,49 +977,57 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int ncw = (blockDim.x >> 5) - 2;
     const int S = p.stages;
+    const int R = p.rows, Pt = p.passes, G = p.flat_groups, wpg = p.tile_warps;  // tiles per trial, groups, warps per group
     const unsigned long long NM = (unsigned long long)p.N * (unsigned long long)p.M;
     const unsigned long long total = (unsigned long long)p.T * NM;
     const unsigned long long total4 = total & ~3ull;
 
-    if (tid == 0) {
+    // the producer thread sets up the barriers and fills the ring before the block builds its tables
+    long long prod_t = blockIdx.x;
+    int prod_q = 0, prod_issued = 0;  // next tile: trial, tile inside the trial
+    auto issue_tile = [&](int st) {
+        const int row0 = prod_q * R;
+        const int nrows = min(R, p.N - row0);
+        const unsigned long long b0 = (unsigned long long)prod_t * NM + (unsigned long long)row0 * p.M;
+        const unsigned long long e0 = b0 + (unsigned long long)nrows * p.M;
+        const unsigned long long b4 = b0 & ~3ull;   // aligned start of the span
+        unsigned long long e4 = (e0 + 3ull) & ~3ull;  // aligned end, inside the tensor
+        if (e4 > total4) e4 = total4;
+        if (e4 < b4) e4 = b4;
+        float *dst = reinterpret_cast<float *>(stage0 + (size_t)st * p.stage_bytes);
+        for (unsigned long long i = e4; i < e0; ++i) dst[i - b4] = p.lat[i];  // at most 3 floats, last tile only
+        const uint32_t bytes = (uint32_t)((e4 - b4) * 4ull);
+        mbar_arrive_expect_tx(&full[st], bytes);
+        if (bytes != 0u) bulk_load_1d(dst, p.lat + b4, bytes, &full[st]);
+        if (++prod_q == Pt) {
+            prod_q = 0;
+            prod_t += gridDim.x;
+        }
+    };
+    if (warp == ncw && lane == 0) {
         for (int i = 0; i < S; ++i) {
             mbar_init(&full[i], 1);
-            mbar_init(&empty[i], ncw);
+            mbar_init(&empty[i], wpg);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        while (prod_issued < S && prod_t < p.T) issue_tile(prod_issued++);
     }
     load_thresholds(p, s, tid, blockDim.x);
-    __syncthreads();
+    __syncthreads();  // also: the initialised barriers are visible to every thread
     build_lut(p, s, tid, blockDim.x);
 
     if (warp == ncw) {
-        // ---------------- producer
+        // ---------------- producer: the rest of the tiles, in order, each into the stage tile i - S has left
         if (lane == 0) {
             int st = 0;
-            uint32_t ph = 0;
-            bool first = true;
-            for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
-                for (int pass = 0; pass < p.passes; ++pass) {
-                    const int row0 = pass * p.rows;
-                    const int nrows = min(p.rows, p.N - row0);
-                    const unsigned long long b0 = (unsigned long long)t * NM + (unsigned long long)row0 * p.M;
-                    const unsigned long long e0 = b0 + (unsigned long long)nrows * p.M;
-                    const unsigned long long b4 = b0 & ~3ull;                       // aligned start of the span
-                    unsigned long long e4 = (e0 + 3ull) & ~3ull;                      // aligned end, inside the tensor
-                    if (e4 > total4) e4 = total4;
-                    if (e4 < b4) e4 = b4;
-                    if (!first) mbar_wait(&empty[st], ph ^ 1u, kErrStageNeverFreed);
-                    float *dst = reinterpret_cast<float *>(stage0 + (size_t)st * p.stage_bytes);
-                    for (unsigned long long i = e4; i < e0; ++i) dst[i - b4] = p.lat[i];  // at most 3 floats, last tile only
-                    const uint32_t bytes = (uint32_t)((e4 - b4) * 4ull);
-                    mbar_arrive_expect_tx(&full[st], bytes);
-                    if (bytes != 0u) bulk_load_1d(dst, p.lat + b4, bytes, &full[st]);
-                    if (++st == S) {
-                        st = 0;
-                        ph ^= 1u;
-                        first = false;
-                    }
+            uint32_t ph = 1;
+            while (prod_t < p.T) {
+                mbar_wait(&empty[st], ph ^ 1u, kErrStageNeverFreed);
+                issue_tile(st);
+                if (++st == S) {
+                    st = 0;
+                    ph ^= 1u;
                 }
             }
         }
@@ -1045,9 +1060,14 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
     ctx.arrive_one = (uint32_t)p.one;
     unsigned off_zero = 0;
     if (RULE == 1) off_zero = bin_offset<false>(0.0f, ctx.lut_lo, ctx.lut_scale, ctx.C, ctx.lut, ctx.tau_b, ctx.K4);
-    const int myrow = min(tid, p.rows - 1);  // threads past the last row read the last row: always inside the stage
-    int st = 0;
-    uint32_t ph = 0;
+    const int grp = warp / wpg;
+    const int r = (warp - grp * wpg) * 32 + lane;  // this thread's row inside its group's tiles (< R)
+    // The block's tiles are numbered i = 0, 1, ... in the producer's order (trial, then tile inside the trial);
+    // tile i uses stage i mod S in ring phase i / S and belongs to group i mod G.  `rel` is this group's next
+    // tile counted from the current trial's first tile.
+    int rel = grp;
+    int st = grp % S;
+    uint32_t ph = (uint32_t)((grp / S) & 1);
     int j = 0;
     for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
         const int b = j & 1;
@@ -1056,18 +1076,20 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
         unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
         float rowmax = 0.0f, fin0 = 0.0f;
         int cnt0 = 0;
-        for (int pass = 0; pass < p.passes; ++pass) {
-            const int row0 = pass * p.rows;
-            const bool valid = (tid < p.rows) && (row0 + tid < p.N);
+        for (; rel < Pt; rel += G) {
+            const int row0 = rel * R;
+            const bool valid = row0 + r < p.N;
             const unsigned long long b0 = (unsigned long long)t * NM + (unsigned long long)row0 * M;
             const int delta = (int)(b0 & 3ull);
             float P = 0.0f;
             unsigned prev = off_zero;
             mbar_wait(&full[st], ph, kErrLoadNeverArrived);
-            const float *row = reinterpret_cast<const float *>(stage0 + (size_t)st * p.stage_bytes) + delta + myrow * M;
+            // (threads past the tile's last row read row r all the same: inside the stage, never counted)
+            const float *row = reinterpret_cast<const float *>(stage0 + (size_t)st * p.stage_bytes) + delta + r * M;
             uint64_t *empty_bar = &empty[st];
-            if (++st == S) {
-                st = 0;
+            st += G;
+            while (st >= S) {
+                st -= S;
                 ph ^= 1u;
             }
             for (int m0 = 0; m0 < M; m0 += 32) {
@@ -1076,10 +1098,11 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
 #pragma unroll
                 for (int e = 0; e < 32; ++e) sample_ref(v, e) = (e < ns) ? row[m0 + e] : 0.0f;
                 consume_chunk<8, RULE, BATCH, false>(v, ns, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0,
-                                              (m0 + 32 >= M) ? empty_bar : nullptr);
+                                                     (m0 + 32 >= M) ? empty_bar : nullptr);
             }
             if (valid) rowmax = fmaxf(rowmax, P);
         }
+        rel -= Pt;
         if (cnt0 > 0) {
             atomicAdd(myhist, cnt0);
             if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
@@ -1461,6 +1484,7 @@ int g_tune_warp_groups = 0;  // 0 = automatic
 int g_tune_box_floats = 0;   // 0 = automatic
 int g_tune_batch = 0;        // 0 = automatic, 1 = off, 2 = on
 int g_tune_direct = 0;       // 0 = automatic (on), 1 = off, 2 = on
+int g_tune_flat_tile_warps = 0, g_tune_flat_groups = 0, g_tune_flat_depth = 0;  // flat kernel; all three or none
 int g_last_simulate_launches = 0;
 int g_last_reduce_launches = 0;
 int g_last_argmax_launches = 0;
@@ -1543,7 +1567,8 @@ int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t
 
 // Shared-memory layout of a block of the staged kernels (tiled and flat): ring depth, histogram copies, table
 // size.  Needs p.stage_bytes, p.chunks and the row-thread count; fills the rest and the dynamic shared bytes.
-int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const DeviceInfo &di, size_t *smem_out)
+int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const DeviceInfo &di, size_t *smem_out,
+                        int stage_cap = 3)
 {
     p.lut_cells = min(kLutCellsMax, 4 * K);
     // Rows that fit one tile gain from looking up a whole group's bins before touching the histogram (the
@@ -1557,20 +1582,25 @@ int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const 
     // 32 / lane_copies banks apart so that equal bins of different lanes do not collide.
     p.nbuf = 2;
     const int ncw = row_threads / 32;
-    const size_t budget = (size_t)di.smem_per_sm / 2 - 1024 - 256;
+    const size_t budget2 = (size_t)di.smem_per_sm / 2 - 1024 - 256;  // two blocks per SM
     size_t smem = 0;
     bool fits = false;
     // Candidates: ring depth first (bytes in flight matter most), then histogram copies, from the
     // preferred configuration down to the smallest one.  The first that leaves room for two blocks per
     // SM wins; the smallest one is taken even if only one block fits.
     // (a ring deeper than three tiles measured slower on every workload, whatever the tile size)
-    const int s_max = g_tune_stages > 0 ? g_tune_stages : min(3, max(2, kStageBudgetBytes / p.stage_bytes));
-    const int s_min = g_tune_stages > 0 ? g_tune_stages : 2;
+    // (a negative stage_cap fixes the ring depth at -stage_cap: the flat kernel's groups x stages per group)
+    const int s_max = stage_cap < 0 ? -stage_cap
+                                    : (g_tune_stages > 0 ? g_tune_stages : min(stage_cap, max(2, kStageBudgetBytes / p.stage_bytes)));
+    const int s_min = stage_cap < 0 ? -stage_cap : (g_tune_stages > 0 ? g_tune_stages : 2);
     const int lc_first = g_tune_lane_copies > 0 ? g_tune_lane_copies : 4;
     const int lc_last = g_tune_lane_copies > 0 ? g_tune_lane_copies : 1;
     const int wg_first = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
     const int wg_last = g_tune_warp_groups > 0 ? wg_first : 1;
     const bool forced = g_tune_stages > 0 && g_tune_lane_copies > 0 && g_tune_warp_groups > 0;
+    // (when a fixed ring alone is too large for two blocks, the same search runs against one block's limit)
+    const size_t ring_min = (size_t)s_min * p.stage_bytes;
+    const size_t budget = (stage_cap < 0 && ring_min + 4096 > budget2) ? (size_t)di.max_smem_optin : budget2;
     for (int st = s_max; st >= s_min && !fits; --st) {
         for (int lc = lc_first; lc >= lc_last && !fits; lc >>= 1) {
             for (int wg = wg_first; wg >= wg_last && !fits; wg >>= 1) {
@@ -1685,18 +1715,39 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     }
 
     if (flat_ok(lat, M)) {
-        // rows per pass: as many whole rows as fit a 32 KB stage (a multiple of 32, at most 256)
-        int cap = (int)((32768 - 64) / (4 * M));
-        cap = min(kMaxRowsPerPass, (cap / 32) * 32);
-        p.passes = (int)((N + cap - 1) / cap);
-        p.rows = (int)((N + p.passes - 1) / p.passes);
-        const int flat_threads = ((p.rows + 31) / 32) * 32;
+        // rows per tile: 32 x the warps of a group, as many as fit a 32 KB stage (whole rows), at most 256 and no
+        // more than the trial has; groups: as many as eight consumer warps allow and the trial has tiles for
+        // Warps per tile wt: the largest power of two whose tile (32 wt whole rows) stays within 32 KB, no more than
+        // the trial has rows for.  Eight: one group, three stages (the tiled kernel's schedule).  Fewer: about six
+        // consumer warps in G groups with one stage each (the groups overlap each other; measured best on rows of
+        // 65, 126 and 255 samples against fewer groups with two stages each and against eight warps).
+        int best_wt = 8;
+        while (best_wt > 1 && (size_t)best_wt * 32 * (size_t)M * 4 + 32 > 32768) best_wt >>= 1;
+        const bool short_rows = best_wt == 8;
+        if ((int64_t)best_wt * 32 > N) best_wt = (int)((N + 31) / 32);
+        const int tiles = (int)((N + (int64_t)best_wt * 32 - 1) / ((int64_t)best_wt * 32));
+        int best_g = short_rows ? 1 : min(best_wt >= 4 ? 2 : 6 / best_wt, tiles);
+        int best_d = best_g == 1 ? 3 : 1;
+        if (g_tune_flat_tile_warps > 0 && g_tune_flat_groups > 0 && g_tune_flat_depth > 0) {
+            best_wt = g_tune_flat_tile_warps;
+            if ((int64_t)best_wt * 32 > N) best_wt = (int)((N + 31) / 32);
+            best_g = g_tune_flat_groups;
+            best_d = g_tune_flat_depth;
+            if (best_g * best_wt > 8 || best_g * best_d > kMaxStages) return DC_ERR_RANGE;
+        }
+        if (best_wt <= 0) return DC_ERR_RANGE;
+        const int wt = best_wt;
+        p.rows = wt * 32;
+        p.tile_warps = wt;
+        p.passes = (int)((N + p.rows - 1) / p.rows);
+        p.flat_groups = min(best_g, p.passes);
+        const int flat_threads = p.flat_groups * wt * 32;
         p.bw = (int)M;
         p.chunks = (int)((M + 31) / 32);
         p.pitch = (int)M * 4;
         p.stage_bytes = (int)((((size_t)p.rows * M * 4 + 32) + 1023) / 1024 * 1024);
         size_t smem = 0;
-        const int lrc0 = choose_block_layout(p, flat_threads, K, rule, di, &smem);
+        const int lrc0 = choose_block_layout(p, flat_threads, K, rule, di, &smem, -(p.flat_groups * best_d));
         if (lrc0 != DC_OK) return lrc0;
         if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
         const int block = flat_threads + 64;
@@ -2108,6 +2159,18 @@ int dc_tune(int32_t key, int32_t value)
     }
     if (key == DC_TUNE_BATCH_LOOKUPS && value >= 0 && value <= 2) {
         g_tune_batch = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_FLAT_TILE_WARPS && value >= 0 && value <= 8) {
+        g_tune_flat_tile_warps = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_FLAT_GROUPS && value >= 0 && value <= 8) {
+        g_tune_flat_groups = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_FLAT_DEPTH && value >= 0 && value <= 4) {
+        g_tune_flat_depth = value;
         return DC_OK;
     }
     if (key == DC_TUNE_DIRECT_BINS && value >= 0 && value <= 2) {

@@ -535,12 +535,14 @@ def test_random_shapes_and_grids(api):
 
 
 def test_flat_kernel_shapes(api):
-    """Rows whose length is not a multiple of 4 (flat kernel: one bulk copy per pass, 4-byte shared loads):
+    """Rows whose length is not a multiple of 4 (flat kernel: one bulk copy per tile, 4-byte shared loads):
     spans that start at every offset modulo 4, a tensor whose size is not a multiple of 4 (its last floats
-    are moved by ordinary loads), several passes, the longest supported row, both rules, and repeated runs
-    under different ring depths."""
+    are moved by ordinary loads), several tiles per trial, the longest supported row, both rules, and repeated
+    runs under different splits of the consumer warps (warps per tile, groups working on different tiles at
+    once, ring stages per group), including more groups than a trial has tiles and trials that end mid-ring."""
     cases = [(7, 3, 5, 9), (5, 1, 1, 3), (3, 257, 30, 64), (6, 513, 6, 33), (4, 100, 255, 40), (9, 64, 33, 100),
-             (11, 37, 10, 16), (2, 2048, 126, 256), (64, 200, 14, 64)]
+             (11, 37, 10, 16), (2, 2048, 126, 256), (64, 200, 14, 64), (13, 300, 65, 48), (5, 1000, 127, 32)]
+    splits = [(0, 0, 0), (1, 8, 1), (1, 4, 2), (2, 4, 1), (2, 2, 2), (1, 3, 2), (4, 2, 1), (1, 5, 1), (8, 1, 2)]
     try:
         for (T, N, M, K) in cases:
             lat = W.iid_latencies("shifted_exp", T, N, M, seed=900 + T + N + M, shift=0.01, mean=0.02).numpy()
@@ -549,12 +551,22 @@ def test_flat_kernel_shapes(api):
             assert api.dc_simulate_plan(lat_d, K) == 2
             for rule in (0, 1):
                 ref = oracle.sweep(lat, taus, 0.07, rule=rule)
-                for stages in (0, 2, 3):
-                    api.dc_tune(api.TUNE_STAGES, stages)
-                    res = run_gpu(api, lat_d, taus_d, 0.07, rule=rule)
-                    compare_sweep(res, ref, f"flat {(T, N, M, K)} rule {rule} stages {stages}")
+                for (wt, groups, depth) in splits:
+                    if wt and wt * 32 * M * 4 + 32 > 32768 * 3:
+                        continue  # such a tile would not fit the shared memory of a block
+                    api.dc_tune(api.TUNE_FLAT_TILE_WARPS, wt)
+                    api.dc_tune(api.TUNE_FLAT_GROUPS, groups)
+                    api.dc_tune(api.TUNE_FLAT_DEPTH, depth)
+                    try:
+                        res = run_gpu(api, lat_d, taus_d, 0.07, rule=rule)
+                    except api.DropComputeError as e:
+                        assert e.status == 4 and wt, (e.status, wt, groups, depth)   # a forced split that does not fit
+                        continue
+                    compare_sweep(res, ref, f"flat {(T, N, M, K)} rule {rule} split {(wt, groups, depth)}")
     finally:
-        api.dc_tune(api.TUNE_STAGES, 0)
+        api.dc_tune(api.TUNE_FLAT_TILE_WARPS, 0)
+        api.dc_tune(api.TUNE_FLAT_GROUPS, 0)
+        api.dc_tune(api.TUNE_FLAT_DEPTH, 0)
     api.dc_device_status()
 
 

@@ -2196,7 +2196,7 @@ int dc_simulate_launches(void) { return g_last_simulate_launches; }
 int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
 int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
 
-const char *dc_kernel_version(void) { return "sweep-tiled-12"; }
+const char *dc_kernel_version(void) { return "sweep-tiled-13"; }
 
 const char *dc_status_string(int status)
 {

@@ -197,6 +197,18 @@ int dc_argmax_tau(const double *stats, const float *taus, int32_t K, int32_t obj
                   int32_t *out_k, float *out_tau, double *out_value, void *stream);
 
 /*
+ * dc_sweep_device — Algorithm 2 from samples to tau* in one host call, everything resident on the DEVICE:
+ * enqueues dc_simulate_ex, dc_reduce_trials and dc_argmax_tau on `stream`, in that order, with the arguments
+ * documented there (out_sync is required here).  Host-visible errors of any of the three are reported before
+ * anything is enqueued.  workspace as for dc_reduce_trials (dc_reduce_workspace_bytes(T, K) bytes).
+ */
+int dc_sweep_device(const float *latencies, int64_t T, int64_t N, int64_t M,
+                    const float *taus, int32_t K, float t_comm, int32_t rule, int32_t objective,
+                    float *out_step, int32_t *out_done, float *out_sync,
+                    double *stats, double *baseline, int32_t *out_k, float *out_tau, double *out_value,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * dc_closed_form — the paper's analytical estimates (App. C.2) on a threshold grid, from the mean `mu` and
  * standard deviation `sigma` of ONE micro-batch latency, for comparison with the simulation (Fig. 3):
  *   out[0][k] = E[M~(tau_k)] / M        = (1/M) sum_{m=1..M} Phi((tau_k - m mu) / sqrt(m sigma^2))     (Eq. 5 / 10)

@@ -26,7 +26,7 @@ STAT_NAMES = ("mean_step", "done_frac", "thr", "thr_mean", "s_eff")
 EXPORTS = (
     "dc_simulate", "dc_simulate_ex", "dc_simulate_tc", "dc_simulate_split_workspace_bytes", "dc_simulate_split",
     "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_reduce_trials_static",
-    "dc_argmax_tau",
+    "dc_argmax_tau", "dc_sweep_device",
     "dc_closed_form", "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan", "dc_read_probe",
     "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string", "dc_tune",
     "dc_kernel_version",
@@ -61,6 +61,7 @@ _lib.dc_reduce_trials.argtypes = [_p, _p, _p, _i64, _i32, _i64, _i64, _p, _p, _p
 _lib.dc_reduce_trials_static.argtypes = [_p, _p, _p, _i64, _i32, _i64, _i64, _p, _p, _p]
 _lib.dc_reduce_trials_static.restype = ctypes.c_int
 _lib.dc_argmax_tau.argtypes = [_p, _p, _i32, _i32, _p, _p, _p, _p]
+_lib.dc_sweep_device.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _i32, _i32, _p, _p, _p, _p, _p, _p, _p, _p, _p, _sz, _p]
 _lib.dc_sweep_host_workspace_bytes.argtypes = [_i64, _i64, _i64, _i32, _i64]
 _lib.dc_sweep_host_workspace_bytes.restype = _sz
 _lib.dc_sweep_host.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _i32, _i32, _i64, _p, _p, _p, _p, _p, _sz, _p]
@@ -322,6 +323,25 @@ class SweepResult(NamedTuple):
     k_star: torch.Tensor     # int32 scalar (device)
     tau_star: torch.Tensor   # fp32 scalar (device)
     value: torch.Tensor      # fp64 scalar (device)
+
+
+def dc_sweep_device(latencies: torch.Tensor, taus: torch.Tensor, t_comm: float, rule: int, objective: int,
+                    out_step: torch.Tensor, out_done: torch.Tensor, out_sync: torch.Tensor, stats: torch.Tensor,
+                    baseline: torch.Tensor, out_k: torch.Tensor, out_tau: torch.Tensor, out_value: torch.Tensor,
+                    workspace: torch.Tensor) -> None:
+    """dc_simulate_ex + dc_reduce_trials + dc_argmax_tau enqueued by one call into the library."""
+    T, N, M = latencies.shape
+    K = taus.shape[0]
+    assert tuple(out_step.shape) == (T, K) and tuple(out_done.shape) == (T, K) and tuple(out_sync.shape) == (T,)
+    assert tuple(stats.shape) == (NSTATS, K) and baseline.numel() == 2
+    with torch.cuda.device(latencies.device):
+        _check(_lib.dc_sweep_device(
+            _dev(latencies, torch.float32, "latencies"), T, N, M, _dev(taus, torch.float32, "taus"), K, float(t_comm),
+            int(rule), int(objective), _dev(out_step, torch.float32, "out_step"), _dev(out_done, torch.int32, "out_done"),
+            _dev(out_sync, torch.float32, "out_sync"), _dev(stats, torch.float64, "stats"),
+            _dev(baseline, torch.float64, "baseline"), _dev(out_k, torch.int32, "out_k"),
+            _dev(out_tau, torch.float32, "out_tau"), _dev(out_value, torch.float64, "out_value"),
+            _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(latencies)), "dc_sweep_device")
 
 
 def sweep(latencies: torch.Tensor, taus: torch.Tensor, t_comm: float, rule: int = RULE_FINISH_BEFORE_TAU,

@@ -1976,6 +1976,28 @@ int dc_argmax_tau(const double *stats, const float *taus, int32_t K, int32_t obj
     return DC_OK;
 }
 
+int dc_sweep_device(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K, float t_comm,
+                    int32_t rule, int32_t objective, float *out_step, int32_t *out_done, float *out_sync, double *stats,
+                    double *baseline, int32_t *out_k, float *out_tau, double *out_value, void *workspace,
+                    size_t workspace_bytes, void *stream)
+{
+    // everything the three steps would refuse is refused before the first of them is enqueued
+    if (!out_sync || !stats || !baseline || !out_k || !out_tau || !out_value) return DC_ERR_NULL;
+    int rc = validate_simulate(latencies, T, N, M, taus, K, out_step, out_done, rule);
+    if (rc != DC_OK) return rc;
+    if (objective != DC_STAT_S_EFF && objective != DC_STAT_THR && objective != DC_STAT_THR_MEAN) return DC_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(stats) & 7) || (reinterpret_cast<uintptr_t>(baseline) & 7) ||
+        (reinterpret_cast<uintptr_t>(out_value) & 7) || (reinterpret_cast<uintptr_t>(out_sync) & 3))
+        return DC_ERR_ALIGN;
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 7) || workspace_bytes < dc_reduce_workspace_bytes(T, K))
+        return DC_ERR_WORKSPACE;
+    rc = simulate_impl(latencies, T, N, M, taus, K, t_comm, nullptr, out_step, out_done, out_sync, rule, stream);
+    if (rc != DC_OK) return rc;
+    rc = dc_reduce_trials(out_step, out_done, out_sync, T, K, N, M, stats, baseline, workspace, workspace_bytes, stream);
+    if (rc != DC_OK) return rc;
+    return dc_argmax_tau(stats, taus, K, objective, out_k, out_tau, out_value, stream);
+}
+
 int dc_closed_form(double mu, double sigma, int64_t M, int64_t N, double t_comm, double mean_T, const float *taus,
                    int32_t K, double *out, double *scalars, void *stream_v)
 {

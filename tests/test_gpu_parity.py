@@ -184,6 +184,39 @@ def test_objectives(api):
     assert torch.equal(stats[:4], res.stats[:4])
 
 
+@pytest.mark.parametrize("rule,objective", [(0, 4), (1, 2), (0, 3)])
+def test_sweep_device_equals_the_three_calls(api, rule, objective):
+    """dc_sweep_device enqueues the same three steps: every output must carry the same bits as the separate calls,
+    and errors any of the steps would raise are raised before anything runs."""
+    T, N, M, K = 37, 300, 36, 40
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=77, shift=0.01, mean=0.02).numpy()
+    taus = grid_for(lat, K, 4)
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    ref = run_gpu(api, lat_d, taus_d, 0.15, rule=rule, objective=objective)
+    step = torch.empty((T, K), dtype=torch.float32, device="cuda")
+    done = torch.empty((T, K), dtype=torch.int32, device="cuda")
+    sync = torch.empty((T,), dtype=torch.float32, device="cuda")
+    stats = torch.empty((api.NSTATS, K), dtype=torch.float64, device="cuda")
+    base = torch.empty((2,), dtype=torch.float64, device="cuda")
+    k = torch.empty((), dtype=torch.int32, device="cuda")
+    tau = torch.empty((), dtype=torch.float32, device="cuda")
+    val = torch.empty((), dtype=torch.float64, device="cuda")
+    ws = torch.empty((api.dc_reduce_workspace_bytes(T, K),), dtype=torch.uint8, device="cuda")
+    api.dc_sweep_device(lat_d, taus_d, 0.15, rule, objective, step, done, sync, stats, base, k, tau, val, ws)
+    torch.cuda.synchronize()
+    for a, b in zip((step, done, sync, stats, base, k, tau, val), ref):
+        assert torch.equal(a.reshape(-1).view(torch.uint8), b.reshape(-1).view(torch.uint8))
+    sw = oracle.sweep(lat, taus, 0.15, rule=rule)
+    assert np.array_equal(done.cpu().numpy(), sw.done)
+    with pytest.raises(api.DropComputeError) as e:   # unknown objective: refused before the sweep is enqueued
+        api.dc_sweep_device(lat_d, taus_d, 0.15, rule, 0, step, done, sync, stats, base, k, tau, val, ws)
+    assert e.value.status == 7
+    with pytest.raises(api.DropComputeError) as e:   # workspace too small
+        api.dc_sweep_device(lat_d, taus_d, 0.15, rule, objective, step, done, sync, stats, base, k, tau, val, ws[:8])
+    assert e.value.status == 9
+    api.dc_device_status()
+
+
 def test_check_inputs(api):
     lat = torch.rand(4, 5, 6, device="cuda")
     taus = torch.tensor([0.1, 0.2, 0.2, INF], device="cuda")

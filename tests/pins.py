@@ -101,6 +101,32 @@ def pin_done_frac_erlang(lib, order="rows"):
         assert abs(st.stats[1, k] - want) <= 5 * se + 2e-6, (k, st.stats[1, k], want, se)
 
 
+def pin_start_rule_memoryless(lib, order="rows"):
+    """The start-before-tau rule (Limitations paragraph) on iid Exp(rate) micro-batches, one worker, more
+    micro-batches than can start before the largest threshold.  Micro-batch m starts iff the m-fold sum before it is
+    < tau, so the number started is 1 + (arrivals of a Poisson process of that rate before tau): mean 1 + rate*tau;
+    and the worker's time is the first arrival at or after tau, which by memorylessness is tau + Exp(rate):
+    mean tau + 1/rate, standard deviation 1/rate, always >= tau."""
+    rate, M, T = 20.0, 64, 40000
+    lat = W.iid_latencies("exp", T, 1, M, 17, rate=rate)
+    taus = np.array([0.05, 0.2, 0.55, 1.0], np.float32)   # rate*tau up to 20, far below M = 64 micro-batches
+    t_comm = 0.25
+    sw, st = _stats(lib, lat, taus, t_comm, rule=1, order=order)
+    assert (sw.step >= taus[None, :] + np.float32(t_comm) - 1e-6).all()
+    for k, tau in enumerate(taus.astype(np.float64)):
+        started = sw.done[:, k].astype(np.float64)
+        want_n = 1.0 + rate * tau
+        assert abs(started.mean() - want_n) <= 5 * math.sqrt(rate * tau / T) + 1e-9, (k, started.mean(), want_n)
+        assert abs(started.var(ddof=1) - rate * tau) <= 0.05 * rate * tau + 0.02, (k, started.var(ddof=1))
+        want_step = tau + 1.0 / rate + t_comm
+        assert abs(st.stats[0, k] - want_step) <= 5 * (1.0 / rate) / math.sqrt(T), (k, st.stats[0, k], want_step)
+        over = sw.step[:, k].astype(np.float64) - t_comm - tau
+        assert abs(over.std(ddof=1) - 1.0 / rate) <= 0.03 / rate, (k, over.std(ddof=1))
+    # the paper's rule on the same samples counts one fewer micro-batch whenever a threshold is crossed
+    sw0, _ = _stats(lib, lat, taus, t_comm, rule=0, order=order)
+    assert np.array_equal(sw.done, np.minimum(sw0.done + 1, M))
+
+
 # --- exhaustive enumeration in rational arithmetic -----------------------------
 
 def _enumerate_exact(values, N, M, taus, t_comm, rule):
@@ -393,7 +419,7 @@ def pin_closed_form(lib, order="rows"):
 ALL_PINS = (
     pin_exp_max_harmonic, pin_normal_max_quadrature, pin_done_frac_normal_eq5, pin_done_frac_erlang,
     pin_enumeration, pin_hand_example, pin_per_iteration_comm, pin_fp32_left_to_right, pin_m1_sort, pin_invariants, pin_argmax,
-    pin_literal_equals_rows, pin_independence_and_bailey, pin_closed_form,
+    pin_literal_equals_rows, pin_independence_and_bailey, pin_closed_form, pin_start_rule_memoryless,
 )
 # a quick subset that still kills every planted mistake (used by the mutation test)
 FAST_PINS = (pin_hand_example, pin_per_iteration_comm, pin_enumeration, pin_fp32_left_to_right, pin_m1_sort, pin_argmax,

@@ -11,12 +11,16 @@
 // A thread owns one worker's row of M latencies and adds them strictly left to right in fp32.
 // Because latencies are >= 0 the running sum P never decreases, and because the thresholds are
 // sorted, [P < tau_k] <=> k >= j(P) with j(P) = #{k : tau_k <= P}.  So each sample falls into one
-// bin j in [0,K] and done[t][k] is the prefix sum of the bin counts.  The thread keeps a cursor
-// (its current bin) that only moves forward and counts samples per bin by position, so the common
-// case costs one add and one compare per sample; bin counts go to per-warp integer histograms in
-// shared memory, which a per-trial epilogue sums, prefix-scans and writes out.  One block owns a
-// whole trial at a time (all N workers), so no global atomics and no scratch memory are needed
-// and every result is an integer sum or an exact maximum: bit-reproducible.
+// bin j in [0,K] and done[t][k] is the prefix sum of the bin counts.  j(P) comes from a lookup
+// table over equal cells of the threshold range, or for evenly spaced thresholds from one
+// multiply-add, and is then settled by comparing P with the thresholds themselves, so the bins
+// are exact.  Whole groups of samples that every lane of a warp still has below the first
+// threshold are counted in a register.  Bin counts go to integer histograms in shared memory,
+// which a dedicated warp sums, prefix-scans and writes out per trial while the other warps are
+// already on the next trial.  One block owns a whole trial at a time (all N workers), so no
+// global atomics and no scratch memory are needed and every result is an integer sum or an exact
+// maximum: bit-reproducible.  The start-before-tau variant of the rule (the paper's Limitations
+// paragraph) needs, besides the count, the largest finish time per bin and a prefix maximum.
 //
 // Data movement.  The kernel is bound by the one read of latencies[T][N][M] from HBM.  Tiles of
 // (rows x up to 128 bytes of each row) are brought into shared memory by the TMA unit
@@ -25,7 +29,9 @@
 // hardware swizzle (128/64/32-byte modes) makes "lane r reads 16 bytes of row r" free of
 // shared-memory bank conflicts.  Rows past N in a trial's last pass and columns past M are
 // out-of-bounds coordinates of the tensor map: they are zero-filled by the TMA unit and cost no
-// HBM traffic.
+// HBM traffic.  Rows whose length is not a multiple of 4 floats cannot be described by a tensor
+// map; they come in as plain bulk copies of whole rows (dc_sweep_flat) or, failing that, by
+// ordinary loads (dc_sweep_plain).
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <math.h>

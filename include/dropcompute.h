@@ -273,9 +273,9 @@ int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M,
  */
 int dc_device_status(uint32_t *flags_host);
 
-/* Which kernel dc_simulate_ex would use for a shape: 0 = tiled kernel (M a multiple of 4, 16-byte aligned
- * pointer), 2 = flat kernel (any other M up to 255, 16-byte aligned pointer), 1 = plain-load kernel (longer
- * such rows, or a pointer only 4-byte aligned), negative = -dc_status. */
+/* Which kernel dc_simulate_ex would use for a shape: 0 = tiled kernel (M a multiple of 4 and a 16-byte aligned
+ * pointer), 2 = flat kernel (any other case with M <= 255: other row lengths, or a pointer that is only 4-byte
+ * aligned), 1 = plain-load kernel (such cases with longer rows), negative = -dc_status. */
 int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K);
 
 /*

@@ -952,7 +952,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 
 // ------------------------------------------------------------------------------------------
 // Flat kernel: rows whose length is not a multiple of 4 (so a tensor map cannot describe them), up to
-// kFlatMaxM samples, base pointer 16-byte aligned.  Consecutive rows of a trial are one contiguous span of the
+// kFlatMaxM samples, and any row length up to that when the base pointer is only 4-byte aligned.  Consecutive rows of a trial are one contiguous span of the
 // tensor.  A tile is `rows` consecutive rows (a multiple of 32, at most 32 KB); the producer brings the 16-byte
 // aligned span that covers it into a stage with ONE plain bulk copy (cp.async.bulk, no tensor map) and thread r
 // of the tile's warps reads its row from float offset delta + r*M with 4-byte shared loads, 32 samples at a time.
@@ -961,8 +961,8 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 // same time.  The ring has a multiple of G stages, so a stage is only ever used by one group and each group sees
 // its own stages in order, like a ring of its own (for short rows G = 1: the tiled kernel's schedule).  Everything
 // after the loads is the tiled kernel's code (consume_chunk, epilogue warp, double-buffered histograms).  The
-// few floats past the last multiple of 4 of the whole tensor cannot be bulk-copied in bounds; the producer
-// moves them with ordinary loads.
+// few floats before the first and after the last 16-byte boundary inside the tensor cannot be bulk-copied in
+// bounds; the producer moves them with ordinary loads.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
 {
@@ -987,7 +987,12 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
     const int R = p.rows, Pt = p.passes, G = p.flat_groups, wpg = p.tile_warps;  // tiles per trial, groups, warps per group
     const unsigned long long NM = (unsigned long long)p.N * (unsigned long long)p.M;
     const unsigned long long total = (unsigned long long)p.T * NM;
-    const unsigned long long total4 = total & ~3ull;
+    // The base pointer is 4-byte aligned; float i of the tensor sits on a 16-byte boundary iff (i + a) % 4 == 0,
+    // where a = floats from the last such boundary to the base.  Bulk copies start and end on such floats INSIDE
+    // the tensor; the up to 3 floats before the first and after the last boundary go by ordinary loads.
+    const unsigned long long a = (unsigned long long)((reinterpret_cast<uintptr_t>(p.lat) & 15u) >> 2);
+    const unsigned long long first4 = (4ull - a) & 3ull;                    // first aligned float of the tensor
+    const unsigned long long last4 = total - ((total + a) & 3ull);          // one past the last aligned group
 
     // the producer thread sets up the barriers and fills the ring before the block builds its tables
     long long prod_t = blockIdx.x;
@@ -997,15 +1002,20 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
         const int nrows = min(R, p.N - row0);
         const unsigned long long b0 = (unsigned long long)prod_t * NM + (unsigned long long)row0 * p.M;
         const unsigned long long e0 = b0 + (unsigned long long)nrows * p.M;
-        const unsigned long long b4 = b0 & ~3ull;   // aligned start of the span
-        unsigned long long e4 = (e0 + 3ull) & ~3ull;  // aligned end, inside the tensor
-        if (e4 > total4) e4 = total4;
-        if (e4 < b4) e4 = b4;
+        // stage float s holds tensor float b0 - delta + s, delta = (b0 + a) % 4: the span's first float keeps
+        // its position inside its 16-byte group
+        const unsigned long long delta = (b0 + a) & 3ull;
+        const unsigned long long c0 = (b0 >= delta) ? b0 - delta : first4;   // aligned start, not before the tensor
+        unsigned long long c1 = e0 + ((4ull - ((e0 + a) & 3ull)) & 3ull);     // aligned end, not past the tensor
+        if (c1 > last4) c1 = last4;
+        if (c1 < c0) c1 = c0;
         float *dst = reinterpret_cast<float *>(stage0 + (size_t)st * p.stage_bytes);
-        for (unsigned long long i = e4; i < e0; ++i) dst[i - b4] = p.lat[i];  // at most 3 floats, last tile only
-        const uint32_t bytes = (uint32_t)((e4 - b4) * 4ull);
+        // floats of the span outside [c0, c1): at most 3 at the very start and 3 at the very end of the tensor
+        for (unsigned long long i = b0; i < e0 && i < c0; ++i) dst[i + delta - b0] = p.lat[i];
+        for (unsigned long long i = (c1 > b0 ? c1 : b0); i < e0; ++i) dst[i + delta - b0] = p.lat[i];
+        const uint32_t bytes = (uint32_t)((c1 - c0) * 4ull);
         mbar_arrive_expect_tx(&full[st], bytes);
-        if (bytes != 0u) bulk_load_1d(dst, p.lat + b4, bytes, &full[st]);
+        if (bytes != 0u) bulk_load_1d(dst + (c0 + delta - b0), p.lat + c0, bytes, &full[st]);
         if (++prod_q == Pt) {
             prod_q = 0;
             prod_t += gridDim.x;
@@ -1087,7 +1097,7 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
             const int row0 = rel * R;
             const bool valid = row0 + r < p.N;
             const unsigned long long b0 = (unsigned long long)t * NM + (unsigned long long)row0 * M;
-            const int delta = (int)(b0 & 3ull);
+            const int delta = (int)((b0 + a) & 3ull);
             float P = 0.0f;
             unsigned prev = off_zero;
             mbar_wait(&full[st], ph, kErrLoadNeverArrived);
@@ -1513,7 +1523,7 @@ int validate_simulate(const float *lat, int64_t T, int64_t N, int64_t M, const f
 bool tiled_ok(const float *lat, int64_t M) { return (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0); }
 bool flat_ok(const float *lat, int64_t M)
 {
-    return !tiled_ok(lat, M) && M <= kFlatMaxM && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0);
+    return !tiled_ok(lat, M) && M <= kFlatMaxM;  // any 4-byte aligned base (validate_simulate checks that)
 }
 
 template <int RULE, bool BATCH>

@@ -102,17 +102,27 @@ def test_edge_shapes_match_oracle(api, T, N, M, K):
     api.dc_device_status()
 
 
-def test_unaligned_base_takes_plain_kernel(api):
-    T, N, M, K = 4, 50, 16, 11
-    lat = W.iid_latencies("uniform", T, N, M, seed=5, lo=0.0, hi=0.1).numpy()
+@pytest.mark.parametrize("T,N,M,K", [(4, 50, 16, 11), (3, 300, 36, 40), (5, 7, 5, 9), (2, 600, 126, 64), (1, 1, 1, 3),
+                                      (6, 33, 255, 20), (3, 20, 300, 16), (2, 9, 1030, 8)])
+def test_base_pointer_only_4_byte_aligned(api, T, N, M, K):
+    """Latency tensors that start 1, 2 or 3 floats past a 16-byte boundary (views into a larger buffer): rows of up
+    to 255 samples take the flat kernel, whose bulk copies begin at the first and end at the last 16-byte boundary
+    inside the tensor with the few floats outside moved by ordinary loads; longer rows take the plain-load kernel.
+    Guard values around the view must not change anything."""
+    lat = W.iid_latencies("uniform", T, N, M, seed=5 + M, lo=0.0, hi=0.1).numpy()
     taus = grid_for(lat, K, 3)
-    buf = torch.zeros(T * N * M + 1, dtype=torch.float32, device="cuda")
-    view = buf[1:].view(T, N, M)
-    view.copy_(torch.from_numpy(lat))
-    assert api.dc_simulate_plan(view, K) == 1
-    assert api.dc_simulate_plan(torch.from_numpy(lat).cuda(), K) == 0
-    res = run_gpu(api, view, torch.from_numpy(taus).cuda(), 0.3)
-    compare_sweep(res, oracle.sweep(lat, taus, 0.3))
+    taus_d = torch.from_numpy(taus).cuda()
+    for rule in (0, 1):
+        ref = oracle.sweep(lat, taus, 0.3, rule=rule)
+        for shift in (1, 2, 3):
+            buf = torch.full((T * N * M + shift + 5,), float("nan"), dtype=torch.float32, device="cuda")
+            view = buf[shift:shift + T * N * M].view(T, N, M)
+            view.copy_(torch.from_numpy(lat))
+            assert api.dc_simulate_plan(view, K) == (2 if M <= 255 else 1)
+            res = run_gpu(api, view, taus_d, 0.3, rule=rule)
+            compare_sweep(res, ref, f"(shift {shift}, rule {rule})")
+    assert api.dc_simulate_plan(torch.from_numpy(lat).cuda(), K) == (0 if M % 4 == 0 else (2 if M <= 255 else 1))
+    api.dc_device_status()
 
 
 @pytest.mark.parametrize("rule", [0, 1])

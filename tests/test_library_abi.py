@@ -63,7 +63,8 @@ def test_argument_errors_need_no_gpu(lib):
     assert lib.dc_simulate_plan(A, 4, 8, 12, 3) == 0
     assert lib.dc_simulate_plan(A, 4, 8, 13, 3) == 2
     assert lib.dc_simulate_plan(A, 4, 8, 301, 3) == 1
-    assert lib.dc_simulate_plan(A + 4, 4, 8, 12, 3) == 1
+    assert lib.dc_simulate_plan(A + 4, 4, 8, 12, 3) == 2
+    assert lib.dc_simulate_plan(A + 4, 4, 8, 300, 3) == 1
     assert lib.dc_simulate_plan(A, 4, 8, 12, 5000) == -4
     # the later entry points
     assert lib.dc_simulate_tc(A, 1, 1, 1, A, 1, None, A, A, None, 0, None) == 1          # per-trial times missing

@@ -1739,8 +1739,6 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     }
 
     if (flat_ok(lat, M)) {
-        // rows per tile: 32 x the warps of a group, as many as fit a 32 KB stage (whole rows), at most 256 and no
-        // more than the trial has; groups: as many as eight consumer warps allow and the trial has tiles for
         // Warps per tile wt: the largest power of two whose tile (32 wt whole rows) stays within 32 KB, no more than
         // the trial has rows for.  Eight: one group, three stages (the tiled kernel's schedule).  Fewer: about six
         // consumer warps in G groups with one stage each (the groups overlap each other; measured best on rows of
@@ -1764,16 +1762,32 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         p.rows = wt * 32;
         p.tile_warps = wt;
         p.passes = (int)((N + p.rows - 1) / p.rows);
-        p.flat_groups = min(best_g, p.passes);
-        const int flat_threads = p.flat_groups * wt * 32;
         p.bw = (int)M;
         p.chunks = (int)((M + 31) / 32);
         p.pitch = (int)M * 4;
         p.stage_bytes = (int)((((size_t)p.rows * M * 4 + 32) + 1023) / 1024 * 1024);
+        // If the ring and the tables of a large grid do not fit a block's shared memory together, take fewer groups
+        // (a single group: three stages, then two).
+        const bool forced_split = g_tune_flat_tile_warps > 0 && g_tune_flat_groups > 0 && g_tune_flat_depth > 0;
+        int groups = min(best_g, p.passes), depth = best_d;
+        if (!forced_split && groups == 1) depth = 3;
         size_t smem = 0;
-        const int lrc0 = choose_block_layout(p, flat_threads, K, rule, di, &smem, -(p.flat_groups * best_d));
-        if (lrc0 != DC_OK) return lrc0;
-        if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
+        int flat_threads = 0;
+        for (;;) {
+            p.flat_groups = groups;
+            flat_threads = groups * wt * 32;
+            const int lrc0 = choose_block_layout(p, flat_threads, K, rule, di, &smem, -(groups * depth));
+            if (lrc0 == DC_OK && smem <= (size_t)di.max_smem_optin) break;
+            if (forced_split) return DC_ERR_RANGE;
+            if (groups > 1) {
+                --groups;
+                depth = groups == 1 ? 3 : 1;
+            } else if (depth > 2) {
+                depth = 2;
+            } else {
+                return DC_ERR_RANGE;
+            }
+        }
         const int block = flat_threads + 64;
         int lrc;
         if (rule == DC_RULE_FINISH_BEFORE_TAU)

@@ -584,7 +584,8 @@ def test_flat_kernel_shapes(api):
     runs under different splits of the consumer warps (warps per tile, groups working on different tiles at
     once, ring stages per group), including more groups than a trial has tiles and trials that end mid-ring."""
     cases = [(7, 3, 5, 9), (5, 1, 1, 3), (3, 257, 30, 64), (6, 513, 6, 33), (4, 100, 255, 40), (9, 64, 33, 100),
-             (11, 37, 10, 16), (2, 2048, 126, 256), (64, 200, 14, 64), (13, 300, 65, 48), (5, 1000, 127, 32)]
+             (11, 37, 10, 16), (2, 2048, 126, 256), (64, 200, 14, 64), (13, 300, 65, 48), (5, 1000, 127, 32),
+             (2, 200, 255, 4096), (2, 300, 126, 3000)]   # the last two: ring and tables compete for shared memory
     splits = [(0, 0, 0), (1, 8, 1), (1, 4, 2), (2, 4, 1), (2, 2, 2), (1, 3, 2), (4, 2, 1), (1, 5, 1), (8, 1, 2)]
     try:
         for (T, N, M, K) in cases:

@@ -152,43 +152,6 @@ __device__ __forceinline__ void named_barrier(int id, int threads)
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-// ------------------------------------------------------------------------------------------
-// One worker's walk along its row (Algorithm 2's inner loop for all tau at once).
-// ------------------------------------------------------------------------------------------
-struct RowWalk {
-    float P;      // running compute time T_{i,n} after the samples seen so far
-    float tcur;   // tau_s[cur]; +inf once cur == K
-    int cur;      // number of thresholds <= the last P that moved the cursor (the current bin)
-    int mflush;   // index of the first sample not yet added to the histogram
-
-    __device__ __forceinline__ void start(const float *tau_s)
-    {
-        P = 0.0f;
-        cur = 0;
-        tcur = tau_s[0];
-        mflush = 0;
-    }
-    // sample number m (0-based) with latency x
-    __device__ __forceinline__ void step(float x, int m, const float *tau_s, int *hist, int K)
-    {
-        P = __fadd_rn(P, x);
-        if (P >= tcur) {  // leaves the current bin: samples mflush..m-1 were in it
-            const int c = m - mflush;
-            if (c > 0) atomicAdd(&hist[cur], c);
-            while (cur < K && P >= tcur) {
-                ++cur;
-                tcur = tau_s[cur];  // tau_s[K] = +inf
-            }
-            mflush = m;
-        }
-    }
-    __device__ __forceinline__ void finish(int M, int *hist)
-    {
-        const int c = M - mflush;
-        if (c > 0) atomicAdd(&hist[cur], c);
-    }
-};
-
 // Start-before-tau rule.  Micro-batch m is run iff the time before it, P_{m-1}, is < tau_k, and a worker's time
 // W_n(k) is the finish time of the last micro-batch it ran (0 if it ran none).  Running sums never decrease, so
 // W_n(k) is also the LARGEST finish time among the micro-batches the worker ran, and the step's compute time is
@@ -202,25 +165,6 @@ __device__ __forceinline__ void raise_max(float *slot, float V)
 {
     atomicMax(reinterpret_cast<int *>(slot), __float_as_int(V));
 }
-
-// Start-before-tau rule, one worker's row with a forward cursor (plain-load kernel).
-struct RowWalkStart {
-    float P;
-    int cur;  // #{k : tau_k <= P}
-    __device__ __forceinline__ void start(const float *tau_s, int K)
-    {
-        P = 0.0f;
-        cur = 0;
-        while (cur < K && 0.0f >= tau_s[cur]) ++cur;
-    }
-    __device__ __forceinline__ void step(float x, const float *tau_s, int *hist, float *fmax, int K)
-    {
-        atomicAdd(&hist[cur], 1);  // P_{m-1} is in bin cur
-        P = __fadd_rn(P, x);
-        raise_max(&fmax[cur], P);
-        while (cur < K && P >= tau_s[cur]) ++cur;
-    }
-};
 
 __device__ __forceinline__ float warp_max(float v)
 {
@@ -476,7 +420,7 @@ __device__ __forceinline__ void bin_sample(float P, float lo, float scale, unsig
     atomicAdd(reinterpret_cast<int *>(hist_b + bin_offset<ONE>(P, lo, scale, C, lut, tau_b, K4)), 1);
 }
 // Start-before-tau rule: micro-batch m with finish time P.  The time before it lies in bin `prev` (byte
-// offset): that bin's count goes up by one and its finish-time maximum is raised to P (see RowWalkStart);
+// offset): that bin's count goes up by one and its finish-time maximum is raised to P (see raise_max);
 // fmax_delta is the byte distance from a histogram entry to the maximum of the same bin and copy.
 // Bin 0 is kept in the thread's registers (cnt0, fin0) and added once per trial: when a straggler lane sends its
 // warp through this path the other lanes are typically all still in bin 0 and would pile up on one entry.  (The
@@ -1131,38 +1075,77 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
 }
 
 // ------------------------------------------------------------------------------------------
-// Plain-load kernel for shapes the tensor map cannot describe (M not a multiple of 4, or a base
-// pointer that is only 4-byte aligned).  Same walk and epilogue; each thread reads its row
-// straight from global memory.
+// Plain-load kernel for what neither staged kernel takes (rows longer than kFlatMaxM whose length is not a
+// multiple of 4 or whose base is only 4-byte aligned).  No TMA: for each chunk of 32 columns a warp loads the
+// 32-float pieces of its 32 rows with ordinary coalesced loads (lane = column), parks them in a 32 x 33 tile of
+// its own in shared memory and each lane then takes its row's 32 samples from there (lane = row).  The walk is
+// the staged kernels' (consume_chunk); the epilogue is done by the whole block per trial.
 // ------------------------------------------------------------------------------------------
+constexpr int kPlainTileFloats = 32 * 33;
+
+template <int RULE>
 __global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepParams p)
 {
-    extern __shared__ unsigned char smem_raw[];
-    const SmemTail s = carve_tail(smem_raw, p);
-    const int tid = threadIdx.x, warp = tid >> 5, nthr = blockDim.x;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
+    float *tile = reinterpret_cast<float *>(smem_raw) + warp * kPlainTileFloats;
+    const SmemTail s = carve_tail(smem_raw + (size_t)(nthr >> 5) * kPlainTileFloats * sizeof(float), p);
     load_thresholds(p, s, tid, nthr);
     __syncthreads();
+    build_lut(p, s, tid, nthr);
+
+    const int K = p.K, M = p.M;
+    BinCtx ctx;
+    ctx.lut_lo = __int_as_float(s.meta[1]);
+    ctx.lut_scale = __int_as_float(s.meta[2]);
+    ctx.C = (unsigned)p.lut_cells;
+    ctx.lut = s.lut;
+    ctx.tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
+    ctx.K4 = 4u * (unsigned)K;
+    ctx.one = s.meta[0] != 0;
+    ctx.dscale = __int_as_float(s.meta[4]);
+    ctx.dshift = __int_as_float(s.meta[5]);
+    ctx.K = (unsigned)K;
+    ctx.tau_first = s.tau_s[0];
+    ctx.tau_last = s.tau_s[K - 1];
+    ctx.arrive_one = 1u;
+    unsigned off_zero = 0;
+    if (RULE == 1) off_zero = bin_offset<false>(0.0f, ctx.lut_lo, ctx.lut_scale, ctx.C, ctx.lut, ctx.tau_b, ctx.K4);
     int *myhist = s.hist + (warp & (p.hist_copies - 1)) * p.hist_stride;
-    float *myfmax = s.fmax + (warp & (p.hist_copies - 1)) * p.hist_stride;  // rule 1 only
+    unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
+    const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));
+
     for (long long t = blockIdx.x; t < p.T; t += gridDim.x) {
-        float rowmax = 0.0f;
+        float rowmax = 0.0f, fin0 = 0.0f;
+        int cnt0 = 0;
         for (int pass = 0; pass < p.passes; ++pass) {
-            const int n = pass * p.rows + tid;
-            if (n < p.N) {
-                const float *row = p.lat + ((size_t)t * p.N + n) * p.M;
-                if (p.rule == DC_RULE_FINISH_BEFORE_TAU) {
-                    RowWalk w;
-                    w.start(s.tau_s);
-                    for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), m, s.tau_s, myhist, p.K);
-                    w.finish(p.M, myhist);
-                    rowmax = fmaxf(rowmax, w.P);
-                } else {
-                    RowWalkStart w;
-                    w.start(s.tau_s, p.K);
-                    for (int m = 0; m < p.M; ++m) w.step(__ldg(row + m), s.tau_s, myhist, myfmax, p.K);
-                    rowmax = fmaxf(rowmax, w.P);
+            const int n0 = pass * p.rows + warp * 32;   // this warp's first row in the trial
+            const bool valid = n0 + lane < p.N;
+            const int nrows = min(32, p.N - n0);         // rows of this warp that exist (may be <= 0)
+            const float *src = p.lat + ((size_t)t * p.N + (size_t)max(n0, 0)) * M;
+            float P = 0.0f;
+            unsigned prev = off_zero;
+            for (int m0 = 0; m0 < M; m0 += 32) {
+                const int ns = min(32, M - m0);
+                // lane = column: row rr's piece is one coalesced read of up to 128 bytes
+#pragma unroll 8
+                for (int rr = 0; rr < 32; ++rr) {
+                    float x = 0.0f;
+                    if (rr < nrows && lane < ns) x = __ldg(src + (size_t)rr * M + m0 + lane);
+                    tile[rr * 33 + lane] = x;
                 }
+                __syncwarp();
+                float4 v[8];  // lane = row
+#pragma unroll
+                for (int e = 0; e < 32; ++e) sample_ref(v, e) = tile[lane * 33 + e];
+                __syncwarp();
+                consume_chunk<8, RULE, false, false>(v, ns, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, nullptr);
             }
+            if (valid) rowmax = fmaxf(rowmax, P);
+        }
+        if (cnt0 > 0) {
+            atomicAdd(myhist, cnt0);
+            if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
         }
         trial_epilogue(p, t, rowmax, tid, nthr, kConsumerBarrier, s.tau_s, s.hist, s.smax, s.wtot, s.fmax, s.wmx);
     }
@@ -1801,15 +1784,19 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     // plain-load kernel
     p.rows = row_threads;  // one row per thread per pass
     p.passes = (int)((N + p.rows - 1) / p.rows);
-    const size_t smem = tail_bytes(K, p.hist_copies, p.hist_stride, 0, p.aux_copies);
+    p.hist_stride = (K + 2 + 3) & ~3;
+    p.hist_copies = floor_pow2(min(row_threads / 32, max(1, kHistBudgetBytes / (int)(sizeof(int) * p.hist_stride))));
+    p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? p.hist_copies : 0;
+    p.lut_cells = min(kLutCellsMax, 4 * K);
+    const size_t smem = (size_t)(row_threads / 32) * kPlainTileFloats * sizeof(float) +
+                        tail_bytes(K, p.hist_copies, p.hist_stride, p.lut_cells, p.aux_copies);
     if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
-    if (cudaFuncSetAttribute(dc_sweep_plain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return DC_ERR_CUDA;
+    auto kernel = rule == DC_RULE_FINISH_BEFORE_TAU ? dc_sweep_plain<0> : dc_sweep_plain<1>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, dc_sweep_plain, p.rows, smem) != cudaSuccess || occ < 1)
-        return DC_ERR_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, p.rows, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
     const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
-    dc_sweep_plain<<<(unsigned)grid, p.rows, smem, stream>>>(p);
+    kernel<<<(unsigned)grid, p.rows, smem, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     g_last_simulate_launches = 1;
     return DC_OK;

@@ -614,6 +614,23 @@ def test_flat_kernel_shapes(api):
     api.dc_device_status()
 
 
+@pytest.mark.parametrize("T,N,M,K", [(3, 600, 257, 64), (2, 300, 301, 17), (5, 33, 514, 256), (2, 1, 999, 5), (40, 7, 258, 1)])
+def test_plain_kernel_shapes(api, T, N, M, K):
+    """Rows longer than 255 samples whose length is not a multiple of 4 (plain-load kernel: a warp stages 32 x 32
+    pieces of its rows through a tile of its own): several passes per trial, ragged last warp and last chunk, a
+    single worker, both rules, dyadic latencies so that running sums land ON thresholds."""
+    lat = W.iid_latencies("dyadic", T, N, M, seed=300 + M, hi=6).numpy()
+    taus = grid_for(lat, K, seed=K + 2)
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    assert api.dc_simulate_plan(lat_d, K) == 1
+    for rule in (0, 1):
+        ref = oracle.sweep(lat, taus, 0.125, rule=rule)
+        res = run_gpu(api, lat_d, taus_d, 0.125, rule=rule)
+        compare_sweep(res, ref, f"(rule {rule})")
+        compare_stats(res, ref, N, M)
+    api.dc_device_status()
+
+
 @pytest.mark.parametrize("T,N,M,K", [(3, 100000, 4, 40), (200000, 8, 4, 16), (2, 40, 4096, 64), (2, 70, 1030, 33),
                                       (1, 300000, 1, 8), (50000, 1, 32, 5)])
 def test_extreme_aspect_ratios(api, T, N, M, K):

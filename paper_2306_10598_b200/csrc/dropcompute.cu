@@ -915,7 +915,8 @@ __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_
                  : "memory");
 }
 
-template <int RULE, bool BATCH>
+// NQ = 16-byte quads of a row per chunk held in registers: 8 (32 samples), fewer for rows of at most 16 samples.
+template <int RULE, bool BATCH, int NQ>
 __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const SweepParams p)
 {
     extern __shared__ unsigned char smem_raw[];
@@ -1053,13 +1054,14 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
                 st -= S;
                 ph ^= 1u;
             }
-            for (int m0 = 0; m0 < M; m0 += 32) {
-                const int ns = min(32, M - m0);
-                float4 v[8];
+            constexpr int CW = 4 * NQ;  // samples per chunk
+            for (int m0 = 0; m0 < M; m0 += CW) {
+                const int ns = min(CW, M - m0);
+                float4 v[NQ];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) sample_ref(v, e) = (e < ns) ? row[m0 + e] : 0.0f;
-                consume_chunk<8, RULE, BATCH, false>(v, ns, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0,
-                                                     (m0 + 32 >= M) ? empty_bar : nullptr);
+                for (int e = 0; e < CW; ++e) sample_ref(v, e) = (e < ns) ? row[m0 + e] : 0.0f;
+                consume_chunk<NQ, RULE, BATCH, false>(v, ns, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0,
+                                                      (m0 + CW >= M) ? empty_bar : nullptr);
             }
             if (valid) rowmax = fmaxf(rowmax, P);
         }
@@ -1509,16 +1511,26 @@ bool flat_ok(const float *lat, int64_t M)
     return !tiled_ok(lat, M) && M <= kFlatMaxM;  // any 4-byte aligned base (validate_simulate checks that)
 }
 
-template <int RULE, bool BATCH>
-int launch_flat(const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di, cudaStream_t stream)
+template <int RULE, bool BATCH, int NQ>
+int launch_flat_q(const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di, cudaStream_t stream)
 {
-    auto kernel = dc_sweep_flat<RULE, BATCH>;
+    auto kernel = dc_sweep_flat<RULE, BATCH, NQ>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
     const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
     kernel<<<(unsigned)grid, block, smem, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+template <int RULE, bool BATCH>
+int launch_flat(const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di, cudaStream_t stream)
+{
+    // rows of at most 16 samples are one short chunk
+    if (p.M <= 4) return launch_flat_q<RULE, BATCH, 1>(p, block, smem, T, di, stream);
+    if (p.M <= 8) return launch_flat_q<RULE, BATCH, 2>(p, block, smem, T, di, stream);
+    if (p.M <= 16) return launch_flat_q<RULE, BATCH, 4>(p, block, smem, T, di, stream);
+    return launch_flat_q<RULE, BATCH, 8>(p, block, smem, T, di, stream);
 }
 
 template <int NQ, int RULE, bool BATCH>

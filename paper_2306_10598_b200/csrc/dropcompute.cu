@@ -455,6 +455,31 @@ struct BinCtx {
     uint32_t arrive_one;      // always 1, opaque to the compiler (ties a stage release to a warp vote)
 };
 
+// The binning context of a block, from the tables build_lut() left in shared memory.
+__device__ __forceinline__ BinCtx make_bin_ctx(const SweepParams &p, const SmemTail &s)
+{
+    BinCtx c;
+    c.lut_lo = __int_as_float(s.meta[1]);
+    c.lut_scale = __int_as_float(s.meta[2]);
+    c.C = (unsigned)p.lut_cells;
+    c.lut = s.lut;
+    c.tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
+    c.K4 = 4u * (unsigned)p.K;
+    c.one = s.meta[0] != 0;
+    c.dscale = __int_as_float(s.meta[4]);
+    c.dshift = __int_as_float(s.meta[5]);
+    c.K = (unsigned)p.K;
+    c.tau_first = s.tau_s[0];
+    c.tau_last = s.tau_s[p.K - 1];
+    c.arrive_one = (uint32_t)p.one;
+    return c;
+}
+// Start-before-tau rule: the bin (byte offset) of a running time of 0, where every row starts.
+__device__ __forceinline__ unsigned bin_of_zero(const BinCtx &c)
+{
+    return bin_offset<false>(0.0f, c.lut_lo, c.lut_scale, c.C, c.lut, c.tau_b, c.K4);
+}
+
 template <int NQ>
 __device__ __forceinline__ float &sample_ref(float4 (&v)[NQ], int e)
 {
@@ -862,32 +887,12 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     }
 
     // ---------------- consumers
-    const int K = p.K;
     int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
     // rule 1: byte distance from a histogram entry to the finish-time maximum of the same buffer, copy and bin
     const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));
-    const unsigned char *tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
-    const unsigned K4 = 4u * (unsigned)K;
-    const bool one = s.meta[0] != 0;
-    const float lut_lo = __int_as_float(s.meta[1]), lut_scale = __int_as_float(s.meta[2]);
-    const unsigned C = (unsigned)p.lut_cells;
-    BinCtx ctx;
-    ctx.lut_lo = lut_lo;
-    ctx.lut_scale = lut_scale;
-    ctx.C = C;
-    ctx.lut = s.lut;
-    ctx.tau_b = tau_b;
-    ctx.K4 = K4;
-    ctx.one = one;
-    ctx.dscale = __int_as_float(s.meta[4]);
-    ctx.dshift = __int_as_float(s.meta[5]);
-    ctx.K = (unsigned)K;
-    ctx.tau_first = s.tau_s[0];
-    ctx.tau_last = s.tau_s[K - 1];
-    ctx.arrive_one = (uint32_t)p.one;
-    // rule 1 only: the bin of a running time of 0
-    unsigned off_zero = 0;
-    if (RULE == 1) off_zero = bin_offset<false>(0.0f, lut_lo, lut_scale, C, s.lut, tau_b, K4);
+    const BinCtx ctx = make_bin_ctx(p, s);
+    const bool one = ctx.one;
+    const unsigned off_zero = RULE == 1 ? bin_of_zero(ctx) : 0u;  // rule 1 only
     if (s.meta[3] != 0 && one && p.direct_bins != 0)
         tiled_trials<NQ, RULE, BATCH, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, myhist0, fmax_delta, off_zero);
     else
@@ -1002,26 +1007,12 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
 
     // ---------------- consumers
     const int bar_threads = ncw * 32 + 32;
-    const int K = p.K, M = p.M;
+    const int M = p.M;
     const int hist_buf_ints = p.hist_copies * p.hist_stride;
     int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
     const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));
-    BinCtx ctx;
-    ctx.lut_lo = __int_as_float(s.meta[1]);
-    ctx.lut_scale = __int_as_float(s.meta[2]);
-    ctx.C = (unsigned)p.lut_cells;
-    ctx.lut = s.lut;
-    ctx.tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
-    ctx.K4 = 4u * (unsigned)K;
-    ctx.one = s.meta[0] != 0;
-    ctx.dscale = __int_as_float(s.meta[4]);
-    ctx.dshift = __int_as_float(s.meta[5]);
-    ctx.K = (unsigned)K;
-    ctx.tau_first = s.tau_s[0];
-    ctx.tau_last = s.tau_s[K - 1];
-    ctx.arrive_one = (uint32_t)p.one;
-    unsigned off_zero = 0;
-    if (RULE == 1) off_zero = bin_offset<false>(0.0f, ctx.lut_lo, ctx.lut_scale, ctx.C, ctx.lut, ctx.tau_b, ctx.K4);
+    const BinCtx ctx = make_bin_ctx(p, s);
+    const unsigned off_zero = RULE == 1 ? bin_of_zero(ctx) : 0u;
     const int grp = warp / wpg;
     const int r = (warp - grp * wpg) * 32 + lane;  // this thread's row inside its group's tiles (< R)
     // The block's tiles are numbered i = 0, 1, ... in the producer's order (trial, then tile inside the trial);
@@ -1096,23 +1087,9 @@ __global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepPar
     __syncthreads();
     build_lut(p, s, tid, nthr);
 
-    const int K = p.K, M = p.M;
-    BinCtx ctx;
-    ctx.lut_lo = __int_as_float(s.meta[1]);
-    ctx.lut_scale = __int_as_float(s.meta[2]);
-    ctx.C = (unsigned)p.lut_cells;
-    ctx.lut = s.lut;
-    ctx.tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
-    ctx.K4 = 4u * (unsigned)K;
-    ctx.one = s.meta[0] != 0;
-    ctx.dscale = __int_as_float(s.meta[4]);
-    ctx.dshift = __int_as_float(s.meta[5]);
-    ctx.K = (unsigned)K;
-    ctx.tau_first = s.tau_s[0];
-    ctx.tau_last = s.tau_s[K - 1];
-    ctx.arrive_one = 1u;
-    unsigned off_zero = 0;
-    if (RULE == 1) off_zero = bin_offset<false>(0.0f, ctx.lut_lo, ctx.lut_scale, ctx.C, ctx.lut, ctx.tau_b, ctx.K4);
+    const int M = p.M;
+    const BinCtx ctx = make_bin_ctx(p, s);
+    const unsigned off_zero = RULE == 1 ? bin_of_zero(ctx) : 0u;
     int *myhist = s.hist + (warp & (p.hist_copies - 1)) * p.hist_stride;
     unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
     const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));

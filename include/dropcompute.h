@@ -201,6 +201,9 @@ int dc_argmax_tau(const double *stats, const float *taus, int32_t K, int32_t obj
  * enqueues dc_simulate_ex, dc_reduce_trials and dc_argmax_tau on `stream`, in that order, with the arguments
  * documented there (out_sync is required here).  Host-visible errors of any of the three are reported before
  * anything is enqueued.  workspace as for dc_reduce_trials (dc_reduce_workspace_bytes(T, K) bytes).
+ * Like the three calls it stands for, it only enqueues kernels: once it has been called normally on a device it
+ * can be recorded in a CUDA stream capture and replayed, which pays off on inputs small enough to be bound by
+ * launch latency.
  */
 int dc_sweep_device(const float *latencies, int64_t T, int64_t N, int64_t M,
                     const float *taus, int32_t K, float t_comm, int32_t rule, int32_t objective,

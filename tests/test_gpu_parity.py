@@ -227,6 +227,49 @@ def test_sweep_device_equals_the_three_calls(api, rule, objective):
     api.dc_device_status()
 
 
+@pytest.mark.parametrize("T,N,M,K,rule", [(64, 8, 4, 16, 0), (40, 200, 32, 64, 1), (9, 300, 30, 33, 0), (3, 70, 301, 20, 1)])
+def test_device_path_in_a_cuda_graph(api, T, N, M, K, rule):
+    """The device-resident path neither allocates nor synchronises, so a stream capture can record it (after one
+    ordinary call, which sets the kernels' attributes) and a replay must reproduce every output bit: tiled, flat
+    and plain-load kernels."""
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=55 + M, shift=0.01, mean=0.02).numpy()
+    taus = grid_for(lat, K, 8)
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    step = torch.empty((T, K), dtype=torch.float32, device="cuda")
+    done = torch.empty((T, K), dtype=torch.int32, device="cuda")
+    sync = torch.empty((T,), dtype=torch.float32, device="cuda")
+    stats = torch.empty((api.NSTATS, K), dtype=torch.float64, device="cuda")
+    base = torch.empty((2,), dtype=torch.float64, device="cuda")
+    k = torch.empty((), dtype=torch.int32, device="cuda")
+    tau = torch.empty((), dtype=torch.float32, device="cuda")
+    val = torch.empty((), dtype=torch.float64, device="cuda")
+    ws = torch.empty((api.dc_reduce_workspace_bytes(T, K),), dtype=torch.uint8, device="cuda")
+    outs = (step, done, sync, stats, base, k, tau, val)
+
+    def call():
+        api.dc_sweep_device(lat_d, taus_d, 0.2, rule, 4, step, done, sync, stats, base, k, tau, val, ws)
+
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        call()
+        torch.cuda.synchronize()
+        want = [o.clone() for o in outs]
+        with torch.cuda.graph(graph, stream=side):
+            call()
+    for _ in range(2):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for o, w_ in zip(outs, want):
+            assert torch.equal(o.reshape(-1).view(torch.uint8), w_.reshape(-1).view(torch.uint8))
+    ref = oracle.sweep(lat, taus, 0.2, rule=rule)
+    assert np.array_equal(done.cpu().numpy(), ref.done)
+    assert np.array_equal(step.cpu().numpy().view(np.uint32), ref.step.view(np.uint32))
+    api.dc_device_status()
+
+
 def test_check_inputs(api):
     lat = torch.rand(4, 5, 6, device="cuda")
     taus = torch.tensor([0.1, 0.2, 0.2, INF], device="cuda")

@@ -1139,7 +1139,7 @@ __global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepPar
 // ------------------------------------------------------------------------------------------
 constexpr int kRedWarps = 8;
 
-__global__ void __launch_bounds__(kRedWarps * 32)
+__global__ void __launch_bounds__(kRedWarps * 32, 4)
 dc_reduce_partial(const float *__restrict__ step, const int32_t *__restrict__ done, const float *__restrict__ sync,
                   long long T, int K, double NM, int chunks, long long rows_per_chunk, double *ws)
 {
@@ -1153,6 +1153,7 @@ dc_reduce_partial(const float *__restrict__ step, const int32_t *__restrict__ do
     double s_step = 0.0, s_ratio = 0.0, s_S = 0.0;
     long long s_done = 0;
     const double nan = __longlong_as_double(0x7ff8000000000000LL);
+    const double inv_NM = 1.0 / NM;
     if (k < K) {
         // four rows in flight per thread (the loads do not depend on each other); summed in row order
         for (long long t = t0 + warp; t < t1; t += 4 * kRedWarps) {
@@ -1174,8 +1175,9 @@ dc_reduce_partial(const float *__restrict__ step, const int32_t *__restrict__ do
                     const double sy = sync ? (double)sy_f[u] : nan;
                     s_step += st;
                     s_done += dn_i[u];
-                    s_ratio += dn / st;
-                    s_S += (sy / st) * (dn / NM);
+                    const double r = 1.0 / st;  // one division per element; the quotients below are products with it
+                    s_ratio += dn * r;
+                    s_S += (sy * r) * (dn * inv_NM);
                 }
             }
         }

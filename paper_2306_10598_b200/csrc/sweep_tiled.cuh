@@ -1,0 +1,296 @@
+// The tiled sweep kernel (TMA tensor map) and the epilogue warp it shares with the flat kernel.
+// Part of dropcompute.cu (one translation unit, included there in this order); everything is internal.
+#pragma once
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// Tiled kernel: TMA-staged rows, persistent over trials.  Warp roles inside a block:
+//   warps 0 .. ncw-1   consumers: thread r owns row (pass*rows + r) of the current trial
+//   warp  ncw          producer: one thread streams the block's tiles through the ring of stages
+//   warp  ncw+1        epilogue: turns a finished trial's histograms into out_done / out_step / out_sync
+// The histograms (and the per-warp maxima) are double-buffered: consumers fill buffer j&1 for their j-th
+// trial and go straight on to the next trial while the epilogue warp sums, scans, writes and clears the
+// buffer.  Named barriers hand the buffers over: kBarReady+b (consumers arrive, epilogue waits) and
+// kBarFree+b (epilogue arrives, consumers wait before reusing the buffer two trials later).
+// NQ = 16-byte quads of a row per chunk held in registers (box width = 4*NQ floats at most).
+// A consumer thread adds its row's samples in order; per group of eight, if every lane of the warp is
+// still below the first threshold the samples are bin 0 (one register add); if every lane is at or
+// above the last threshold they are in the bin nobody reads; otherwise each running sum is binned
+// through the lookup table.
+// ------------------------------------------------------------------------------------------
+constexpr int kBarReady = 2;  // +0, +1
+constexpr int kBarFree = 4;   // +0, +1
+
+// Barrier numbers are compile-time immediates (a run-time number would make the compiler reserve all 16
+// hardware barriers for every block); b selects between the two buffers' barriers.
+template <int ID>
+__device__ __forceinline__ void bar_sync_imm(int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"n"(ID), "r"(threads) : "memory");
+}
+template <int ID>
+__device__ __forceinline__ void bar_arrive_imm(int threads)
+{
+    asm volatile("bar.arrive %0, %1;" ::"n"(ID), "r"(threads) : "memory");
+}
+template <int BASE>
+__device__ __forceinline__ void buffer_barrier_sync(int b, int threads)
+{
+    if (b == 0) bar_sync_imm<BASE>(threads);
+    else bar_sync_imm<BASE + 1>(threads);
+}
+template <int BASE>
+__device__ __forceinline__ void buffer_barrier_arrive(int b, int threads)
+{
+    if (b == 0) bar_arrive_imm<BASE>(threads);
+    else bar_arrive_imm<BASE + 1>(threads);
+}
+
+// The epilogue warp's loop (all 32 lanes).  Bins are taken 32 at a time: lane l sums bin k0+l over the
+// copies (and clears it), a warp scan gives the prefix, a carry links the blocks of 32.
+template <int RULE>
+__device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTail &s, int lane, int ncw)
+{
+    const int K = p.K, H = p.hist_copies, HS = p.hist_stride;
+    const int bar_threads = ncw * 32 + 32;
+    int j = 0;
+    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
+        const int b = j & 1;
+        buffer_barrier_sync<kBarReady>(b, bar_threads);  // every consumer has finished trial t
+        int *hist = s.hist + b * H * HS;
+        float *fmax = s.fmax + b * H * HS;  // rule 1 only
+        const float Tmax = warp_max(lane < ncw ? s.smax[32 * b + lane] : 0.0f);
+        const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
+        float *step_row = p.out_step + t * K;
+        int32_t *done_row = p.out_done + t * K;
+        int carry = 0;
+        float fm_carry = 0.0f;
+        // Four consecutive bins per lane, 128 bins per step, with 16-byte accesses throughout (when the shapes and
+        // pointers allow): a quarter of the scans and well under half the instructions of the scalar loop below.
+        for (int k0 = 0; p.epi_vec && k0 < K; k0 += 128) {
+            const int k = k0 + 4 * lane;
+            const bool in = k < K;  // K is a multiple of 4: a lane's four bins are all inside or all outside
+            int4 h = make_int4(0, 0, 0, 0);
+            float4 fm = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            if (in) {
+#pragma unroll 2
+                for (int c = 0; c < H; ++c) {
+                    int4 *hp = reinterpret_cast<int4 *>(hist + c * HS + k);
+                    const int4 v = *hp;
+                    *hp = make_int4(0, 0, 0, 0);
+                    h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
+                    if (RULE == 1) {
+                        float4 *fp = reinterpret_cast<float4 *>(fmax + c * HS + k);
+                        const float4 f = *fp;
+                        *fp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                        fm.x = fmaxf(fm.x, f.x); fm.y = fmaxf(fm.y, f.y); fm.z = fmaxf(fm.z, f.z); fm.w = fmaxf(fm.w, f.w);
+                    }
+                }
+            }
+            h.y += h.x; h.z += h.y; h.w += h.z;  // inclusive inside the lane
+            const int incl = warp_inclusive_scan(h.w, lane);
+            const int base = carry + incl - h.w;  // everything before this lane's bins
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+            float4 st;
+            if (RULE == 0) {
+                const float4 tq = in ? *reinterpret_cast<const float4 *>(s.tau_s + k) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                st.x = fminf(tq.x, Tmax); st.y = fminf(tq.y, Tmax); st.z = fminf(tq.z, Tmax); st.w = fminf(tq.w, Tmax);
+            } else {
+                // max_n W_n(k) = max_{j <= k} fmax[j]
+                fm.y = fmaxf(fm.y, fm.x); fm.z = fmaxf(fm.z, fm.y); fm.w = fmaxf(fm.w, fm.z);
+                const float fincl = warp_inclusive_max_scan(fm.w, lane);
+                float before = __shfl_up_sync(0xffffffffu, fincl, 1);
+                before = fmaxf(fm_carry, lane > 0 ? before : 0.0f);
+                fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fincl, 31));
+                st.x = fmaxf(before, fm.x); st.y = fmaxf(before, fm.y); st.z = fmaxf(before, fm.z); st.w = fmaxf(before, fm.w);
+            }
+            if (in) {
+                *reinterpret_cast<int4 *>(done_row + k) = make_int4(base + h.x, base + h.y, base + h.z, base + h.w);
+                *reinterpret_cast<float4 *>(step_row + k) =
+                    make_float4(__fadd_rn(st.x, t_comm), __fadd_rn(st.y, t_comm), __fadd_rn(st.z, t_comm), __fadd_rn(st.w, t_comm));
+            }
+        }
+        // Otherwise: 32 bins at a time, lane l sums bin k0+l over the copies (and clears it), a warp scan gives the
+        // prefix, a carry links the blocks of 32.
+        for (int k0 = p.epi_vec ? K : 0; k0 < K; k0 += 32) {
+            const int k = k0 + lane;
+            int h = 0;
+            float fm = 0.0f;
+            if (k < K) {
+                for (int c = 0; c < H; ++c) {
+                    h += hist[c * HS + k];
+                    hist[c * HS + k] = 0;
+                    if (RULE == 1) {
+                        fm = fmaxf(fm, fmax[c * HS + k]);
+                        fmax[c * HS + k] = 0.0f;
+                    }
+                }
+            }
+            const int incl = warp_inclusive_scan(h, lane);
+            float step;
+            if (RULE == 0) {
+                step = __fadd_rn(fminf(k < K ? s.tau_s[k] : 0.0f, Tmax), t_comm);
+            } else {
+                const float fm_incl = warp_inclusive_max_scan(fm, lane);
+                step = __fadd_rn(fmaxf(fm_carry, fm_incl), t_comm);
+                fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fm_incl, 31));
+            }
+            if (k < K) {
+                done_row[k] = carry + incl;
+                step_row[k] = step;
+            }
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        for (int c = lane; c < H; c += 32) {  // the two bins past the last threshold
+            hist[c * HS + K] = 0;
+            hist[c * HS + K + 1] = 0;
+        }
+        if (RULE == 1) {
+            for (int c = lane; c < H; c += 32) {
+                fmax[c * HS + K] = 0.0f;
+                fmax[c * HS + K + 1] = 0.0f;
+            }
+        }
+        if (lane == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
+        buffer_barrier_arrive<kBarFree>(b, bar_threads);  // buffer b is clear again
+    }
+}
+
+// The consumer threads' loop over the block's trials (tiled kernel).
+template <int NQ, int RULE, bool BATCH, bool DIRECT>
+__device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTail &s, const BinCtx &ctx, unsigned char *stage0,
+                                             uint64_t *full, uint64_t *empty, int tid, int lane, int warp, int ncw,
+                                             int *myhist0, unsigned fmax_delta, unsigned off_zero)
+{
+    const int S = p.stages;
+    const int bar_threads = ncw * 32 + 32;
+    const int hist_buf_ints = p.hist_copies * p.hist_stride;
+    // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
+    // (threads past the last row of the box read the last row instead: always inside the stage)
+    const uint32_t row_off = (uint32_t)min(tid, p.rows - 1) * (uint32_t)p.pitch;
+    const uint32_t swz = ((row_off >> 7) & (uint32_t)p.swz_mask) << 4;
+    int st = 0;
+    uint32_t ph = 0;
+    int j = 0;
+    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
+        const int b = j & 1;
+        if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
+        int *myhist = myhist0 + b * hist_buf_ints;
+        unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
+        float rowmax = 0.0f, fin0 = 0.0f;
+        int cnt0 = 0;
+        for (int pass = 0; pass < p.passes; ++pass) {
+            const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
+            float P = 0.0f;
+            unsigned prev = off_zero;  // rule 1: bin (byte offset) of the running time before the next micro-batch
+            for (int c = 0; c < p.chunks; ++c) {
+                mbar_wait(&full[st], ph, kErrLoadNeverArrived);
+                const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes + row_off;
+                uint64_t *empty_bar = &empty[st];
+                if (++st == S) {
+                    st = 0;
+                    ph ^= 1u;
+                }
+                const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
+                float4 v[NQ];
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
+                    else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                }
+                consume_chunk<NQ, RULE, BATCH, DIRECT>(v, 4 * nq, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, empty_bar);
+            }
+            if (valid) rowmax = fmaxf(rowmax, P);
+        }
+        if (cnt0 > 0) {
+            atomicAdd(myhist, cnt0);
+            if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
+        }
+        rowmax = warp_max(rowmax);
+        if (lane == 0) s.smax[32 * b + warp] = rowmax;
+        buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
+    }
+}
+
+template <int NQ, int RULE, bool BATCH>
+__global__ void __launch_bounds__(kMaxRowsPerPass + 64, NQ <= 4 ? 3 : 2)
+dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    // 1024-byte alignment by pointer arithmetic on the shared array itself (a round trip through an integer
+    // would hide the address space from the compiler and turn every shared access into a generic one)
+    unsigned char *smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+    unsigned char *stage0 = smem;
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)p.stages * p.stage_bytes);
+    uint64_t *empty = full + kMaxStages;
+    const SmemTail s = carve_tail(reinterpret_cast<unsigned char *>(empty + kMaxStages), p);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int ncw = (blockDim.x >> 5) - 2;  // consumer warps; then the producer warp, then the epilogue warp
+    const int S = p.stages;
+
+    // The producer thread sets up the barriers and fills the whole ring before the block builds its tables: the
+    // first tiles are on their way from HBM while the thresholds are read and the lookup table is built.
+    // (tile = one chunk of one pass of one trial; the block's tiles in order: trial, pass, chunk)
+    long long prod_t = blockIdx.x;
+    int prod_pass = 0, prod_c = 0, prod_issued = 0;
+    auto issue_tile = [&](int st) {
+        mbar_arrive_expect_tx(&full[st], (uint32_t)(p.rows * p.pitch));
+        tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, prod_c * p.bw, prod_pass * p.rows, (int)prod_t, &full[st]);
+        if (++prod_c == p.chunks) {
+            prod_c = 0;
+            if (++prod_pass == p.passes) {
+                prod_pass = 0;
+                prod_t += gridDim.x;
+            }
+        }
+    };
+    if (warp == ncw && lane == 0) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(&full[i], 1);
+            mbar_init(&empty[i], ncw);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        while (prod_issued < S && prod_t < p.T) issue_tile(prod_issued++);
+    }
+    load_thresholds(p, s, tid, blockDim.x);
+    __syncthreads();  // also: the initialised barriers are visible to every thread
+    build_lut(p, s, tid, blockDim.x);
+
+    if (warp == ncw) {
+        // ---------------- producer: the rest of the tiles, each into the stage its predecessor has been read out of
+        if (lane == 0) {
+            int st = 0;
+            uint32_t ph = 1;  // parity of the current use of stage st (every stage has been used once)
+            while (prod_t < p.T) {
+                mbar_wait(&empty[st], ph ^ 1u, kErrStageNeverFreed);
+                issue_tile(st);
+                if (++st == S) {
+                    st = 0;
+                    ph ^= 1u;
+                }
+            }
+        }
+        return;
+    }
+    if (warp == ncw + 1) {
+        epilogue_warp<RULE>(p, s, lane, ncw);
+        return;
+    }
+
+    // ---------------- consumers
+    int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
+    // rule 1: byte distance from a histogram entry to the finish-time maximum of the same buffer, copy and bin
+    const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));
+    const BinCtx ctx = make_bin_ctx(p, s);
+    const bool one = ctx.one;
+    const unsigned off_zero = RULE == 1 ? bin_of_zero(ctx) : 0u;  // rule 1 only
+    if (s.meta[3] != 0 && one && p.direct_bins != 0)
+        tiled_trials<NQ, RULE, BATCH, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, myhist0, fmax_delta, off_zero);
+    else
+        tiled_trials<NQ, RULE, BATCH, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, myhist0, fmax_delta, off_zero);
+}
+
+}  // namespace

@@ -31,3 +31,29 @@ def test_non_zero_rank_of_reference_arm_does_nothing():
                          cwd=ROOT, env=env)
     assert out.returncode == 0, out.stderr[-2000:]
     assert out.stdout.strip() == ""
+
+
+import pytest
+
+
+@pytest.mark.gpu
+def test_gpu_arm_prints_one_json_line_with_roofline_and_e2e():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "paper_scale", "--trials", "2048",
+                          "--steps", "3", "--warmup", "3"], capture_output=True, text=True, timeout=900, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "roofline", "cpu_baseline", "e2e", "gpu_launches", "clocks"):
+        assert key in d, key
+    assert d["n_gpus"] == 1 and d["steps"] == 3 and d["dtype"] == "f32" and d["data"] == "synthetic"
+    r = d["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 0 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    assert r["algorithmic_bytes_per_launch"] == 4 * 2048 * 200 * 32 + 8 * 2048 * 64 + 4 * 2048
+    assert d["gpu_launches"] == 3 * 4                      # sweep + two reduction kernels + arg-max, per step
+    e = d["e2e"]
+    assert e["h2d_bytes_per_step"] == 4 * 2048 * 200 * 32 + 4 * 64 and e["d2h_bytes_per_step"] > 0 and e["value"] > 0
+    assert e["value"] < d["value"]                         # the copies are inside its timed region
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] > 0
+    assert d["result"]["k_star"] == e["k_star"]

@@ -76,10 +76,10 @@ typedef enum {
  *   out_done[t][k] = #{ (n,m) : P_{t,n,m} < taus[k] }          (= N * M~_t(tau_k); strict '<', fp32)
  *   out_step[t][k] = fl32( fminf(taus[k], max_n P_{t,n,M-1}) + t_comm )   (= min{tau,T} + T^c)
  *
- *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; finite and >= 0.  16-byte aligned with M a
- *              multiple of 4 takes the fastest (tiled) kernel, 16-byte aligned with any other M <= 255 the
- *              flat kernel; any 4-byte aligned pointer and any M are accepted (plain-load kernel, slow);
- *              see dc_simulate_plan
+ *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; finite and >= 0; 4-byte aligned.  A 16-byte aligned
+ *              pointer with M a multiple of 4 takes the fastest (tiled) kernel; every other case takes the flat
+ *              kernel when M <= 255 and the plain-load kernel beyond (roughly 0.3-0.7 and 0.3-0.5 of the tiled
+ *              kernel's rate); see dc_simulate_plan
  *   T, N, M    > 0, N*M <= INT32_MAX
  *   taus       DEVICE, [K] fp32, non-decreasing, no NaN; +infinity is allowed (gives the
  *              synchronous baseline); 4-byte aligned.  1 <= K <= DC_MAX_K

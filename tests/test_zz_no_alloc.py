@@ -19,6 +19,8 @@ RTOL_STATS = 1e-9  # the tolerance the parity tests use for fp64 statistics
 
 @pytest.fixture(scope="module")
 def api():
+    from paper_2306_10598_b200 import build
+    build.build_library()   # compiles the library in-tree if it is missing or older than its sources
     from paper_2306_10598_b200 import api as _api
     assert torch.cuda.is_available(), "GPU tests need a CUDA device"
     return _api

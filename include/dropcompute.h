@@ -76,7 +76,8 @@ typedef enum {
  *   out_done[t][k] = #{ (n,m) : P_{t,n,m} < taus[k] }          (= N * M~_t(tau_k); strict '<', fp32)
  *   out_step[t][k] = fl32( fminf(taus[k], max_n P_{t,n,M-1}) + t_comm )   (= min{tau,T} + T^c)
  *
- *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; finite and >= 0; 4-byte aligned.  A 16-byte aligned
+ *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; finite, >= 0 and small enough that a worker's M
+ *              latencies add up to a finite fp32 number; 4-byte aligned.  A 16-byte aligned
  *              pointer with M a multiple of 4 takes the fastest (tiled) kernel; every other case takes the flat
  *              kernel when M <= 255 and the plain-load kernel beyond (roughly 0.3-0.7 and 0.3-0.5 of the tiled
  *              kernel's rate); see dc_simulate_plan

@@ -164,6 +164,27 @@ def test_zero_and_tie_latencies(api):
     compare_stats(res, ref, N, M)
 
 
+@pytest.mark.parametrize("rule", [0, 1])
+def test_subnormal_and_huge_latencies(api, rule):
+    """Both sides add in IEEE binary32 without flushing: latencies and thresholds in the subnormal range, and
+    latencies near the top of the range (row sums up to 3.2e38, still finite as the interface requires)."""
+    rng = np.random.default_rng(3)
+    T, N, M, K = 3, 40, 16, 24
+    tiny = (rng.integers(0, 2000, (T, N, M)).astype(np.float64) * 1e-42).astype(np.float32)     # multiples of ~1e-42
+    taus = np.sort((rng.integers(0, 20000, K).astype(np.float64) * 1e-42).astype(np.float32))
+    assert tiny.max() < np.finfo(np.float32).tiny and tiny.max() > 0
+    ref = oracle.sweep(tiny, taus, 0.0, rule=rule)
+    res = run_gpu(api, torch.from_numpy(tiny).cuda(), torch.from_numpy(taus).cuda(), 0.0, rule=rule)
+    compare_sweep(res, ref, "(subnormal)")
+    assert ref.done.max() > 0 and ref.done.min() < N * M          # the grid really cuts through the data
+    huge = rng.uniform(1e37, 2e37, (T, N, M)).astype(np.float32)
+    taus = np.array([1e37, 1e38, 2e38, 3e38, 3.3e38, np.inf], np.float32)
+    ref = oracle.sweep(huge, taus, 1e30, rule=rule)
+    assert np.isfinite(ref.sync).all()
+    res = run_gpu(api, torch.from_numpy(huge).cuda(), torch.from_numpy(taus).cuda(), 1e30, rule=rule)
+    compare_sweep(res, ref, "(huge)")
+
+
 def test_thresholds_outside_the_data(api):
     T, N, M = 5, 20, 8
     lat = W.iid_latencies("uniform", T, N, M, seed=7, lo=0.01, hi=0.02).numpy()

@@ -260,9 +260,10 @@ int dc_read_probe(const float *data, int64_t count, float *sink, void *stream);
 
 /*
  * dc_check_inputs — SYNCHRONOUS check of the data preconditions of dc_simulate on `stream`:
- * returns DC_ERR_LATENCIES if any latency is negative, NaN or infinite, DC_ERR_TAUS if the grid is
- * not non-decreasing or holds a NaN, DC_OK otherwise.  report_host (HOST, [2] int64, may be NULL)
- * receives the number of bad latencies and of bad thresholds.
+ * returns DC_ERR_LATENCIES if any latency is negative, NaN or infinite or a worker's latencies add up
+ * (left to right, in fp32) to infinity, DC_ERR_TAUS if the grid is not non-decreasing or holds a NaN,
+ * DC_OK otherwise.  report_host (HOST, [2] int64, may be NULL) receives the number of bad latencies
+ * plus overflowing rows, and the number of bad thresholds.
  *   counters  DEVICE scratch, [2] int64 (16 bytes, 8-byte aligned)
  */
 int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M,

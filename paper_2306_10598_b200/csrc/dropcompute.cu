@@ -674,7 +674,8 @@ int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M, con
     const unsigned long long total = (unsigned long long)T * (unsigned long long)N * (unsigned long long)M;
     unsigned long long want = (total + 255) / 256;
     const unsigned grid = (unsigned)(want < (unsigned long long)di.sms * 8 ? (want ? want : 1) : (unsigned long long)di.sms * 8);
-    dc_check_kernel<<<grid, 256, 0, stream>>>(latencies, total, taus, K, reinterpret_cast<unsigned long long *>(counters));
+    dc_check_kernel<<<grid, 256, 0, stream>>>(latencies, total, (unsigned long long)T * (unsigned long long)N, (int)M, taus, K,
+                                              reinterpret_cast<unsigned long long *>(counters));
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     int64_t host[2] = {0, 0};
     if (cudaMemcpyAsync(host, counters, 16, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return DC_ERR_CUDA;

@@ -236,17 +236,28 @@ dc_combine_groups(const float *__restrict__ g_step, const int32_t *__restrict__ 
     }
 }
 
-// Data precondition check: counts latencies that are negative, NaN or infinite, and thresholds
-// that are NaN or smaller than their predecessor.
+// Data precondition check: counts latencies that are negative, NaN or infinite, rows (one worker's M latencies)
+// of good values whose left-to-right fp32 sum is not finite, and thresholds that are NaN or smaller than their
+// predecessor.
 __global__ void __launch_bounds__(256)
-dc_check_kernel(const float *__restrict__ lat, unsigned long long total, const float *__restrict__ taus, int K,
-                unsigned long long *counters)
+dc_check_kernel(const float *__restrict__ lat, unsigned long long total, unsigned long long rows, int M,
+                const float *__restrict__ taus, int K, unsigned long long *counters)
 {
     unsigned long long bad = 0;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
         const float x = lat[i];
         if (!(x >= 0.0f) || !(x <= 3.402823466e38f)) ++bad;
+    }
+    for (unsigned long long r = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; r < rows; r += stride) {
+        float P = 0.0f;
+        bool good = true;
+        for (int m = 0; m < M; ++m) {
+            const float x = lat[r * (unsigned long long)M + m];
+            good = good && (x >= 0.0f) && (x <= 3.402823466e38f);
+            P = __fadd_rn(P, x);
+        }
+        if (good && !(P <= 3.402823466e38f)) ++bad;
     }
     if (bad) atomicAdd(&counters[0], bad);
     if (blockIdx.x == 0) {

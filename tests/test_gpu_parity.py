@@ -305,6 +305,13 @@ def test_check_inputs(api):
     bad[1, 2, 3] = float("nan")
     with pytest.raises(api.DropComputeError):
         api.dc_check_inputs(bad, taus)
+    over = lat.clone()
+    over[2, 1, :] = 1e38                       # every value is fine, their sum is not
+    with pytest.raises(api.DropComputeError) as e:
+        api.dc_check_inputs(over, taus)
+    assert e.value.status == 8
+    over[2, 1, 3:] = 0.0                       # 3e38: finite again
+    api.dc_check_inputs(over, taus)
     with pytest.raises(api.DropComputeError) as e:
         api.dc_check_inputs(lat, torch.tensor([0.3, 0.2], device="cuda"))
     assert e.value.status == 5

@@ -41,20 +41,28 @@ __global__ void __launch_bounds__(kMaxRowsPerPass) dc_sweep_plain(const SweepPar
             const float *src = p.lat + ((size_t)t * p.N + (size_t)max(n0, 0)) * M;
             float P = 0.0f;
             unsigned prev = off_zero;
+            // lane = column: row rr's piece of a chunk is one coalesced read of up to 128 bytes.  The next chunk's
+            // pieces are requested before the current chunk is walked, so the loads overlap the walk.
+            float nx[32];
+            auto fetch = [&](int m0) {
+                const int ns = min(32, M - m0);
+#pragma unroll
+                for (int rr = 0; rr < 32; ++rr) {
+                    nx[rr] = 0.0f;
+                    if (rr < nrows && lane < ns) nx[rr] = __ldg(src + (size_t)rr * M + m0 + lane);
+                }
+            };
+            fetch(0);
             for (int m0 = 0; m0 < M; m0 += 32) {
                 const int ns = min(32, M - m0);
-                // lane = column: row rr's piece is one coalesced read of up to 128 bytes
-#pragma unroll 8
-                for (int rr = 0; rr < 32; ++rr) {
-                    float x = 0.0f;
-                    if (rr < nrows && lane < ns) x = __ldg(src + (size_t)rr * M + m0 + lane);
-                    tile[rr * 33 + lane] = x;
-                }
+#pragma unroll
+                for (int rr = 0; rr < 32; ++rr) tile[rr * 33 + lane] = nx[rr];
                 __syncwarp();
                 float4 v[8];  // lane = row
 #pragma unroll
                 for (int e = 0; e < 32; ++e) sample_ref(v, e) = tile[lane * 33 + e];
                 __syncwarp();
+                if (m0 + 32 < M) fetch(m0 + 32);
                 consume_chunk<8, RULE, false, false>(v, ns, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, nullptr);
             }
             if (valid) rowmax = fmaxf(rowmax, P);

@@ -79,7 +79,7 @@ typedef enum {
  *   latencies  DEVICE, [T][N][M] fp32, contiguous, m fastest; finite, >= 0 and small enough that a worker's M
  *              latencies add up to a finite fp32 number; 4-byte aligned.  A 16-byte aligned
  *              pointer with M a multiple of 4 takes the fastest (tiled) kernel; every other case takes the flat
- *              kernel when M <= 255 and the plain-load kernel beyond (roughly 0.3-0.7 and 0.3-0.5 of the tiled
+ *              kernel when M <= 127 and the plain-load kernel beyond (roughly 0.3-0.7 and 0.4-0.6 of the tiled
  *              kernel's rate); see dc_simulate_plan
  *   T, N, M    > 0, N*M <= INT32_MAX
  *   taus       DEVICE, [K] fp32, non-decreasing, no NaN; +infinity is allowed (gives the
@@ -279,8 +279,8 @@ int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M,
 int dc_device_status(uint32_t *flags_host);
 
 /* Which kernel dc_simulate_ex would use for a shape: 0 = tiled kernel (M a multiple of 4 and a 16-byte aligned
- * pointer), 2 = flat kernel (any other case with M <= 255: other row lengths, or a pointer that is only 4-byte
- * aligned), 1 = plain-load kernel (such cases with longer rows), negative = -dc_status. */
+ * pointer), 2 = flat kernel (any other case with M <= 127, or up to DC_TUNE_FLAT_MAX_M: other row lengths, or a
+ * pointer that is only 4-byte aligned), 1 = plain-load kernel (such cases with longer rows), negative = -dc_status. */
 int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K);
 
 /*
@@ -294,6 +294,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  *   DC_TUNE_BOX_FLOATS   floats of a row fetched per tile (16 or 32; 16 needs M to be a multiple of 16)
  *   DC_TUNE_DIRECT_BINS  1 = always bin through the lookup table, 2 = bin evenly spaced thresholds arithmetically
  *                        (one multiply-add and one comparison per sample, no table read) in the tiled kernel
+ *   DC_TUNE_FLAT_MAX_M   longest row (1..255) the flat kernel is given instead of the plain-load kernel (default 127)
  *   DC_TUNE_FLAT_TILE_WARPS, DC_TUNE_FLAT_GROUPS, DC_TUNE_FLAT_DEPTH  flat kernel (row length not a multiple
  *                        of 4): warps per tile (tile = 32 x that many rows), groups of warps working on different
  *                        tiles at once, ring stages per group; used only when all three are set, and a setting
@@ -309,6 +310,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
 #define DC_TUNE_FLAT_TILE_WARPS 7
 #define DC_TUNE_FLAT_GROUPS 8
 #define DC_TUNE_FLAT_DEPTH 9
+#define DC_TUNE_FLAT_MAX_M 11
 int dc_tune(int32_t key, int32_t value);
 
 /* Number of kernel launches the last successful call of each entry point enqueues (for accounting). */

@@ -106,6 +106,7 @@ int g_tune_warp_groups = 0;  // 0 = automatic
 int g_tune_box_floats = 0;   // 0 = automatic
 int g_tune_batch = 0;        // 0 = automatic, 1 = off, 2 = on
 int g_tune_direct = 0;       // 0 = automatic (on), 1 = off, 2 = on
+int g_tune_flat_max_m = 0;   // 0 = automatic (kFlatAutoMaxM), else the longest row the flat kernel is given (<= kFlatMaxM)
 int g_tune_flat_tile_warps = 0, g_tune_flat_groups = 0, g_tune_flat_depth = 0;  // flat kernel; all three or none
 int g_last_simulate_launches = 0;
 int g_last_reduce_launches = 0;
@@ -128,7 +129,8 @@ int validate_simulate(const float *lat, int64_t T, int64_t N, int64_t M, const f
 bool tiled_ok(const float *lat, int64_t M) { return (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0); }
 bool flat_ok(const float *lat, int64_t M)
 {
-    return !tiled_ok(lat, M) && M <= kFlatMaxM;  // any 4-byte aligned base (validate_simulate checks that)
+    // any 4-byte aligned base; rows beyond kFlatAutoMaxM measured faster in the plain-load kernel
+    return !tiled_ok(lat, M) && M <= (g_tune_flat_max_m > 0 ? g_tune_flat_max_m : kFlatAutoMaxM);
 }
 
 template <int RULE, bool BATCH, int NQ>
@@ -839,6 +841,10 @@ int dc_tune(int32_t key, int32_t value)
     }
     if (key == DC_TUNE_BATCH_LOOKUPS && value >= 0 && value <= 2) {
         g_tune_batch = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_FLAT_MAX_M && value >= 0 && value <= kFlatMaxM) {
+        g_tune_flat_max_m = value;
         return DC_OK;
     }
     if (key == DC_TUNE_FLAT_TILE_WARPS && value >= 0 && value <= 8) {

@@ -15,7 +15,8 @@ constexpr int kHistBudgetBytes = 32 * 1024;   // shared memory spent on per-warp
 constexpr uint32_t kWaitLimit = 1u << 22;     // polls of one mbarrier wait before giving up (roughly a second)
 constexpr int kReduceChunksMax = 64;          // partial sums per threshold in dc_reduce_trials
 constexpr int kConsumerBarrier = 1;           // named barrier used by the consumer warps
-constexpr int kFlatMaxM = 255;                // longest row the flat kernel takes (32 rows of it fill a stage)
+constexpr int kFlatMaxM = 255;                // longest row the flat kernel can take (32 rows of it fill a 32 KB stage)
+constexpr int kFlatAutoMaxM = 127;            // longest row it is given by default (32 rows within 16 KB)
 constexpr int kLutCellsMax = 4096;            // cells of the bin lookup table (4 per threshold up to this)
 
 constexpr uint32_t kErrLoadNeverArrived = 1u;

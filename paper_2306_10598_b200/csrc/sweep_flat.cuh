@@ -6,7 +6,8 @@ namespace {
 
 // ------------------------------------------------------------------------------------------
 // Flat kernel: rows whose length is not a multiple of 4 (so a tensor map cannot describe them), up to
-// kFlatMaxM samples, and any row length up to that when the base pointer is only 4-byte aligned.  Consecutive rows of a trial are one contiguous span of the
+// kFlatAutoMaxM samples (kFlatMaxM on request), and any row length up to that when the base pointer is only 4-byte
+// aligned.  Consecutive rows of a trial are one contiguous span of the
 // tensor.  A tile is `rows` consecutive rows (a multiple of 32, at most 32 KB); the producer brings the 16-byte
 // aligned span that covers it into a stage with ONE plain bulk copy (cp.async.bulk, no tensor map) and thread r
 // of the tile's warps reads its row from float offset delta + r*M with 4-byte shared loads, 32 samples at a time.

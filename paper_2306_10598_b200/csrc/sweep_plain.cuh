@@ -5,7 +5,7 @@
 namespace {
 
 // ------------------------------------------------------------------------------------------
-// Plain-load kernel for what neither staged kernel takes (rows longer than kFlatMaxM whose length is not a
+// Plain-load kernel for what neither staged kernel takes (rows longer than kFlatAutoMaxM whose length is not a
 // multiple of 4 or whose base is only 4-byte aligned).  No TMA: for each chunk of 32 columns a warp loads the
 // 32-float pieces of its 32 rows with ordinary coalesced loads (lane = column), parks them in a 32 x 33 tile of
 // its own in shared memory and each lane then takes its row's 32 samples from there (lane = row).  The walk is

@@ -120,10 +120,10 @@ def test_base_pointer_only_4_byte_aligned(api, T, N, M, K):
             buf = torch.full((T * N * M + shift + 5,), float("nan"), dtype=torch.float32, device="cuda")
             view = buf[shift:shift + T * N * M].view(T, N, M)
             view.copy_(torch.from_numpy(lat))
-            assert api.dc_simulate_plan(view, K) == (2 if M <= 255 else 1)
+            assert api.dc_simulate_plan(view, K) == (2 if M <= 127 else 1)
             res = run_gpu(api, view, taus_d, 0.3, rule=rule)
             compare_sweep(res, ref, f"(shift {shift}, rule {rule})")
-    assert api.dc_simulate_plan(torch.from_numpy(lat).cuda(), K) == (0 if M % 4 == 0 else (2 if M <= 255 else 1))
+    assert api.dc_simulate_plan(torch.from_numpy(lat).cuda(), K) == (0 if M % 4 == 0 else (2 if M <= 127 else 1))
     api.dc_device_status()
 
 
@@ -661,6 +661,7 @@ def test_flat_kernel_shapes(api):
              (2, 200, 255, 4096), (2, 300, 126, 3000)]   # the last two: ring and tables compete for shared memory
     splits = [(0, 0, 0), (1, 8, 1), (1, 4, 2), (2, 4, 1), (2, 2, 2), (1, 3, 2), (4, 2, 1), (1, 5, 1), (8, 1, 2)]
     try:
+        api.dc_tune(api.TUNE_FLAT_MAX_M, 255)      # rows of 128-255 samples go to the plain-load kernel by default
         for (T, N, M, K) in cases:
             lat = W.iid_latencies("shifted_exp", T, N, M, seed=900 + T + N + M, shift=0.01, mean=0.02).numpy()
             taus = grid_for(lat, K, seed=K + 5)
@@ -681,15 +682,17 @@ def test_flat_kernel_shapes(api):
                         continue
                     compare_sweep(res, ref, f"flat {(T, N, M, K)} rule {rule} split {(wt, groups, depth)}")
     finally:
+        api.dc_tune(api.TUNE_FLAT_MAX_M, 0)
         api.dc_tune(api.TUNE_FLAT_TILE_WARPS, 0)
         api.dc_tune(api.TUNE_FLAT_GROUPS, 0)
         api.dc_tune(api.TUNE_FLAT_DEPTH, 0)
     api.dc_device_status()
 
 
-@pytest.mark.parametrize("T,N,M,K", [(3, 600, 257, 64), (2, 300, 301, 17), (5, 33, 514, 256), (2, 1, 999, 5), (40, 7, 258, 1)])
+@pytest.mark.parametrize("T,N,M,K", [(3, 600, 257, 64), (2, 300, 301, 17), (5, 33, 514, 256), (2, 1, 999, 5), (40, 7, 258, 1),
+                                      (4, 300, 129, 40), (3, 100, 255, 33), (6, 64, 150, 16)])
 def test_plain_kernel_shapes(api, T, N, M, K):
-    """Rows longer than 255 samples whose length is not a multiple of 4 (plain-load kernel: a warp stages 32 x 32
+    """Rows longer than 127 samples whose length is not a multiple of 4 (plain-load kernel: a warp stages 32 x 32
     pieces of its rows through a tile of its own): several passes per trial, ragged last warp and last chunk, a
     single worker, both rules, dyadic latencies so that running sums land ON thresholds."""
     lat = W.iid_latencies("dyadic", T, N, M, seed=300 + M, hi=6).numpy()

@@ -63,6 +63,7 @@ def test_argument_errors_need_no_gpu(lib):
     assert lib.dc_simulate_plan(A, 4, 8, 12, 3) == 0
     assert lib.dc_simulate_plan(A, 4, 8, 13, 3) == 2
     assert lib.dc_simulate_plan(A, 4, 8, 301, 3) == 1
+    assert lib.dc_simulate_plan(A, 4, 8, 127, 3) == 2 and lib.dc_simulate_plan(A, 4, 8, 129, 3) == 1
     assert lib.dc_simulate_plan(A + 4, 4, 8, 12, 3) == 2
     assert lib.dc_simulate_plan(A + 4, 4, 8, 300, 3) == 1
     assert lib.dc_simulate_plan(A, 4, 8, 12, 5000) == -4

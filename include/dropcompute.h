@@ -110,8 +110,8 @@ int dc_simulate_ex(const float *latencies, int64_t T, int64_t N, int64_t M,
                    int32_t rule, void *stream);
 
 /*
- * dc_simulate_tc — dc_simulate_ex with the communication time given per trial, as Algorithm 2 has it
- * ("communication time for each iteration T_i^c"):
+ * dc_simulate_tc — dc_simulate_ex with one communication time per trial (Algorithm 2, input T_i^c: the
+ * algorithm takes a measured value for every iteration):
  *   t_comm_trials  DEVICE, [T] fp32; trial t uses t_comm_trials[t] wherever dc_simulate_ex uses t_comm.
  * Everything else as dc_simulate_ex.  dc_reduce_trials needs no change: it works from out_step and out_sync.
  */
@@ -172,7 +172,9 @@ int dc_reduce_trials(const float *out_step, const int32_t *out_done, const float
  * Same arguments, results and error codes as dc_reduce_trials without the workspace pair, plus:
  *   K <= DC_STATIC_MAX_K, otherwise DC_ERR_RANGE (the array is sized for that many thresholds; use
  *   dc_reduce_trials with your own workspace beyond it).  T is not limited.
- * The call allocates and frees nothing, neither directly nor through a library routine.
+ * The call allocates and frees nothing, neither directly nor through a library routine.  (What the CUDA runtime
+ * itself does when a device first uses this library is outside the call's control: the library image, the array
+ * included, is made resident on that device at the first call of any entry point there.)
  * The first call on each device looks up the array's device address (one runtime query, cached); make that
  * first call outside any stream capture.
  * All calls on a device share the one array.  Nothing in it has to be cleared between calls — each call

@@ -65,7 +65,7 @@ def build(force: bool = False, source: str | None = None, out: str | None = None
 def _bind(lib):
     i64, i32, f32 = ctypes.c_int64, ctypes.c_int, ctypes.c_float
     p = ctypes.c_void_p
-    for name in ("dco_sweep_literal", "dco_sweep_rows"):
+    for name in ("dco_sweep_definition", "dco_sweep_rows"):
         fn = getattr(lib, name)
         fn.argtypes = [p, i64, i64, i64, p, i64, f32, p, i32, p, p, p]
         fn.restype = i32
@@ -73,8 +73,8 @@ def _bind(lib):
     lib.dco_reduce_trials.restype = i32
     lib.dco_argmax.argtypes = [p, i64]
     lib.dco_argmax.restype = i64
-    lib.dco_algorithm2.argtypes = [p, i64, i64, i64, p, i64, f32, p, p]
-    lib.dco_algorithm2.restype = i32
+    lib.dco_s_eff_fractional.argtypes = [p, i64, i64, i64, p, i64, f32, p, p]
+    lib.dco_s_eff_fractional.restype = i32
     f64 = ctypes.c_double
     lib.dco_closed_form.argtypes = [f64, f64, i64, i64, f64, f64, p, i64, p, p]
     lib.dco_closed_form.restype = i32
@@ -126,7 +126,8 @@ def _f32c(a, ndim):
 def sweep(lat, taus, t_comm: float, rule: int = 0, order: str = "rows", lib=None) -> Sweep:
     """Per-(iteration, tau) step time and completed count.
 
-    ``order='literal'`` runs Algorithm 2's loop nest as printed (tau outermost);
+    ``order='definition'`` writes out each iteration's table of finish times and reads every quantity off
+    it, one threshold at a time (Sec. 4.3's definitions as they stand);
     ``order='rows'`` reads every sample once (same predicate, same integers).
     ``t_comm`` is one number, or an array of T numbers (Algorithm 2's per-iteration T_i^c)."""
     lib = lib or load()
@@ -137,7 +138,7 @@ def sweep(lat, taus, t_comm: float, rule: int = 0, order: str = "rows", lib=None
     step = np.empty((T, K), np.float32)
     done = np.empty((T, K), np.int32)
     sync = np.empty((T,), np.float32)
-    fn = {"literal": lib.dco_sweep_literal, "rows": lib.dco_sweep_rows}[order]
+    fn = {"definition": lib.dco_sweep_definition, "rows": lib.dco_sweep_rows}[order]
     tc_vec = None
     if np.ndim(t_comm) > 0:
         tc_vec = np.ascontiguousarray(t_comm, dtype=np.float32)
@@ -172,8 +173,9 @@ def argmax(objective, lib=None) -> int:
     return int(lib.dco_argmax(obj.ctypes.data, obj.shape[0]))
 
 
-def algorithm2(lat, taus, t_comm: float, lib=None):
-    """Algorithm 2 start to finish as printed (floating-point 1/N accumulation)."""
+def s_eff_fractional(lat, taus, t_comm: float, lib=None):
+    """S_eff(tau) and its first maximum with M~ accumulated as a floating-point mean over workers (Sec. 4.3's
+    (1/N) sum_n form) instead of the integer count used everywhere else."""
     lib = lib or load()
     lat = _f32c(lat, 3)
     taus = _f32c(taus, 1)
@@ -181,10 +183,10 @@ def algorithm2(lat, taus, t_comm: float, lib=None):
     K = taus.shape[0]
     s_eff = np.empty((K,), np.float64)
     k_star = ctypes.c_int64(-1)
-    rc = lib.dco_algorithm2(lat.ctypes.data, T, N, M, taus.ctypes.data, K, np.float32(t_comm),
+    rc = lib.dco_s_eff_fractional(lat.ctypes.data, T, N, M, taus.ctypes.data, K, np.float32(t_comm),
                             s_eff.ctypes.data, ctypes.byref(k_star))
     if rc != 0:
-        raise ValueError(f"oracle algorithm2 failed with status {rc}")
+        raise ValueError(f"oracle s_eff_fractional failed with status {rc}")
     return s_eff, int(k_star.value)
 
 

@@ -7,19 +7,20 @@
  * include, link or call it, and it shares no code with the CUDA sources.
  *
  * What is stated here (paper: DropCompute, arXiv 2306.10598):
- *   - Algorithm 2 ("Automatic choice for the optimal threshold tau"), App. C.1:
- *     the loop nest, the running sum T_{i,n} += t_{i,n}^{(m)}, the strict test
- *     T_{i,n} < tau, T_i = max_n T_{i,n}, S_i(tau), S_eff(tau), tau*.
- *   - Sec. 4.3: completed micro-batches M~ (inclusive running sum < tau) and
- *     the DropCompute step time min{tau, T} + T^c.
+ *   - Sec. 4.3: a worker's finish times T_n^{(m)} (inclusive running sums), the
+ *     completed micro-batches M~ (those with T_n^{(m)} < tau, strict) and the
+ *     DropCompute step time min{tau, T} + T^c with T = max_n T_n^{(M)}.
+ *   - Algorithm 2, App. C.1 (the automatic choice of tau): what it evaluates per
+ *     candidate tau and measured iteration (the quantities above), the
+ *     per-iteration speedup S_i(tau), its mean S_eff(tau), and tau* = arg max.
  *   - Sec. 4.4, Eq. 6: effective speedup and throughput N*M~ / (min{tau,T}+T^c).
  *
  * Readings taken where the paper is silent (each is listed in the design notes):
  *   - samples, running sums, comparisons and step times are IEEE binary32;
  *     one rounding per addition, micro-batches strictly in the order m=1..M;
  *   - M~ is kept as the integer number of completed micro-batches summed over
- *     workers (Algorithm 2 adds 1/N per hit; the integer count divided once at
- *     the end is the same number in exact arithmetic);
+ *     workers (the paper averages over workers in floating point; the integer
+ *     count divided once at the end is the same number in exact arithmetic);
  *   - T^c is given per iteration as in Algorithm 2, or as one scalar used for all iterations;
  *   - statistics over iterations are binary64;
  *   - argmax takes the first maximum and never selects a NaN.
@@ -31,7 +32,8 @@
  * last micro-batch it ran.
  *
  * Pins (tests/test_oracle_pins.py and friends): harmonic-number mean of the
- * max of exponentials, quadrature of Eq. 3 for normals, Eq. 5 (exact for
+ * max of exponentials, quadrature of Eq. 3 for normals (which also bounds
+ * Eq. 4's approximation from one side), Eq. 5 (exact for
  * normal micro-batches), Erlang CDF for shifted exponentials, exhaustive
  * enumeration of tiny dyadic laws in rational arithmetic, a hand-worked
  * example, M=1 against sort/searchsorted, invariants, and mutation checks.
@@ -47,66 +49,83 @@
 #define DCO_NSTATS 5 /* mean_step, done_frac, thr, thr_mean, s_eff */
 
 /* ---------------------------------------------------------------------------
- * Algorithm 2 in the paper's own loop order: tau outermost, then iteration i,
- * worker n, micro-batch m.  Writes the per-(iteration, tau) quantities.
+ * The per-(iteration, tau) quantities straight from their definitions in Sec. 4.3.
+ * For every iteration the table of finish times T_n^{(m)} = sum_{j<=m} t_n^{(j)}
+ * is written out first; everything else is read off that table, one threshold
+ * at a time:
+ *   completed micro-batches   N * M~(tau) = #{(n,m) : T_n^{(m)} < tau}
+ *   slowest worker            T = max_n T_n^{(M)}
+ *   step time                 min{tau, T} + T^c
+ * This is also what Algorithm 2 (App. C.1) evaluates for each candidate tau.
  *   lat      [T,N,M] binary32, m fastest
  *   taus     [K]
- *   out_step [T,K]  min(tau, T_i) + T^c            (rule 0)
+ *   out_step [T,K]  step time
  *   out_done [T,K]  N * M~_i(tau) as an integer
  *   out_sync [T]    T_i + T^c   (the tau = infinity step time)
- *   t_comm_per_iter [T] or NULL: Algorithm 2 takes the communication time T_i^c per iteration; when this is
+ *   t_comm_per_iter [T] or NULL: Algorithm 2's input T_i^c, one value per iteration; when this is
  *                   NULL the one scalar t_comm is used for every iteration.
+ * rule 1 (Limitations paragraph): micro-batch m starts at T_n^{(m-1)} (0 for the first) and is run
+ * iff that is < tau; the worker's time is the finish time of the last micro-batch it ran, and the
+ * step time is the slowest worker's time plus T^c.
  * ------------------------------------------------------------------------- */
-int dco_sweep_literal(const float *lat, int64_t T, int64_t N, int64_t M,
-                      const float *taus, int64_t K, float t_comm, const float *t_comm_per_iter, int rule,
-                      float *out_step, int32_t *out_done, float *out_sync)
+int dco_sweep_definition(const float *lat, int64_t T, int64_t N, int64_t M,
+                         const float *taus, int64_t K, float t_comm, const float *t_comm_per_iter, int rule,
+                         float *out_step, int32_t *out_done, float *out_sync)
 {
     if (!lat || !taus || !out_step || !out_done || !out_sync) return 1;
     if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return 2;
     if (rule != 0 && rule != 1) return 7;
-    for (int64_t k = 0; k < K; ++k) {
-        const float tau = taus[k];
-        for (int64_t i = 0; i < T; ++i) {
-            const float tc = t_comm_per_iter ? t_comm_per_iter[i] : t_comm;  /* T_i^c of Algorithm 2 */
-            int64_t done = 0;      /* N * M~_i(tau) */
-            float Ti = 0.0f;       /* slowest worker's full compute time */
-            float Wi = 0.0f;       /* slowest worker's time under the threshold (rule 1) */
-            for (int64_t n = 0; n < N; ++n) {
-                const float *t = lat + (i * N + n) * M;
-                float Tin = 0.0f;  /* running compute time of worker n */
-                float Win = 0.0f;  /* finish time of the last micro-batch it ran (rule 1) */
-                for (int64_t m = 0; m < M; ++m) {
-                    if (rule == 0) {
-                        Tin = Tin + t[m];
-                        if (Tin < tau) done += 1;
-                    } else {
-                        /* started iff the time elapsed BEFORE it is < tau */
-                        if (Tin < tau) {
-                            done += 1;
-                            Win = Tin + t[m];
-                        }
-                        Tin = Tin + t[m];
-                    }
-                }
-                Ti = fmaxf(Ti, Tin);
-                Wi = fmaxf(Wi, Win);
+    float *finish = (float *)malloc((size_t)N * (size_t)M * sizeof(float));
+    if (!finish) return 6;
+    for (int64_t i = 0; i < T; ++i) {
+        const float tc = t_comm_per_iter ? t_comm_per_iter[i] : t_comm;
+        /* finish times: binary32, one rounding per addition, micro-batches in order */
+        for (int64_t n = 0; n < N; ++n) {
+            const float *row = lat + (i * N + n) * M;
+            float elapsed = 0.0f;
+            for (int64_t m = 0; m < M; ++m) {
+                elapsed = elapsed + row[m];
+                finish[n * M + m] = elapsed;
             }
-            if (rule == 0)
-                out_step[i * K + k] = fminf(tau, Ti) + tc;
-            else
-                out_step[i * K + k] = Wi + tc;
-            out_done[i * K + k] = (int32_t)done;
-            out_sync[i] = Ti + tc;
+        }
+        float slowest_full = 0.0f; /* T = max_n T_n^{(M)} */
+        for (int64_t n = 0; n < N; ++n) slowest_full = fmaxf(slowest_full, finish[n * M + (M - 1)]);
+        out_sync[i] = slowest_full + tc;
+        for (int64_t k = 0; k < K; ++k) {
+            const float tau = taus[k];
+            int64_t completed = 0;
+            float slowest_cut = 0.0f; /* rule 1: max_n (finish time of the last micro-batch worker n ran) */
+            for (int64_t n = 0; n < N; ++n) {
+                const float *f = finish + n * M;
+                if (rule == 0) {
+                    for (int64_t m = 0; m < M; ++m) completed += (f[m] < tau) ? 1 : 0;
+                } else {
+                    int64_t last_run = -1;
+                    for (int64_t m = 0; m < M; ++m) {
+                        const float start = (m == 0) ? 0.0f : f[m - 1];
+                        if (start < tau) {
+                            completed += 1;
+                            last_run = m;
+                        }
+                    }
+                    slowest_cut = fmaxf(slowest_cut, last_run >= 0 ? f[last_run] : 0.0f);
+                }
+            }
+            out_done[i * K + k] = (int32_t)completed;
+            out_step[i * K + k] = (rule == 0) ? (fminf(tau, slowest_full) + tc) : (slowest_cut + tc);
         }
     }
+    free(finish);
     return 0;
 }
 
 /* ---------------------------------------------------------------------------
- * The same quantities with the loops in the order iteration, worker,
+ * The same quantities in one pass over the samples: iteration, worker,
  * micro-batch, tau.  The predicate evaluated for every (i,n,m,k) is the same
- * and the counts are integers, so no output bit can differ from the literal
- * order; this form reads the samples once and is the one used on large inputs.
+ * and the counts are integers, so no output bit can differ from the form
+ * above; this one reads the samples once and is used on large inputs.
+ * Under rule 1 each worker keeps, per threshold, the finish time of the last
+ * micro-batch it ran; the step takes the maximum of those over workers.
  * Iterations are independent and are spread over OpenMP threads.
  * ------------------------------------------------------------------------- */
 int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
@@ -120,45 +139,49 @@ int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
 #pragma omp parallel
     {
         int64_t *cnt = (int64_t *)malloc((size_t)K * sizeof(int64_t));
-        float *wmax = (float *)malloc((size_t)K * sizeof(float));
-        if (!cnt || !wmax) {
+        float *wmax = (float *)malloc((size_t)K * sizeof(float));   /* rule 1: slowest worker's time per threshold */
+        float *wlast = (float *)malloc((size_t)K * sizeof(float));  /* rule 1: this worker's time per threshold */
+        if (!cnt || !wmax || !wlast) {
 #pragma omp atomic write
             failed = 1;
         }
 #pragma omp for schedule(dynamic, 1)
         for (int64_t i = 0; i < T; ++i) {
-            if (!cnt || !wmax) continue;
-            const float tc = t_comm_per_iter ? t_comm_per_iter[i] : t_comm;  /* T_i^c of Algorithm 2 */
-            float Ti = 0.0f;
+            if (!cnt || !wmax || !wlast) continue;
+            const float tc = t_comm_per_iter ? t_comm_per_iter[i] : t_comm;
+            float slowest_full = 0.0f;
             for (int64_t k = 0; k < K; ++k) { cnt[k] = 0; wmax[k] = 0.0f; }
             for (int64_t n = 0; n < N; ++n) {
-                const float *t = lat + (i * N + n) * M;
-                float Tin = 0.0f;
+                const float *row = lat + (i * N + n) * M;
+                float elapsed = 0.0f;
+                if (rule == 1) for (int64_t k = 0; k < K; ++k) wlast[k] = 0.0f;
                 for (int64_t m = 0; m < M; ++m) {
                     if (rule == 0) {
-                        Tin = Tin + t[m];
-                        for (int64_t k = 0; k < K; ++k) cnt[k] += (Tin < taus[k]) ? 1 : 0;
+                        elapsed = elapsed + row[m];
+                        for (int64_t k = 0; k < K; ++k) cnt[k] += (elapsed < taus[k]) ? 1 : 0;
                     } else {
-                        const float before = Tin;
-                        Tin = Tin + t[m];
+                        const float start = elapsed;
+                        elapsed = elapsed + row[m];
                         for (int64_t k = 0; k < K; ++k) {
-                            if (before < taus[k]) {
+                            if (start < taus[k]) {
                                 cnt[k] += 1;
-                                wmax[k] = fmaxf(wmax[k], Tin);
+                                wlast[k] = elapsed;
                             }
                         }
                     }
                 }
-                Ti = fmaxf(Ti, Tin);
+                slowest_full = fmaxf(slowest_full, elapsed);
+                if (rule == 1) for (int64_t k = 0; k < K; ++k) wmax[k] = fmaxf(wmax[k], wlast[k]);
             }
-            out_sync[i] = Ti + tc;
+            out_sync[i] = slowest_full + tc;
             for (int64_t k = 0; k < K; ++k) {
-                out_step[i * K + k] = (rule == 0) ? (fminf(taus[k], Ti) + tc) : (wmax[k] + tc);
+                out_step[i * K + k] = (rule == 0) ? (fminf(taus[k], slowest_full) + tc) : (wmax[k] + tc);
                 out_done[i * K + k] = (int32_t)cnt[k];
             }
         }
         free(cnt);
         free(wmax);
+        free(wlast);
     }
     return failed ? 6 : 0;
 }
@@ -218,36 +241,51 @@ int64_t dco_argmax(const double *objective, int64_t K)
 }
 
 /* ---------------------------------------------------------------------------
- * Algorithm 2 start to finish, exactly as printed, including the 1/N
- * accumulation of M~ in floating point (binary64 here) — used only to check
- * that the integer-count reading above gives the same S_eff and tau*.
+ * S_eff(tau) with M~ taken as a floating-point mean over workers, the way
+ * Sec. 4.3 writes it: M~_i(tau) = (1/N) sum_n c_n, c_n = #{m : T_n^{(m)} < tau},
+ * accumulated in binary64 one worker at a time; then Eq. 6 per iteration,
+ *   S_i(tau) = (M~_i / M) * (T_i + T^c) / (min{tau, T_i} + T^c),
+ * the mean over iterations, and the first maximum.  Exists only so that a test can
+ * show that keeping N * M~ as an integer (the reading used everywhere else in this
+ * file) gives the same S_eff and the same tau*.
  * ------------------------------------------------------------------------- */
-int dco_algorithm2(const float *lat, int64_t T, int64_t N, int64_t M,
-                   const float *taus, int64_t K, float t_comm,
-                   double *s_eff, int64_t *k_star)
+int dco_s_eff_fractional(const float *lat, int64_t T, int64_t N, int64_t M,
+                         const float *taus, int64_t K, float t_comm,
+                         double *s_eff, int64_t *k_star)
 {
     if (!lat || !taus || !s_eff || !k_star) return 1;
     if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return 2;
-    for (int64_t k = 0; k < K; ++k) {
-        const float tau = taus[k];
-        double acc = 0.0;
-        for (int64_t i = 0; i < T; ++i) {
-            double Mt = 0.0;
-            float Ti = 0.0f;
+    float *total = (float *)malloc((size_t)N * sizeof(float));
+    int64_t *c = (int64_t *)malloc((size_t)N * sizeof(int64_t));
+    if (!total || !c) { free(total); free(c); return 6; }
+    for (int64_t k = 0; k < K; ++k) s_eff[k] = 0.0;
+    for (int64_t i = 0; i < T; ++i) {
+        for (int64_t k = 0; k < K; ++k) {
+            const float tau = taus[k];
             for (int64_t n = 0; n < N; ++n) {
-                float Tin = 0.0f;
+                const float *row = lat + (i * N + n) * M;
+                float elapsed = 0.0f;
+                c[n] = 0;
                 for (int64_t m = 0; m < M; ++m) {
-                    Tin = Tin + lat[(i * N + n) * M + m];
-                    Mt = Mt + (1.0 / (double)N) * ((Tin < tau) ? 1.0 : 0.0);
+                    elapsed = elapsed + row[m];
+                    c[n] += (elapsed < tau) ? 1 : 0;
                 }
-                Ti = fmaxf(Ti, Tin);
+                total[n] = elapsed;
             }
-            const float num = Ti + t_comm;
-            const float den = fminf(tau, Ti) + t_comm;
-            acc += ((double)num / (double)den) * (Mt / (double)M);
+            double m_tilde = 0.0;
+            float slowest = 0.0f;
+            for (int64_t n = 0; n < N; ++n) {
+                m_tilde += (double)c[n] / (double)N;
+                slowest = fmaxf(slowest, total[n]);
+            }
+            const double sync_time = (double)(slowest + t_comm);
+            const double drop_time = (double)(fminf(tau, slowest) + t_comm);
+            s_eff[k] += (m_tilde / (double)M) * (sync_time / drop_time);
         }
-        s_eff[k] = acc / (double)T;
     }
+    for (int64_t k = 0; k < K; ++k) s_eff[k] /= (double)T;
+    free(total);
+    free(c);
     *k_star = dco_argmax(s_eff, K);
     return 0;
 }
@@ -259,7 +297,7 @@ int dco_algorithm2(const float *lat, int64_t T, int64_t N, int64_t M,
  *   Phi        standard normal CDF, here 0.5 erfc(-x / sqrt 2)
  *   Phi^-1     its inverse; libm has none, so it is found by bisection on Phi
  *   Eq. 4 / 12 E[T] ~ sqrt(M sigma^2) ((1-g) Phi^-1(1 - 1/N) + g Phi^-1(1 - 1/(e N))) + M mu,
- *              g the Euler-Mascheroni constant.  Eq. 12 as printed also adds T^c; in this build T
+ *              g the Euler-Mascheroni constant.  Eq. 12 as printed also adds T^c; here T
  *              never contains T^c (the paper adds it separately in Eq. 6, Eq. 11 and Algorithm 2).
  *   Eq. 5 / 10 E[M~(tau)] ~ sum_{m=1..M} Phi((tau - m mu) / sqrt(m sigma^2))
  *   Eq. 11     E[S_eff(tau)] ~ (E[M~]/M) (E[T] + T^c) / (min(tau, E[T]) + T^c)     (numerator as in Eq. 6)

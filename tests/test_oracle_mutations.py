@@ -12,22 +12,25 @@ SRC = os.path.join(os.path.dirname(oracle.__file__), "dc_oracle.c")
 
 # (name, [(old, new, expected_occurrences)])
 MUTANTS = [
-    ("non_strict_compare", [("if (Tin < tau) done += 1;", "if (Tin <= tau) done += 1;", 1),
-                            ("cnt[k] += (Tin < taus[k]) ? 1 : 0;", "cnt[k] += (Tin <= taus[k]) ? 1 : 0;", 1)]),
-    ("last_worker_not_max", [("Ti = fmaxf(Ti, Tin);", "Ti = Tin;", 3)]),
-    ("double_accumulator", [("float Tin = 0.0f;", "double Tin = 0.0;", 3)]),
-    ("no_min_with_tau", [("out_step[i * K + k] = fminf(tau, Ti) + tc;", "out_step[i * K + k] = tau + tc;", 1),
-                         ("(fminf(taus[k], Ti) + tc)", "(taus[k] + tc)", 1)]),
-    ("sync_without_comm", [("out_sync[i] = Ti + tc;", "out_sync[i] = Ti;", 2)]),
-    ("step_without_comm", [("out_step[i * K + k] = fminf(tau, Ti) + tc;", "out_step[i * K + k] = fminf(tau, Ti);", 1),
-                           ("(fminf(taus[k], Ti) + tc)", "(fminf(taus[k], Ti))", 1)]),
-    ("transposed_layout", [("const float *t = lat + (i * N + n) * M;", "const float *t = lat + (i * M + n) * N;", 2)]),
-    ("skips_first_microbatch", [("for (int64_t m = 0; m < M; ++m) {\n                    if (rule == 0) {",
-                                 "for (int64_t m = 1; m < M; ++m) {\n                    if (rule == 0) {", 2)]),
-    ("exclusive_prefix_rule0", [("Tin = Tin + t[m];\n                        if (Tin < tau) done += 1;",
-                                 "if (Tin < tau) done += 1;\n                        Tin = Tin + t[m];", 1),
-                                ("Tin = Tin + t[m];\n                        for (int64_t k = 0; k < K; ++k) cnt[k] += (Tin < taus[k]) ? 1 : 0;",
-                                 "for (int64_t k = 0; k < K; ++k) cnt[k] += (Tin < taus[k]) ? 1 : 0;\n                        Tin = Tin + t[m];", 1)]),
+    ("non_strict_compare", [("completed += (f[m] < tau) ? 1 : 0;", "completed += (f[m] <= tau) ? 1 : 0;", 1),
+                            ("cnt[k] += (elapsed < taus[k]) ? 1 : 0;", "cnt[k] += (elapsed <= taus[k]) ? 1 : 0;", 1)]),
+    ("last_worker_not_max", [("slowest_full = fmaxf(slowest_full, finish[n * M + (M - 1)]);", "slowest_full = finish[n * M + (M - 1)];", 1),
+                             ("slowest_full = fmaxf(slowest_full, elapsed);", "slowest_full = elapsed;", 1)]),
+    ("double_accumulator", [("float elapsed = 0.0f;", "double elapsed = 0.0;", 3)]),
+    ("no_min_with_tau", [("(fminf(tau, slowest_full) + tc)", "(tau + tc)", 1),
+                         ("(fminf(taus[k], slowest_full) + tc)", "(taus[k] + tc)", 1)]),
+    ("sync_without_comm", [("out_sync[i] = slowest_full + tc;", "out_sync[i] = slowest_full;", 2)]),
+    ("step_without_comm", [("(fminf(tau, slowest_full) + tc)", "(fminf(tau, slowest_full))", 1),
+                           ("(fminf(taus[k], slowest_full) + tc)", "(fminf(taus[k], slowest_full))", 1)]),
+    ("transposed_layout", [("const float *row = lat + (i * N + n) * M;", "const float *row = lat + (i * M + n) * N;", 3)]),
+    ("skips_first_microbatch", [("elapsed = elapsed + row[m];\n                finish[n * M + m] = elapsed;",
+                                 "if (m > 0) elapsed = elapsed + row[m];\n                finish[n * M + m] = elapsed;", 1),
+                                ("for (int64_t m = 0; m < M; ++m) {\n                    if (rule == 0) {",
+                                 "for (int64_t m = 1; m < M; ++m) {\n                    if (rule == 0) {", 1)]),
+    ("exclusive_prefix_rule0", [("elapsed = elapsed + row[m];\n                finish[n * M + m] = elapsed;",
+                                 "finish[n * M + m] = elapsed;\n                elapsed = elapsed + row[m];", 1),
+                                ("elapsed = elapsed + row[m];\n                        for (int64_t k = 0; k < K; ++k) cnt[k] += (elapsed < taus[k]) ? 1 : 0;",
+                                 "for (int64_t k = 0; k < K; ++k) cnt[k] += (elapsed < taus[k]) ? 1 : 0;\n                        elapsed = elapsed + row[m];", 1)]),
     ("speedup_forgets_workers", [("(dn / NM)", "(dn / (double)M)", 1)]),
     ("speedup_inverted_ratio", [("((double)sync[i] / st)", "(st / (double)sync[i])", 1)]),
     ("thr_mean_is_ratio_of_means", [("sum_ratio / (double)T", "((double)sum_done / sum_step)", 1)]),
@@ -36,8 +39,13 @@ MUTANTS = [
     ("bailey_weights_swapped", [("(1.0 - g) * dco_phi_inv(1.0 - 1.0 / (double)N) + g * dco_phi_inv(", "g * dco_phi_inv(1.0 - 1.0 / (double)N) + (1.0 - g) * dco_phi_inv(", 1)]),
     ("eq5_variance_not_scaled_by_m", [("sqrt((double)m * sigma * sigma)", "sqrt(sigma * sigma)", 1)]),
     ("eq11_numerator_without_comm", [("* (ET + t_comm) / step", "* ET / step", 1)]),
-    ("rule1_inclusive", [("if (before < taus[k]) {", "if (Tin < taus[k]) {", 1),
-                         ("if (Tin < tau) {\n                            done += 1;", "if (Tin + t[m] < tau) {\n                            done += 1;", 1)]),
+    ("rule1_inclusive", [("const float start = (m == 0) ? 0.0f : f[m - 1];", "const float start = f[m];", 1),
+                         ("if (start < taus[k]) {", "if (elapsed < taus[k]) {", 1)]),
+    ("rule1_time_is_start_of_last", [("last_run >= 0 ? f[last_run] : 0.0f", "last_run > 0 ? f[last_run - 1] : 0.0f", 1),
+                                     ("wlast[k] = elapsed;", "wlast[k] = start;", 1)]),
+    ("rule1_last_worker_not_max", [("slowest_cut = fmaxf(slowest_cut, last_run >= 0 ? f[last_run] : 0.0f);",
+                                    "slowest_cut = last_run >= 0 ? f[last_run] : 0.0f;", 1),
+                                   ("wmax[k] = fmaxf(wmax[k], wlast[k]);", "wmax[k] = wlast[k];", 1)]),
 ]
 
 
@@ -54,7 +62,7 @@ def test_planted_mistake_is_caught(tmp_path, name, edits):
     oracle.build(force=True, source=str(c), out=so)
     lib = oracle.load(so)
     caught = []
-    for order in ("rows", "literal"):
+    for order in ("rows", "definition"):
         missed = True
         for pin in pins.FAST_PINS:
             try:
@@ -64,3 +72,19 @@ def test_planted_mistake_is_caught(tmp_path, name, edits):
                 caught.append((order, pin.__name__))
                 break
         assert not missed, f"no pin noticed mutant {name} in order {order}"
+
+
+def test_swapped_bailey_weights_die_on_the_quadrature_pin(tmp_path):
+    """Eq. 4's two weights exchanged: the pin that notices must be the one that compares with the exact
+    E[max] from Eq. 3's integral, not a retyped copy of the formula."""
+    with open(SRC) as f:
+        src = f.read()
+    old, new, count = dict((m[0], m[1]) for m in MUTANTS)["bailey_weights_swapped"][0]
+    assert src.count(old) == count
+    c = tmp_path / "bailey.c"
+    c.write_text(src.replace(old, new))
+    so = str(tmp_path / "bailey.so")
+    oracle.build(force=True, source=str(c), out=so)
+    with pytest.raises(AssertionError):
+        pins.pin_bailey_against_quadrature(oracle.load(so))
+    pins.pin_bailey_against_quadrature(oracle.load())

@@ -5,9 +5,9 @@ import pytest
 import pins
 
 
-@pytest.mark.parametrize("order", ["rows", "literal"])
+@pytest.mark.parametrize("order", ["rows", "definition"])
 @pytest.mark.parametrize("pin", pins.ALL_PINS, ids=lambda f: f.__name__)
 def test_pin(oracle_lib, pin, order):
-    if pin in (pins.pin_argmax, pins.pin_literal_equals_rows) and order == "literal":
+    if pin in (pins.pin_argmax, pins.pin_definition_equals_rows) and order == "definition":
         pytest.skip("order-independent")
     pin(oracle_lib, order=order)

@@ -332,7 +332,9 @@ def run_ours(args, w: W.Workload):
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "read_only_pass_ms": read_probe_ms, "read_only_pass_gbs": 4 * samples / (read_probe_ms * 1e-3) / 1e9,
                      "sweep_over_read_only_pass": (sim_avg_s * 1e3) / read_probe_ms},
-        "gpu_launches": args.steps * sum(api.launches().values()),
+        "gpu_launches": args.steps * (api.dc_launch_count(api.ENTRY_SIMULATE, T, N, M, K) +
+                                      api.dc_launch_count(api.ENTRY_REDUCE_TRIALS, T, N, M, K) +
+                                      api.dc_launch_count(api.ENTRY_ARGMAX_TAU, T, N, M, K)),
         "clocks": clocks,
     }
 

@@ -13,8 +13,11 @@
  *   latencies[t][n][m] = t_{i,n}^{(m)}: seconds worker n spent on micro-batch m in trial t
  *
  * Every pointer argument says whether it is a DEVICE or a HOST pointer.  The library never
- * allocates or frees device memory, keeps no per-call state, and never synchronises the device
- * unless the function says so: work is enqueued on `stream` (a cudaStream_t passed as void*; NULL
+ * allocates or frees device memory, keeps no per-call state (any number of host threads may call it
+ * at the same time, on the same or different streams and devices; what it caches per device or per
+ * process -- device properties, kernel attributes, the expert settings of dropcompute_dev.h -- is
+ * guarded by locks, and a call works from one consistent copy of the settings taken when it
+ * starts), and never synchronises the device unless the function says so: work is enqueued on `stream` (a cudaStream_t passed as void*; NULL
  * is the default stream) and the call returns.  Buffers belong to the caller and must stay valid
  * until the enqueued work has run.  Outputs are overwritten, never accumulated into.
  *
@@ -252,15 +255,6 @@ int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M,
                   void *workspace, size_t workspace_bytes, void *stream);
 
 /*
- * dc_read_probe — measurement aid with no counterpart in the paper: enqueues a kernel that reads
- * data[0 .. count - count % 4) once with 16-byte loads and does nothing else.  Timed on a latency tensor it gives
- * the duration of a plain read-only pass over those bytes, which benchmarks report beside the sweep's.
- *   data   DEVICE, 16-byte aligned, count floats (all >= 0, as latencies are)
- *   sink   DEVICE, one float; never written for such data
- */
-int dc_read_probe(const float *data, int64_t count, float *sink, void *stream);
-
-/*
  * dc_check_inputs — SYNCHRONOUS check of the data preconditions of dc_simulate on `stream`:
  * returns DC_ERR_LATENCIES if any latency is negative, NaN or infinite or a worker's latencies add up
  * (left to right, in fp32) to infinity, DC_ERR_TAUS if the grid is not non-decreasing or holds a NaN,
@@ -280,50 +274,7 @@ int dc_check_inputs(const float *latencies, int64_t T, int64_t N, int64_t M,
  */
 int dc_device_status(uint32_t *flags_host);
 
-/* Which kernel dc_simulate_ex would use for a shape: 0 = tiled kernel (M a multiple of 4 and a 16-byte aligned
- * pointer), 2 = flat kernel (any other case with M <= 127, or up to DC_TUNE_FLAT_MAX_M: other row lengths, or a
- * pointer that is only 4-byte aligned), 1 = plain-load kernel (such cases with longer rows), negative = -dc_status. */
-int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, int32_t K);
-
-/*
- * dc_tune — expert knob for performance experiments; affects later dc_simulate* calls of this process.
- * Results never depend on it.  value 0 restores the automatic choice.
- *   DC_TUNE_STAGES       depth of the shared-memory ring the tiled kernel streams rows through (2..8)
- *   DC_TUNE_LANE_COPIES  histogram copies a warp spreads its lanes over in the tiled kernel (1, 2, 4 or 8)
- *   DC_TUNE_WARP_GROUPS  groups of warps with histogram copies of their own (1..8)
- *   DC_TUNE_BATCH_LOOKUPS 1 = bin each running sum and update the histogram at once, 2 = look up the bins of a
- *                        whole group of eight first (lower latency, better for trials that fit one tile)
- *   DC_TUNE_BOX_FLOATS   floats of a row fetched per tile (16 or 32; 16 needs M to be a multiple of 16)
- *   DC_TUNE_DIRECT_BINS  1 = always bin through the lookup table, 2 = bin evenly spaced thresholds arithmetically
- *                        (one multiply-add and one comparison per sample, no table read) in the tiled kernel
- *   DC_TUNE_FLAT_MAX_M   longest row (1..255) the flat kernel is given instead of the plain-load kernel (default 127)
- *   DC_TUNE_FLAT_TILE_WARPS, DC_TUNE_FLAT_GROUPS, DC_TUNE_FLAT_DEPTH  flat kernel (row length not a multiple
- *                        of 4): warps per tile (tile = 32 x that many rows), groups of warps working on different
- *                        tiles at once, ring stages per group; used only when all three are set, and a setting
- *                        whose tiles or ring do not fit makes dc_simulate* return DC_ERR_RANGE
- * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
- */
-#define DC_TUNE_STAGES 1
-#define DC_TUNE_LANE_COPIES 2
-#define DC_TUNE_WARP_GROUPS 3
-#define DC_TUNE_BOX_FLOATS 4
-#define DC_TUNE_BATCH_LOOKUPS 5
-#define DC_TUNE_DIRECT_BINS 6
-#define DC_TUNE_FLAT_TILE_WARPS 7
-#define DC_TUNE_FLAT_GROUPS 8
-#define DC_TUNE_FLAT_DEPTH 9
-#define DC_TUNE_FLAT_MAX_M 11
-int dc_tune(int32_t key, int32_t value);
-
-/* Number of kernel launches the last successful call of each entry point enqueues (for accounting). */
-int dc_simulate_launches(void);
-int dc_reduce_trials_launches(void);
-int dc_argmax_tau_launches(void);
-
 const char *dc_status_string(int status);
-
-/* A short tag that changes whenever the sweep kernels change (profiles are filed under it). */
-const char *dc_kernel_version(void);
 
 #ifdef __cplusplus
 }

@@ -1,4 +1,5 @@
-"""Thin Python binding of the C ABI in ``include/dropcompute.h``.
+"""Thin Python binding of the C ABI in ``include/dropcompute.h`` (and of the measurement and tuning aids in
+``include/dropcompute_dev.h``).
 
 Argument marshalling only: every function checks dtype/device/contiguity of the torch tensors it is
 given, passes their device pointers and the current CUDA stream to the library entry point of the
@@ -27,10 +28,10 @@ EXPORTS = (
     "dc_simulate", "dc_simulate_ex", "dc_simulate_tc", "dc_simulate_split_workspace_bytes", "dc_simulate_split",
     "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_reduce_trials_static",
     "dc_argmax_tau", "dc_sweep_device",
-    "dc_closed_form", "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status", "dc_simulate_plan", "dc_read_probe",
-    "dc_simulate_launches", "dc_reduce_trials_launches", "dc_argmax_tau_launches", "dc_status_string", "dc_tune",
-    "dc_kernel_version",
+    "dc_closed_form", "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status",
+    "dc_status_string",
 )
+DEV_EXPORTS = ("dc_simulate_plan", "dc_tune", "dc_launch_count", "dc_read_probe", "dc_kernel_version")
 
 
 class DropComputeError(RuntimeError):
@@ -77,9 +78,9 @@ _lib.dc_status_string.argtypes = [ctypes.c_int]
 _lib.dc_status_string.restype = ctypes.c_char_p
 _lib.dc_kernel_version.argtypes = []
 _lib.dc_kernel_version.restype = ctypes.c_char_p
+_lib.dc_launch_count.argtypes = [_i32, _i64, _i64, _i64, _i32, _i64]
 for _name in ("dc_simulate", "dc_simulate_ex", "dc_reduce_trials", "dc_argmax_tau", "dc_sweep_host", "dc_check_inputs",
-              "dc_device_status", "dc_simulate_plan", "dc_simulate_launches", "dc_reduce_trials_launches",
-              "dc_argmax_tau_launches"):
+              "dc_device_status", "dc_simulate_plan", "dc_launch_count", "dc_sweep_device", "dc_read_probe"):
     getattr(_lib, _name).restype = ctypes.c_int
 
 
@@ -307,9 +308,15 @@ def dc_tune(key: int, value: int) -> None:
     _check(_lib.dc_tune(int(key), int(value)), "dc_tune")
 
 
-def launches() -> dict:
-    return {"dc_simulate": _lib.dc_simulate_launches(), "dc_reduce_trials": _lib.dc_reduce_trials_launches(),
-            "dc_argmax_tau": _lib.dc_argmax_tau_launches()}
+ENTRY_SIMULATE, ENTRY_SIMULATE_SPLIT, ENTRY_REDUCE_TRIALS, ENTRY_ARGMAX_TAU, ENTRY_SWEEP_DEVICE, ENTRY_SWEEP_HOST = range(6)
+
+
+def dc_launch_count(entry_point: int, T: int, N: int, M: int, K: int, chunk_trials: int = 0) -> int:
+    """Kernels one successful call of an entry point enqueues for this shape (``dc_launch_count``)."""
+    n = int(_lib.dc_launch_count(int(entry_point), T, N, M, K, int(chunk_trials)))
+    if n < 0:
+        raise DropComputeError(-n, "dc_launch_count")
+    return n
 
 
 # --- convenience wrapper (allocation + the three calls); still nothing but calls into the library ---------------

@@ -1,6 +1,7 @@
 """Builds libdropcompute.so (the C-ABI library) in-tree with nvcc for sm_100a."""
 from __future__ import annotations
 
+import hashlib
 import os
 import shutil
 import subprocess
@@ -8,7 +9,7 @@ import subprocess
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 SRC = os.path.join(PKG, "csrc", "dropcompute.cu")
-HDR = os.path.join(ROOT, "include", "dropcompute.h")
+HDRS = (os.path.join(ROOT, "include", "dropcompute.h"), os.path.join(ROOT, "include", "dropcompute_dev.h"))
 LIB = os.path.join(PKG, "libdropcompute.so")
 
 NVCC_FLAGS = [
@@ -25,20 +26,35 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found: the CUDA library cannot be built")
 
 
+def _cuda_sources():
+    csrc = os.path.dirname(SRC)
+    return sorted(os.path.join(csrc, f) for f in os.listdir(csrc) if f.endswith((".cu", ".cuh")))
+
+
+def source_hash() -> str:
+    """Hash of the CUDA sources (names and contents), baked into the library as dc_kernel_version(): a profile
+    filed under one hash is never reported for a library built from other kernels."""
+    h = hashlib.sha1()
+    for path in _cuda_sources():
+        h.update(os.path.basename(path).encode())
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
 def is_stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    csrc = os.path.dirname(SRC)
-    parts = [os.path.join(csrc, f) for f in os.listdir(csrc) if f.endswith((".cu", ".cuh"))]
-    return any(os.path.getmtime(f) > t for f in (*parts, HDR, os.path.abspath(__file__)))
+    return any(os.path.getmtime(f) > t for f in (*_cuda_sources(), *HDRS, os.path.abspath(__file__)))
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
     if not force and not is_stale():
         return LIB
     tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", os.path.dirname(SRC), "-o", tmp, SRC]
+    cmd = [_nvcc(), *NVCC_FLAGS, f'-DDC_SOURCE_HASH="{source_hash()}"', "-I", os.path.join(ROOT, "include"),
+           "-I", os.path.dirname(SRC), "-o", tmp, SRC]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

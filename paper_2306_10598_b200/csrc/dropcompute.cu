@@ -40,6 +40,7 @@
 #include <string.h>
 
 #include "dropcompute.h"
+#include "dropcompute_dev.h"
 
 #include "sweep_common.cuh"
 #include "sweep_tiled.cuh"
@@ -58,7 +59,9 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 EncodeTiledFn get_encode_fn()
 {
+    static std::mutex lock;
     static EncodeTiledFn fn = nullptr;
+    std::lock_guard<std::mutex> guard(lock);
     if (fn) return fn;
     void *ptr = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -76,9 +79,11 @@ struct DeviceInfo {
 };
 bool device_info(DeviceInfo *out)
 {
+    static std::mutex lock;
     static DeviceInfo cache[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    std::lock_guard<std::mutex> guard(lock);
     if (cache[dev].sms == 0) {
         int sms = 0, smem = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
@@ -100,17 +105,25 @@ int floor_pow2(int v)
     return p;
 }
 
-int g_tune_stages = 0;       // 0 = automatic
-int g_tune_lane_copies = 0;  // 0 = automatic
-int g_tune_warp_groups = 0;  // 0 = automatic
-int g_tune_box_floats = 0;   // 0 = automatic
-int g_tune_batch = 0;        // 0 = automatic, 1 = off, 2 = on
-int g_tune_direct = 0;       // 0 = automatic (on), 1 = off, 2 = on
-int g_tune_flat_max_m = 0;   // 0 = automatic (kFlatAutoMaxM), else the longest row the flat kernel is given (<= kFlatMaxM)
-int g_tune_flat_tile_warps = 0, g_tune_flat_groups = 0, g_tune_flat_depth = 0;  // flat kernel; all three or none
-int g_last_simulate_launches = 0;
-int g_last_reduce_launches = 0;
-int g_last_argmax_launches = 0;
+// Expert settings (dc_tune).  They are process-wide, but every call works from ONE consistent copy taken under
+// the lock when it starts, so a dc_tune from another host thread can never tear a launch configuration.
+struct Tune {
+    int stages = 0;        // 0 = automatic
+    int lane_copies = 0;   // 0 = automatic
+    int warp_groups = 0;   // 0 = automatic
+    int box_floats = 0;    // 0 = automatic
+    int batch = 0;         // 0 = automatic, 1 = off, 2 = on
+    int direct = 0;        // 0 = automatic (on), 1 = off, 2 = on
+    int flat_max_m = 0;    // 0 = automatic (kFlatAutoMaxM), else the longest row the flat kernel is given (<= kFlatMaxM)
+    int flat_tile_warps = 0, flat_groups = 0, flat_depth = 0;  // flat kernel; all three or none
+};
+std::mutex g_tune_lock;
+Tune g_tune;
+Tune tune_snapshot()
+{
+    std::lock_guard<std::mutex> guard(g_tune_lock);
+    return g_tune;
+}
 
 int validate_simulate(const float *lat, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K,
                       const float *out_step, const int32_t *out_done, int32_t rule)
@@ -127,10 +140,10 @@ int validate_simulate(const float *lat, int64_t T, int64_t N, int64_t M, const f
 }
 
 bool tiled_ok(const float *lat, int64_t M) { return (M % 4 == 0) && ((reinterpret_cast<uintptr_t>(lat) & 15) == 0); }
-bool flat_ok(const float *lat, int64_t M)
+bool flat_ok(const float *lat, int64_t M, const Tune &tune)
 {
     // any 4-byte aligned base; rows beyond kFlatAutoMaxM measured faster in the plain-load kernel
-    return !tiled_ok(lat, M) && M <= (g_tune_flat_max_m > 0 ? g_tune_flat_max_m : kFlatAutoMaxM);
+    return !tiled_ok(lat, M) && M <= (tune.flat_max_m > 0 ? tune.flat_max_m : kFlatAutoMaxM);
 }
 
 template <int RULE, bool BATCH, int NQ>
@@ -201,16 +214,16 @@ int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t
 
 // Shared-memory layout of a block of the staged kernels (tiled and flat): ring depth, histogram copies, table
 // size.  Needs p.stage_bytes, p.chunks and the row-thread count; fills the rest and the dynamic shared bytes.
-int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const DeviceInfo &di, size_t *smem_out,
-                        int stage_cap = 3)
+int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const DeviceInfo &di, const Tune &tune,
+                        size_t *smem_out, int stage_cap = 3)
 {
     p.lut_cells = min(kLutCellsMax, 4 * K);
     // Rows that fit one tile gain from looking up a whole group's bins before touching the histogram (the
     // chains overlap); longer rows measured faster with lookups and updates interleaved.
-    p.batch_lookups = g_tune_batch > 0 ? g_tune_batch - 1 : ((p.chunks == 1 || p.short_launch) ? 1 : 0);
+    p.batch_lookups = tune.batch > 0 ? tune.batch - 1 : ((p.chunks == 1 || p.short_launch) ? 1 : 0);
     // Arithmetic binning of evenly spaced thresholds measured faster wherever a group's bins are computed before
     // its updates (rows of one tile, and the start-before-tau rule), slower for long rows under the paper's rule.
-    p.direct_bins = g_tune_direct > 0 ? g_tune_direct - 1
+    p.direct_bins = tune.direct > 0 ? tune.direct - 1
                                       : ((rule == DC_RULE_START_BEFORE_TAU || p.chunks == 1 || p.short_launch) ? 1 : 0);
     // Shared memory per block: aim at two resident blocks per SM.  Histogram copies: lane l of warp w
     // adds into copy (w % warp_groups) * lane_copies + (l % lane_copies); copies used by one warp start
@@ -226,13 +239,13 @@ int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const 
     // (a ring deeper than three tiles measured slower on every workload, whatever the tile size)
     // (a negative stage_cap fixes the ring depth at -stage_cap: the flat kernel's groups x stages per group)
     const int s_max = stage_cap < 0 ? -stage_cap
-                                    : (g_tune_stages > 0 ? g_tune_stages : min(stage_cap, max(2, kStageBudgetBytes / p.stage_bytes)));
-    const int s_min = stage_cap < 0 ? -stage_cap : (g_tune_stages > 0 ? g_tune_stages : 2);
-    const int lc_first = g_tune_lane_copies > 0 ? g_tune_lane_copies : 4;
-    const int lc_last = g_tune_lane_copies > 0 ? g_tune_lane_copies : 1;
-    const int wg_first = g_tune_warp_groups > 0 ? min(g_tune_warp_groups, ncw) : min(2, ncw);
-    const int wg_last = g_tune_warp_groups > 0 ? wg_first : 1;
-    const bool forced = g_tune_stages > 0 && g_tune_lane_copies > 0 && g_tune_warp_groups > 0;
+                                    : (tune.stages > 0 ? tune.stages : min(stage_cap, max(2, kStageBudgetBytes / p.stage_bytes)));
+    const int s_min = stage_cap < 0 ? -stage_cap : (tune.stages > 0 ? tune.stages : 2);
+    const int lc_first = tune.lane_copies > 0 ? tune.lane_copies : 4;
+    const int lc_last = tune.lane_copies > 0 ? tune.lane_copies : 1;
+    const int wg_first = tune.warp_groups > 0 ? min(tune.warp_groups, ncw) : min(2, ncw);
+    const int wg_last = tune.warp_groups > 0 ? wg_first : 1;
+    const bool forced = tune.stages > 0 && tune.lane_copies > 0 && tune.warp_groups > 0;
     // (when a fixed ring alone is too large for two blocks, the same search runs against one block's limit)
     const size_t ring_min = (size_t)s_min * p.stage_bytes;
     const size_t budget = (stage_cap < 0 && ring_min + 4096 > budget2) ? (size_t)di.max_smem_optin : budget2;
@@ -271,6 +284,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     DeviceInfo di;
     if (!device_info(&di)) return DC_ERR_CUDA;
+    const Tune tune = tune_snapshot();
 
     SweepParams p;
     memset(&p, 0, sizeof(p));
@@ -307,9 +321,9 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         // and their tail: 16-float tiles need fewer registers and less shared memory, so three blocks fit an SM,
         // more loads are in flight from the first microsecond and the last wave is finer.  Measured 5-25 % faster
         // on 0.4 GB inputs of 32- to 128-sample rows, 3-5 % slower on inputs of 2 GB and more.
-        p.short_launch = (g_tune_box_floats == 0 && M >= 32 && M % 16 == 0 &&
+        p.short_launch = (tune.box_floats == 0 && M >= 32 && M % 16 == 0 &&
                           (uint64_t)T * (uint64_t)N * (uint64_t)M * 4ull < (1ull << 30)) ? 1 : 0;
-        if ((g_tune_box_floats == 16 && M % 16 == 0) || p.short_launch) p.bw = 16;
+        if ((tune.box_floats == 16 && M % 16 == 0) || p.short_launch) p.bw = 16;
         p.chunks = (int)((M + p.bw - 1) / p.bw);
         const int last_cols = (int)(M - (int64_t)(p.chunks - 1) * p.bw);
         p.nq_last = last_cols / 4;
@@ -322,7 +336,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         p.stage_bytes = ((p.rows * p.pitch + 1023) / 1024) * 1024;
         size_t smem = 0;
         {
-            const int lrc0 = choose_block_layout(p, row_threads, K, rule, di, &smem);
+            const int lrc0 = choose_block_layout(p, row_threads, K, rule, di, tune, &smem);
             if (lrc0 != DC_OK) return lrc0;
         }
 
@@ -351,11 +365,10 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
             else if (nq <= 4) lrc = launch_tiled<4, 1>(map, p, block, smem, T, di, stream);
             else lrc = launch_tiled<8, 1>(map, p, block, smem, T, di, stream);
         }
-        if (lrc == DC_OK) g_last_simulate_launches = 1;
         return lrc;
     }
 
-    if (flat_ok(lat, M)) {
+    if (flat_ok(lat, M, tune)) {
         // Warps per tile wt: the largest power of two whose tile (32 wt whole rows) stays within 32 KB, no more than
         // the trial has rows for.  Eight: one group, three stages (the tiled kernel's schedule).  Fewer: about six
         // consumer warps in G groups with one stage each (the groups overlap each other; measured best on rows of
@@ -367,11 +380,11 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         const int tiles = (int)((N + (int64_t)best_wt * 32 - 1) / ((int64_t)best_wt * 32));
         int best_g = short_rows ? 1 : min(best_wt >= 4 ? 2 : 6 / best_wt, tiles);
         int best_d = best_g == 1 ? 3 : 1;
-        if (g_tune_flat_tile_warps > 0 && g_tune_flat_groups > 0 && g_tune_flat_depth > 0) {
-            best_wt = g_tune_flat_tile_warps;
+        if (tune.flat_tile_warps > 0 && tune.flat_groups > 0 && tune.flat_depth > 0) {
+            best_wt = tune.flat_tile_warps;
             if ((int64_t)best_wt * 32 > N) best_wt = (int)((N + 31) / 32);
-            best_g = g_tune_flat_groups;
-            best_d = g_tune_flat_depth;
+            best_g = tune.flat_groups;
+            best_d = tune.flat_depth;
             if (best_g * best_wt > 8 || best_g * best_d > kMaxStages) return DC_ERR_RANGE;
         }
         if (best_wt <= 0) return DC_ERR_RANGE;
@@ -385,7 +398,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         p.stage_bytes = (int)((((size_t)p.rows * M * 4 + 32) + 1023) / 1024 * 1024);
         // If the ring and the tables of a large grid do not fit a block's shared memory together, take fewer groups
         // (a single group: three stages, then two).
-        const bool forced_split = g_tune_flat_tile_warps > 0 && g_tune_flat_groups > 0 && g_tune_flat_depth > 0;
+        const bool forced_split = tune.flat_tile_warps > 0 && tune.flat_groups > 0 && tune.flat_depth > 0;
         int groups = min(best_g, p.passes), depth = best_d;
         if (!forced_split && groups == 1) depth = 3;
         size_t smem = 0;
@@ -393,7 +406,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         for (;;) {
             p.flat_groups = groups;
             flat_threads = groups * wt * 32;
-            const int lrc0 = choose_block_layout(p, flat_threads, K, rule, di, &smem, -(groups * depth));
+            const int lrc0 = choose_block_layout(p, flat_threads, K, rule, di, tune, &smem, -(groups * depth));
             if (lrc0 == DC_OK && smem <= (size_t)di.max_smem_optin) break;
             if (forced_split) return DC_ERR_RANGE;
             if (groups > 1) {
@@ -411,7 +424,6 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
             lrc = p.batch_lookups ? launch_flat<0, true>(p, block, smem, T, di, stream) : launch_flat<0, false>(p, block, smem, T, di, stream);
         else
             lrc = launch_flat<1, false>(p, block, smem, T, di, stream);
-        if (lrc == DC_OK) g_last_simulate_launches = 1;
         return lrc;
     }
 
@@ -432,7 +444,6 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
     kernel<<<(unsigned)grid, p.rows, smem, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
-    g_last_simulate_launches = 1;
     return DC_OK;
 }
 
@@ -536,7 +547,6 @@ int dc_simulate_split(const float *latencies, int64_t T, int64_t N, int64_t M, c
     const long long items = (long long)T * K > T ? (long long)T * K : T;
     dc_combine_groups<<<(unsigned)((items + 255) / 256), 256, 0, stream>>>(g_step, g_done, g_sync, T, (int)G, K, out_step, out_done, out_sync);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
-    g_last_simulate_launches = 2;
     return DC_OK;
 }
 
@@ -547,7 +557,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
     if (K > DC_MAX_K || N > INT32_MAX || M > INT32_MAX || N * M > (int64_t)INT32_MAX || T > (int64_t)INT32_MAX)
         return -DC_ERR_RANGE;
     if (reinterpret_cast<uintptr_t>(latencies) & 3) return -DC_ERR_ALIGN;
-    return tiled_ok(latencies, M) ? 0 : (flat_ok(latencies, M) ? 2 : 1);
+    return tiled_ok(latencies, M) ? 0 : (flat_ok(latencies, M, tune_snapshot()) ? 2 : 1);
 }
 
 size_t dc_reduce_workspace_bytes(int64_t T, int32_t K)
@@ -562,7 +572,7 @@ int dc_reduce_trials(const float *out_step, const int32_t *out_done, const float
 {
     if (!out_step || !out_done || !stats || !baseline) return DC_ERR_NULL;
     if (T <= 0 || K <= 0 || N <= 0 || M <= 0) return DC_ERR_SHAPE;
-    if (K > DC_MAX_K || N * M > (int64_t)INT32_MAX) return DC_ERR_RANGE;
+    if (K > DC_MAX_K || N > INT32_MAX || M > INT32_MAX || N * M > (int64_t)INT32_MAX) return DC_ERR_RANGE;
     if ((reinterpret_cast<uintptr_t>(stats) & 7) || (reinterpret_cast<uintptr_t>(baseline) & 7)) return DC_ERR_ALIGN;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 7) || workspace_bytes < dc_reduce_workspace_bytes(T, K))
         return DC_ERR_WORKSPACE;
@@ -575,7 +585,6 @@ int dc_reduce_trials(const float *out_step, const int32_t *out_done, const float
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     dc_reduce_final<<<(unsigned)((K + 31) / 32), kRedWarps * 32, 0, stream>>>(ws, T, K, NM, r.chunks, stats, baseline);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
-    g_last_reduce_launches = 2;
     return DC_OK;
 }
 
@@ -584,7 +593,7 @@ int dc_reduce_trials_static(const float *out_step, const int32_t *out_done, cons
 {
     if (!out_step || !out_done || !stats || !baseline) return DC_ERR_NULL;
     if (T <= 0 || K <= 0 || N <= 0 || M <= 0) return DC_ERR_SHAPE;
-    if (K > DC_STATIC_MAX_K || N * M > (int64_t)INT32_MAX) return DC_ERR_RANGE;
+    if (K > DC_STATIC_MAX_K || N > INT32_MAX || M > INT32_MAX || N * M > (int64_t)INT32_MAX) return DC_ERR_RANGE;
     if ((reinterpret_cast<uintptr_t>(stats) & 7) || (reinterpret_cast<uintptr_t>(baseline) & 7)) return DC_ERR_ALIGN;
     // Device address of the built-in scratch, looked up once per device with that device current.
     static std::mutex lock;
@@ -623,7 +632,6 @@ int dc_argmax_tau(const double *stats, const float *taus, int32_t K, int32_t obj
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     dc_argmax_kernel<<<1, 32, 0, stream>>>(stats + (size_t)objective * K, taus, K, out_k, out_tau, out_value);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
-    g_last_argmax_launches = 1;
     return DC_OK;
 }
 
@@ -783,8 +791,13 @@ int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M, 
         DC_TRY(cudaEventCreateWithFlags(&ready[i], cudaEventDisableTiming));
         DC_TRY(cudaEventCreateWithFlags(&freed[i], cudaEventDisableTiming));
     }
+    // The private copy stream starts after everything the caller has enqueued on `stream` so far (which may
+    // still be using the workspace).
+    cudaEvent_t entered = nullptr;
+    DC_TRY(cudaEventCreateWithFlags(&entered, cudaEventDisableTiming));
+    DC_TRY(cudaEventRecord(entered, stream));
+    DC_TRY(cudaStreamWaitEvent(copy_stream, entered, 0));
     DC_TRY(cudaMemcpyAsync(d_taus, taus_host, (size_t)K * 4, cudaMemcpyHostToDevice, stream));
-    int launches = 0;
     const int64_t nchunks = (T + chunk_trials - 1) / chunk_trials;
     for (int64_t c = 0; c < nchunks && !cuda_fail && rc == DC_OK; ++c) {
         const int b = (int)(c & 1);
@@ -798,7 +811,6 @@ int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M, 
         if (!cuda_fail) {
             rc = simulate_impl(buf[b], tn, N, M, d_taus, K, t_comm, nullptr, d_step + (size_t)t0 * K, d_done + (size_t)t0 * K,
                                d_sync + t0, rule, stream);
-            launches += 1;
         }
         DC_TRY(cudaEventRecord(freed[b], stream));
     }
@@ -819,62 +831,86 @@ int dc_sweep_host(const float *latencies_host, int64_t T, int64_t N, int64_t M, 
         if (ready[i]) cudaEventDestroy(ready[i]);
         if (freed[i]) cudaEventDestroy(freed[i]);
     }
+    if (entered) cudaEventDestroy(entered);
     if (copy_stream) cudaStreamDestroy(copy_stream);
     if (cuda_fail) return DC_ERR_CUDA;
-    if (rc == DC_OK) g_last_simulate_launches = launches;
     return rc;
 }
 
 int dc_tune(int32_t key, int32_t value)
 {
+    std::lock_guard<std::mutex> guard(g_tune_lock);
+    Tune &tune = g_tune;
     if (key == DC_TUNE_STAGES && (value == 0 || (value >= 2 && value <= kMaxStages))) {
-        g_tune_stages = value;
+        tune.stages = value;
         return DC_OK;
     }
     if (key == DC_TUNE_LANE_COPIES && (value == 0 || value == 1 || value == 2 || value == 4 || value == 8)) {
-        g_tune_lane_copies = value;
+        tune.lane_copies = value;
         return DC_OK;
     }
     if (key == DC_TUNE_WARP_GROUPS && value >= 0 && value <= 8) {
-        g_tune_warp_groups = value;
+        tune.warp_groups = value;
         return DC_OK;
     }
     if (key == DC_TUNE_BATCH_LOOKUPS && value >= 0 && value <= 2) {
-        g_tune_batch = value;
+        tune.batch = value;
         return DC_OK;
     }
     if (key == DC_TUNE_FLAT_MAX_M && value >= 0 && value <= kFlatMaxM) {
-        g_tune_flat_max_m = value;
+        tune.flat_max_m = value;
         return DC_OK;
     }
     if (key == DC_TUNE_FLAT_TILE_WARPS && value >= 0 && value <= 8) {
-        g_tune_flat_tile_warps = value;
+        tune.flat_tile_warps = value;
         return DC_OK;
     }
     if (key == DC_TUNE_FLAT_GROUPS && value >= 0 && value <= 8) {
-        g_tune_flat_groups = value;
+        tune.flat_groups = value;
         return DC_OK;
     }
     if (key == DC_TUNE_FLAT_DEPTH && value >= 0 && value <= 4) {
-        g_tune_flat_depth = value;
+        tune.flat_depth = value;
         return DC_OK;
     }
     if (key == DC_TUNE_DIRECT_BINS && value >= 0 && value <= 2) {
-        g_tune_direct = value;
+        tune.direct = value;
         return DC_OK;
     }
     if (key == DC_TUNE_BOX_FLOATS && (value == 0 || value == 16 || value == 32)) {
-        g_tune_box_floats = value;
+        tune.box_floats = value;
         return DC_OK;
     }
     return DC_ERR_UNSUPPORTED;
 }
 
-int dc_simulate_launches(void) { return g_last_simulate_launches; }
-int dc_reduce_trials_launches(void) { return g_last_reduce_launches; }
-int dc_argmax_tau_launches(void) { return g_last_argmax_launches; }
+int dc_launch_count(int32_t entry_point, int64_t T, int64_t N, int64_t M, int32_t K, int64_t chunk_trials)
+{
+    if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return -DC_ERR_SHAPE;
+    switch (entry_point) {
+    case DC_ENTRY_SIMULATE: return 1;
+    case DC_ENTRY_SIMULATE_SPLIT: {
+        DeviceInfo di;
+        if (!device_info(&di)) return -DC_ERR_CUDA;
+        return split_groups(T, N, di.sms) > 1 ? 2 : 1;
+    }
+    case DC_ENTRY_REDUCE_TRIALS: return 2;
+    case DC_ENTRY_ARGMAX_TAU: return 1;
+    case DC_ENTRY_SWEEP_DEVICE: return 4;
+    case DC_ENTRY_SWEEP_HOST: {
+        if (chunk_trials <= 0) return -DC_ERR_SHAPE;
+        if (chunk_trials > T) chunk_trials = T;
+        const int64_t nchunks = (T + chunk_trials - 1) / chunk_trials;
+        return nchunks + 3 > (int64_t)INT32_MAX ? -DC_ERR_RANGE : (int)(nchunks + 3);
+    }
+    default: return -DC_ERR_UNSUPPORTED;
+    }
+}
 
-const char *dc_kernel_version(void) { return "sweep-tiled-13"; }
+#ifndef DC_SOURCE_HASH
+#define DC_SOURCE_HASH "unhashed"
+#endif
+const char *dc_kernel_version(void) { return "sweep-" DC_SOURCE_HASH; }
 
 const char *dc_status_string(int status)
 {

@@ -746,3 +746,61 @@ def test_split_entry_point_matches(api, T, N, M, K):
             api.dc_simulate_split(lat_d, taus_d, 0.02, step, done, sync, None, 0)
         assert e.value.status == 9
     api.dc_device_status()
+
+
+def test_two_host_threads_on_two_streams(api):
+    """Two host threads, each with a stream of its own, sweep different inputs at the same time while the main
+    thread keeps changing the expert settings: every result must carry the oracle's bits (the library keeps no
+    per-call state and every call works from one consistent copy of the settings)."""
+    import threading
+    cases = [(40, 200, 32, 64, 0), (25, 300, 36, 40, 1)]
+    inputs, refs = [], []
+    for i, (T, N, M, K, rule) in enumerate(cases):
+        lat = W.iid_latencies("shifted_exp", T, N, M, seed=1200 + i, shift=0.01, mean=0.02).numpy()
+        taus = grid_for(lat, K, seed=50 + i)
+        inputs.append((torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()))
+        refs.append(oracle.sweep(lat, taus, 0.11, rule=rule))
+    torch.cuda.synchronize()
+    errors = []
+
+    def worker(i):
+        try:
+            T, N, M, K, rule = cases[i]
+            lat_d, taus_d = inputs[i]
+            stream = torch.cuda.Stream()
+            step = torch.empty((T, K), dtype=torch.float32, device="cuda")
+            done = torch.empty((T, K), dtype=torch.int32, device="cuda")
+            sync = torch.empty((T,), dtype=torch.float32, device="cuda")
+            with torch.cuda.stream(stream):
+                for _ in range(40):
+                    step.fill_(-1.0)
+                    done.fill_(-1)
+                    api.dc_simulate_ex(lat_d, taus_d, 0.11, step, done, sync, rule)
+                    stream.synchronize()
+                    ok = (np.array_equal(done.cpu().numpy(), refs[i].done)
+                          and np.array_equal(step.cpu().numpy().view(np.uint32), refs[i].step.view(np.uint32))
+                          and np.array_equal(sync.cpu().numpy().view(np.uint32), refs[i].sync.view(np.uint32)))
+                    if not ok:
+                        errors.append((i, "bits differ"))
+                        return
+        except Exception as e:  # noqa: BLE001 - reported by the main thread
+            errors.append((i, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(len(cases))]
+    for t in threads:
+        t.start()
+    try:
+        n = 0
+        while any(t.is_alive() for t in threads):
+            api.dc_tune(api.TUNE_STAGES, (0, 2, 3)[n % 3])
+            api.dc_tune(api.TUNE_LANE_COPIES, (0, 1, 2, 4)[n % 4])
+            api.dc_tune(api.TUNE_DIRECT_BINS, n % 3)
+            n += 1
+    finally:
+        for t in threads:
+            t.join()
+        api.dc_tune(api.TUNE_STAGES, 0)
+        api.dc_tune(api.TUNE_LANE_COPIES, 0)
+        api.dc_tune(api.TUNE_DIRECT_BINS, 0)
+    assert not errors, errors
+    api.dc_device_status()

@@ -8,6 +8,7 @@ import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 HEADER = os.path.join(ROOT, "include", "dropcompute.h")
+DEV_HEADER = os.path.join(ROOT, "include", "dropcompute_dev.h")
 
 
 @pytest.fixture(scope="module")
@@ -18,8 +19,8 @@ def lib():
     return api._lib
 
 
-def declared_functions():
-    with open(HEADER) as f:
+def declared_functions(header=HEADER):
+    with open(header) as f:
         text = f.read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     names = re.findall(r"\b(dc_[a-z_0-9]+)\s*\(", text)
@@ -33,6 +34,13 @@ def test_header_functions_are_exported(lib):
         assert hasattr(lib, n), f"{n} is declared in dropcompute.h but not exported"
     from paper_2306_10598_b200 import api
     assert sorted(api.EXPORTS) == names, "the Python binding must list exactly the header's functions"
+    # the measurement and tuning aids live in a header of their own, outside the product interface
+    dev = declared_functions(DEV_HEADER)
+    assert sorted(api.DEV_EXPORTS) == dev and not set(dev) & set(names)
+    for n in dev:
+        assert hasattr(lib, n), f"{n} is declared in dropcompute_dev.h but not exported"
+    for n in ("dc_tune", "dc_read_probe", "dc_kernel_version", "dc_launch_count"):
+        assert n in dev and n not in names
 
 
 def test_argument_errors_need_no_gpu(lib):
@@ -81,6 +89,62 @@ def test_argument_errors_need_no_gpu(lib):
     for key in (1, 2, 3, 4, 5):
         assert lib.dc_tune(key, 0) == 0
     assert lib.dc_kernel_version().startswith(b"sweep-")
+    from paper_2306_10598_b200 import build
+    assert lib.dc_kernel_version() == b"sweep-" + build.source_hash().encode()   # the tag follows the sources
+    # sizes that would overflow N*M are refused, not multiplied
+    assert lib.dc_reduce_trials(A, A, A, 4, 4, 1 << 62, 1 << 62, A, A, A, 1 << 20, None) == 4
+    assert lib.dc_reduce_trials_static(A, A, A, 4, 4, 1 << 62, 4, A, A, None) == 4
+    # launch counts are a pure function of the shape
+    assert lib.dc_launch_count(0, 5, 5, 5, 5, 0) == 1 and lib.dc_launch_count(2, 5, 5, 5, 5, 0) == 2
+    assert lib.dc_launch_count(3, 5, 5, 5, 5, 0) == 1 and lib.dc_launch_count(4, 5, 5, 5, 5, 0) == 4
+    assert lib.dc_launch_count(5, 10, 5, 5, 5, 3) == 4 + 3 and lib.dc_launch_count(5, 10, 5, 5, 5, 0) == -2
+    assert lib.dc_launch_count(9, 5, 5, 5, 5, 0) == -7 and lib.dc_launch_count(0, 0, 5, 5, 5, 0) == -2
+
+
+def test_two_host_threads_and_the_tuning_knobs(lib):
+    """The library is called from two host threads at once while a third keeps changing the expert settings:
+    every call must come back with the status its own arguments deserve (argument errors need no GPU; with valid
+    arguments a call ends with DC_ERR_CUDA on a machine without a GPU and DC_OK on one with)."""
+    import threading
+    A = 0x10000
+    f = ctypes.c_float(0.1)
+    stop = threading.Event()
+    bad = []
+
+    def tuner():
+        i = 0
+        while not stop.is_set():
+            for key, vals in ((1, (0, 2, 3, 4)), (2, (0, 1, 2, 4)), (3, (0, 1, 2)), (5, (0, 1, 2)), (6, (0, 1, 2)), (11, (0, 200))):
+                if lib.dc_tune(key, vals[i % len(vals)]) != 0:
+                    bad.append(("tune", key))
+            if lib.dc_tune(99, 0) != 7:
+                bad.append(("tune", 99))
+            i += 1
+
+    def caller(seed):
+        for i in range(3000):
+            j = (i + seed) % 5
+            if j == 0 and lib.dc_simulate(None, 1, 1, 1, A, 1, f, A, A, None) != 1:
+                bad.append(("null", i))
+            if j == 1 and lib.dc_simulate(A, 1, 1, 1, A, 4097, f, A, A, None) != 4:
+                bad.append(("range", i))
+            if j == 2 and lib.dc_simulate_ex(A, 1, 1, 1, A, 1, f, A, A, None, 5, None) != 7:
+                bad.append(("rule", i))
+            if j == 3 and lib.dc_simulate_plan(A, 4, 8, 129 + (i % 2) * 72, 3) not in (1, 2):
+                bad.append(("plan", i))
+            if j == 4 and lib.dc_reduce_trials(A, A, A, 100, 8, 1, 1, A, A, A, 8, None) != 9:
+                bad.append(("workspace", i))
+
+    threads = [threading.Thread(target=tuner)] + [threading.Thread(target=caller, args=(s,)) for s in (0, 2)]
+    for t in threads:
+        t.start()
+    for t in threads[1:]:
+        t.join()
+    stop.set()
+    threads[0].join()
+    for key in (1, 2, 3, 5, 6, 11):
+        assert lib.dc_tune(key, 0) == 0
+    assert not bad, bad[:5]
 
 
 def test_workspace_sizes(lib):

@@ -38,6 +38,10 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  *                        of 4): warps per tile (tile = 32 x that many rows), groups of warps working on different
  *                        tiles at once, ring stages per group; used only when all three are set, and a setting
  *                        whose tiles or ring do not fit makes dc_simulate* return DC_ERR_RANGE
+ *   DC_TUNE_LEAN_LOOP    1 = always the general consumer loop, 2 (and 0) = the short loop wherever every chunk of a
+ *                        row is full (tiled kernel)
+ *   DC_TUNE_TILE_TRIALS  the most trials of few workers (N <= 128) that may share one tile of the tiled kernel
+ *                        (1 = one trial per tile)
  * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
  */
 #define DC_TUNE_STAGES 1
@@ -50,6 +54,8 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
 #define DC_TUNE_FLAT_GROUPS 8
 #define DC_TUNE_FLAT_DEPTH 9
 #define DC_TUNE_FLAT_MAX_M 11
+#define DC_TUNE_LEAN_LOOP 12
+#define DC_TUNE_TILE_TRIALS 13
 int dc_tune(int32_t key, int32_t value);
 
 /*

@@ -98,6 +98,18 @@ bool device_info(DeviceInfo *out)
     return true;
 }
 
+// Blocks for `units` equal pieces of work (trials, or tiles of several trials) that the blocks take round-robin:
+// no more than `resident` (what fits the GPU at once), and of those the FEWEST that still finish in the same number
+// of rounds.  The last round then has no idle blocks to wait for, and a bandwidth-bound kernel loses nothing by
+// running on a few blocks less (4096 trials on 444 resident blocks: ten rounds either way; 410 blocks all work
+// through all ten, whereas with 444 blocks 344 of them sit out the tenth).
+long long even_grid(long long units, long long resident)
+{
+    if (units <= resident) return units;
+    const long long rounds = (units + resident - 1) / resident;
+    return (units + rounds - 1) / rounds;
+}
+
 int floor_pow2(int v)
 {
     int p = 1;
@@ -116,6 +128,8 @@ struct Tune {
     int direct = 0;        // 0 = automatic (on), 1 = off, 2 = on
     int flat_max_m = 0;    // 0 = automatic (kFlatAutoMaxM), else the longest row the flat kernel is given (<= kFlatMaxM)
     int flat_tile_warps = 0, flat_groups = 0, flat_depth = 0;  // flat kernel; all three or none
+    int lean = 0;          // 0 = automatic (on), 1 = off, 2 = on: the short consumer loop for rows of full chunks
+    int tile_trials = 0;   // 0 = automatic, else the most trials of few workers that share a tile
 };
 std::mutex g_tune_lock;
 Tune g_tune;
@@ -153,7 +167,7 @@ int launch_flat_q(const SweepParams &p, int block, size_t smem, long long T, con
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
-    const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
+    const long long grid = even_grid(T, (long long)occ * di.sms);
     kernel<<<(unsigned)grid, block, smem, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
@@ -196,7 +210,7 @@ int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size
             last[dev].occ = occ;
         }
     }
-    const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
+    const long long grid = even_grid(T, (long long)occ * di.sms);
     kernel<<<(unsigned)grid, block, smem, stream>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
@@ -229,6 +243,7 @@ int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const 
     // adds into copy (w % warp_groups) * lane_copies + (l % lane_copies); copies used by one warp start
     // 32 / lane_copies banks apart so that equal bins of different lanes do not collide.
     p.nbuf = 2;
+    p.spare = 1;
     const int ncw = row_threads / 32;
     const size_t budget2 = (size_t)di.smem_per_sm / 2 - 1024 - 256;  // two blocks per SM
     size_t smem = 0;
@@ -241,9 +256,12 @@ int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const 
     const int s_max = stage_cap < 0 ? -stage_cap
                                     : (tune.stages > 0 ? tune.stages : min(stage_cap, max(2, kStageBudgetBytes / p.stage_bytes)));
     const int s_min = stage_cap < 0 ? -stage_cap : (tune.stages > 0 ? tune.stages : 2);
-    const int lc_first = tune.lane_copies > 0 ? tune.lane_copies : 4;
+    // Several small trials per tile: the fewer workers a trial has, the more trials a warp's lanes are spread over
+    // and the fewer histogram copies per trial are worth their shared memory.
+    const int lc_auto = p.g > 1 ? (p.N >= 32 ? 4 : (p.N >= 16 ? 2 : 1)) : 4;
+    const int lc_first = tune.lane_copies > 0 ? tune.lane_copies : lc_auto;
     const int lc_last = tune.lane_copies > 0 ? tune.lane_copies : 1;
-    const int wg_first = tune.warp_groups > 0 ? min(tune.warp_groups, ncw) : min(2, ncw);
+    const int wg_first = tune.warp_groups > 0 ? min(tune.warp_groups, ncw) : (p.g > 1 ? 1 : min(2, ncw));
     const int wg_last = tune.warp_groups > 0 ? wg_first : 1;
     const bool forced = tune.stages > 0 && tune.lane_copies > 0 && tune.warp_groups > 0;
     // (when a fixed ring alone is too large for two blocks, the same search runs against one block's limit)
@@ -261,9 +279,13 @@ int choose_block_layout(SweepParams &p, int row_threads, int K, int rule, const 
                 p.hist_stride = (K + 2 + 3) & ~3;  // a multiple of 4: copies start 16-byte aligned
                 while (lc > 1 && p.hist_stride % 32 != want % 32) ++p.hist_stride;
                 smem = 1024 + 2 * kMaxStages * sizeof(uint64_t) + (size_t)st * p.stage_bytes +
-                       tail_bytes(K, p.nbuf * p.hist_copies, p.hist_stride, p.lut_cells, p.nbuf * p.aux_copies);
+                       tail_bytes(K, hist_slots(p), p.hist_stride, p.lut_cells, fmax_slots(p), p.nbuf * p.g);
                 p.epi_vec = (K % 4 == 0) && ((reinterpret_cast<uintptr_t>(p.out_step) & 15) == 0) &&
                             ((reinterpret_cast<uintptr_t>(p.out_done) & 15) == 0);
+                // Several small trials per tile: when K/4 is a power of two up to 32 the epilogue warp takes 32/(K/4)
+                // trials at once.
+                p.epi_sub = 0;
+                if (p.g > 1 && p.epi_vec && K <= 128 && ((K / 4) & (K / 4 - 1)) == 0) p.epi_sub = K / 4;
                 const bool smallest = (st == s_min && lc == lc_last && wg == wg_last);
                 if (smem <= budget || smallest || forced) fits = true;
             }
@@ -309,6 +331,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.lut_cells = 0;
     p.one = 1;
     p.nbuf = 1;
+    p.g = 1;
     p.batch_lookups = 0;
     p.rule = rule;
     p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? p.hist_copies : 0;
@@ -316,7 +339,17 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     if (tiled_ok(lat, M)) {
         EncodeTiledFn encode = get_encode_fn();
         if (!encode) return DC_ERR_CUDA;
+        // Chunk length (floats of a row per box).  Rows all of whose chunks are full take the short consumer loop,
+        // so a row length that 32 does not divide is cut into equal chunks of 12, 16 or 24 floats when that works.
         p.bw = (int)(M < 32 ? M : 32);
+        if (M > 32 && M % 32 != 0) {
+            for (int cand : {24, 16, 12}) {
+                if (M % cand == 0) {
+                    p.bw = cand;
+                    break;
+                }
+            }
+        }
         // Launches of well under a second's worth of bandwidth (below 1 GiB of latencies) are shaped by their start
         // and their tail: 16-float tiles need fewer registers and less shared memory, so three blocks fit an SM,
         // more loads are in flight from the first microsecond and the last wave is finer.  Measured 5-25 % faster
@@ -324,10 +357,32 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         p.short_launch = (tune.box_floats == 0 && M >= 32 && M % 16 == 0 &&
                           (uint64_t)T * (uint64_t)N * (uint64_t)M * 4ull < (1ull << 30)) ? 1 : 0;
         if ((tune.box_floats == 16 && M % 16 == 0) || p.short_launch) p.bw = 16;
+        if (tune.box_floats == 32) p.bw = (int)(M < 32 ? M : 32);
         p.chunks = (int)((M + p.bw - 1) / p.bw);
         const int last_cols = (int)(M - (int64_t)(p.chunks - 1) * p.bw);
         p.nq_last = last_cols / 4;
         p.pitch = p.bw * 4;
+        const int nq = p.bw / 4;
+        // the kernel is compiled for 1, 2, 3, 4, 6 and 8 quads per chunk; other chunk lengths run in the next size up
+        const int nq_inst = nq <= 4 ? nq : (nq <= 6 ? 6 : 8);
+        p.lean = (tune.lean != 1 && last_cols == p.bw && nq == nq_inst) ? 1 : 0;
+        // Several whole trials of few workers share a tile: g trials of N rows each, g N <= 256, as many as it takes
+        // to give every resident block about one tile, within what the histograms of g trials may take.
+        if (N <= kMaxRowsPerPass / 2) {
+            int64_t gmax = kMaxRowsPerPass / N;
+            const int64_t hist_cap = (int64_t)kHistBudgetBytes / (2 * 4 * (int64_t)(K + 8));
+            if (gmax > hist_cap) gmax = hist_cap;
+            if (tune.tile_trials > 0 && gmax > tune.tile_trials) gmax = tune.tile_trials;
+            int64_t g = (T + 2 * (int64_t)di.sms - 1) / (2 * (int64_t)di.sms);
+            if (g > gmax) g = gmax;
+            if (g < 1) g = 1;
+            if (g > 1) {
+                p.g = (int)g;
+                p.passes = 1;
+                p.rows = (int)(g * N);
+            }
+        }
+        const int row_threads_t = ((p.rows + 31) / 32) * 32;
         CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_NONE;
         p.swz_mask = 0;
         if (p.pitch == 128) { swz = CU_TENSOR_MAP_SWIZZLE_128B; p.swz_mask = 7; }
@@ -336,14 +391,14 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         p.stage_bytes = ((p.rows * p.pitch + 1023) / 1024) * 1024;
         size_t smem = 0;
         {
-            const int lrc0 = choose_block_layout(p, row_threads, K, rule, di, tune, &smem);
+            const int lrc0 = choose_block_layout(p, row_threads_t, K, rule, di, tune, &smem);
             if (lrc0 != DC_OK) return lrc0;
         }
 
         CUtensorMap map;
         const cuuint64_t gdim[3] = {(cuuint64_t)M, (cuuint64_t)N, (cuuint64_t)T};
         const cuuint64_t gstride[2] = {(cuuint64_t)M * 4, (cuuint64_t)N * (cuuint64_t)M * 4};
-        const cuuint32_t box[3] = {(cuuint32_t)p.bw, (cuuint32_t)p.rows, 1};
+        const cuuint32_t box[3] = {(cuuint32_t)p.bw, (cuuint32_t)(p.g > 1 ? N : p.rows), (cuuint32_t)p.g};
         const cuuint32_t estr[3] = {1, 1, 1};
         if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(lat), gdim, gstride, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -351,19 +406,27 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
             return DC_ERR_CUDA;
 
         if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
-        const int block = row_threads + 64;
-        const int nq = p.bw / 4;
+        const int block = row_threads_t + 64;
+        const long long tiles = (T + p.g - 1) / p.g;
         int lrc;
         if (rule == DC_RULE_FINISH_BEFORE_TAU) {
-            if (nq <= 1) lrc = launch_tiled<1, 0>(map, p, block, smem, T, di, stream);
-            else if (nq <= 2) lrc = launch_tiled<2, 0>(map, p, block, smem, T, di, stream);
-            else if (nq <= 4) lrc = launch_tiled<4, 0>(map, p, block, smem, T, di, stream);
-            else lrc = launch_tiled<8, 0>(map, p, block, smem, T, di, stream);
+            switch (nq_inst) {
+            case 1: lrc = launch_tiled<1, 0>(map, p, block, smem, tiles, di, stream); break;
+            case 2: lrc = launch_tiled<2, 0>(map, p, block, smem, tiles, di, stream); break;
+            case 3: lrc = launch_tiled<3, 0>(map, p, block, smem, tiles, di, stream); break;
+            case 4: lrc = launch_tiled<4, 0>(map, p, block, smem, tiles, di, stream); break;
+            case 6: lrc = launch_tiled<6, 0>(map, p, block, smem, tiles, di, stream); break;
+            default: lrc = launch_tiled<8, 0>(map, p, block, smem, tiles, di, stream); break;
+            }
         } else {
-            if (nq <= 1) lrc = launch_tiled<1, 1>(map, p, block, smem, T, di, stream);
-            else if (nq <= 2) lrc = launch_tiled<2, 1>(map, p, block, smem, T, di, stream);
-            else if (nq <= 4) lrc = launch_tiled<4, 1>(map, p, block, smem, T, di, stream);
-            else lrc = launch_tiled<8, 1>(map, p, block, smem, T, di, stream);
+            switch (nq_inst) {
+            case 1: lrc = launch_tiled<1, 1>(map, p, block, smem, tiles, di, stream); break;
+            case 2: lrc = launch_tiled<2, 1>(map, p, block, smem, tiles, di, stream); break;
+            case 3: lrc = launch_tiled<3, 1>(map, p, block, smem, tiles, di, stream); break;
+            case 4: lrc = launch_tiled<4, 1>(map, p, block, smem, tiles, di, stream); break;
+            case 6: lrc = launch_tiled<6, 1>(map, p, block, smem, tiles, di, stream); break;
+            default: lrc = launch_tiled<8, 1>(map, p, block, smem, tiles, di, stream); break;
+            }
         }
         return lrc;
     }
@@ -435,13 +498,13 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? p.hist_copies : 0;
     p.lut_cells = min(kLutCellsMax, 4 * K);
     const size_t smem = (size_t)(row_threads / 32) * kPlainTileFloats * sizeof(float) +
-                        tail_bytes(K, p.hist_copies, p.hist_stride, p.lut_cells, p.aux_copies);
+                        tail_bytes(K, hist_slots(p), p.hist_stride, p.lut_cells, fmax_slots(p), p.nbuf * p.g);
     if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
     auto kernel = rule == DC_RULE_FINISH_BEFORE_TAU ? dc_sweep_plain<0> : dc_sweep_plain<1>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, p.rows, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
-    const long long grid = (T < (long long)occ * di.sms) ? T : (long long)occ * di.sms;
+    const long long grid = even_grid(T, (long long)occ * di.sms);
     kernel<<<(unsigned)grid, p.rows, smem, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return DC_ERR_CUDA;
     return DC_OK;
@@ -879,6 +942,14 @@ int dc_tune(int32_t key, int32_t value)
     }
     if (key == DC_TUNE_BOX_FLOATS && (value == 0 || value == 16 || value == 32)) {
         tune.box_floats = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_LEAN_LOOP && value >= 0 && value <= 2) {
+        tune.lean = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_TILE_TRIALS && value >= 0 && value <= kMaxRowsPerPass) {
+        tune.tile_trials = value;
         return DC_OK;
     }
     return DC_ERR_UNSUPPORTED;

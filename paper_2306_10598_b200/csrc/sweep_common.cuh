@@ -12,7 +12,8 @@ constexpr int kMaxRowsPerPass = 256;          // rows (threads) of one trial han
 constexpr int kMaxStages = 8;
 constexpr int kStageBudgetBytes = 96 * 1024;  // shared memory spent on the ring of stages per block
 constexpr int kHistBudgetBytes = 32 * 1024;   // shared memory spent on per-warp histograms per block
-constexpr uint32_t kWaitLimit = 1u << 22;     // polls of one mbarrier wait before giving up (roughly a second)
+constexpr uint32_t kWaitHintNs = 10000;       // longest one try of an mbarrier wait may keep the thread parked
+constexpr uint32_t kWaitLimit = 1u << 20;     // tries of one mbarrier wait before giving up (a fraction of a second to a few seconds)
 constexpr int kReduceChunksMax = 64;          // partial sums per threshold in dc_reduce_trials
 constexpr int kConsumerBarrier = 1;           // named barrier used by the consumer warps
 constexpr int kFlatMaxM = 255;                // longest row the flat kernel can take (32 rows of it fill a 32 KB stage)
@@ -59,7 +60,16 @@ struct SweepParams {
     int short_launch;  // host only: under 1 GiB of latencies (see simulate_impl)
     int epi_vec;       // staged kernels: the epilogue warp may take four bins per lane with 16-byte accesses
                        // (K a multiple of 4, out_step / out_done 16-byte aligned, hist_stride a multiple of 4)
+    int g;             // staged kernels: trials per tile (several whole trials of few workers share a tile; else 1)
+    int epi_sub;       // tiled kernel, g > 1: lanes of the epilogue warp per trial (K/4, a power of two), or 0 for one
+                       // trial at a time
+    int lean;          // tiled kernel: 1 = every chunk of a row is full, so the short form of the consumer loop applies
+    int spare;         // 1 = one more histogram copy (and finish-time copy) after the real ones, which nothing reads:
+                       // lanes without a row of their own add there
 };
+// copies of one trial's histogram in shared memory, over all buffers and trials of a tile, plus the spare one
+__host__ __device__ inline int hist_slots(const SweepParams &p) { return p.nbuf * p.g * p.hist_copies + p.spare; }
+__host__ __device__ inline int fmax_slots(const SweepParams &p) { return p.aux_copies ? p.nbuf * p.g * p.aux_copies + p.spare : 0; }
 
 // ------------------------------------------------------------------------------------------
 // small PTX wrappers
@@ -78,17 +88,19 @@ __device__ __forceinline__ void mbar_arrive_count(uint64_t *bar, uint32_t count)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
 }
+// One try: the hardware may park the thread for up to kWaitHintNs before it answers "not yet", so a waiting warp
+// costs the scheduler next to nothing instead of spinning through issue slots that other warps could use.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n"
         ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
         "selp.u32 %0, 1, 0, p;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(smem_addr(bar)), "r"(parity)
+        : "r"(smem_addr(bar)), "r"(parity), "r"(kWaitHintNs)
         : "memory");
     return ok != 0;
 }
@@ -99,7 +111,6 @@ __device__ __forceinline__ void mbar_wait(uint64_t *bar, uint32_t parity, uint32
 {
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-        if (it > 64) __nanosleep(128);
     }
     atomicOr(&g_wait_expired, err_bit);
 }
@@ -113,6 +124,38 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, i
 __device__ __forceinline__ void named_barrier(int id, int threads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// Shared-memory accesses by 32-bit shared-window address, for the consumer loop.  Through ordinary pointers every
+// address there is a 64-bit sum (two integer instructions per access, and the bins need two accesses per sample); a
+// 32-bit base plus a byte offset is one.  The increments are the constant 1 on purpose: for that the assembler emits
+// the form of the shared-memory atomic that adds up lanes with equal addresses in one step, whereas a variable
+// increment serialises them (measured: eight times the bank conflicts).
+__device__ __forceinline__ float lds_f32(uint32_t addr)
+{
+    float v;
+    asm("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));  // thresholds and tables: written once before the block's first barrier
+    return v;
+}
+__device__ __forceinline__ unsigned lds_u16(uint32_t addr)
+{
+    unsigned short v;
+    asm("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float4 lds_stage_f32x4(uint32_t addr)
+{
+    float4 v;  // volatile: stays between the wait for the stage and its release
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void red_shared_inc(uint32_t addr)
+{
+    asm volatile("red.shared.add.u32 [%0], 1;" ::"r"(addr));
+}
+__device__ __forceinline__ void red_shared_max(uint32_t addr, int v)
+{
+    asm volatile("red.shared.max.s32 [%0], %1;" ::"r"(addr), "r"(v));
 }
 
 // Start-before-tau rule.  Micro-batch m is run iff the time before it, P_{m-1}, is < tau_k, and a worker's time
@@ -238,40 +281,47 @@ struct SmemTail {
     float *smax;
     int *wtot;
     int *meta;           // [0] lookup table has at most one finite threshold per cell, [1..2] lo, scale (as bits),
-                         // [3] the thresholds are evenly spaced enough for direct binning, [4..5] its scale, shift
+                         // [3] the thresholds are evenly spaced enough for direct binning, [4..5] its scale, shift,
+                         // [6] the last finite threshold (as bits)
     unsigned short *lut; // lut_cells + 1 entries (tiled kernel only)
     float *wmx;          // rule 1, plain kernel: warp totals of the prefix-maximum scan
-    float *fmax;         // rule 1: [nbuf][hist_copies][hist_stride], laid out like hist: largest finish time among
+    float *fmax;         // rule 1: [nbuf][g][hist_copies][hist_stride], laid out like hist: largest finish time among
                          // the micro-batches whose start time lies in the bin
+    int *segmax;         // staged kernels: [nbuf][g] largest row total of each trial of a tile (bit pattern of a
+                         // non-negative float, raised with atomicMax)
 };
 __device__ __forceinline__ SmemTail carve_tail(unsigned char *base, const SweepParams &p)
 {
     SmemTail s;
     s.tau_s = reinterpret_cast<float *>(base);
     s.hist = reinterpret_cast<int *>(s.tau_s + ((p.K + 4) & ~3));  // K + 1 thresholds, padded to 16 bytes
-    s.smax = reinterpret_cast<float *>(s.hist + p.nbuf * p.hist_copies * p.hist_stride);
+    s.smax = reinterpret_cast<float *>(s.hist + hist_slots(p) * p.hist_stride);
     s.wtot = reinterpret_cast<int *>(s.smax + 32);
     s.meta = s.wtot + 32;
     s.lut = reinterpret_cast<unsigned short *>(s.meta + 8);
     s.wmx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(s.lut) +
                                       (((size_t)(p.lut_cells + 1) * sizeof(unsigned short) + 15) & ~(size_t)15));
     s.fmax = s.wmx + 32;
+    s.segmax = reinterpret_cast<int *>(s.fmax + fmax_slots(p) * p.hist_stride);
     return s;
 }
-// hist_copies and fmax_copies count all buffers (nbuf times the copies of one buffer)
-__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride, int lut_cells, int fmax_copies)
+// hist_copies and fmax_copies count all buffers and trials of a tile and the spare copy (hist_slots, fmax_slots);
+// seg_slots = nbuf * g
+__host__ __device__ inline size_t tail_bytes(int K, int hist_copies, int hist_stride, int lut_cells, int fmax_copies,
+                                             int seg_slots = 0)
 {
     return sizeof(float) * (size_t)((K + 4) & ~3) + sizeof(int) * (size_t)hist_copies * hist_stride + 72 * sizeof(int) +
            (((size_t)(lut_cells + 1) * sizeof(unsigned short) + 15) & ~(size_t)15) + 32 * sizeof(float) +
-           sizeof(float) * (size_t)fmax_copies * hist_stride;
+           sizeof(float) * (size_t)fmax_copies * hist_stride + sizeof(int) * (size_t)((seg_slots + 3) & ~3);
 }
 
 __device__ __forceinline__ void load_thresholds(const SweepParams &p, const SmemTail &s, int tid, int nthr)
 {
     for (int k = tid; k < p.K; k += nthr) s.tau_s[k] = p.taus[k];
     if (tid == 0) s.tau_s[p.K] = __int_as_float(0x7f800000);  // +inf sentinel
-    for (int i = tid; i < p.nbuf * p.hist_copies * p.hist_stride; i += nthr) s.hist[i] = 0;
-    for (int i = tid; i < p.nbuf * p.aux_copies * p.hist_stride; i += nthr) s.fmax[i] = 0.0f;
+    for (int i = tid; i < hist_slots(p) * p.hist_stride; i += nthr) s.hist[i] = 0;
+    for (int i = tid; i < fmax_slots(p) * p.hist_stride; i += nthr) s.fmax[i] = 0.0f;
+    for (int i = tid; i < p.nbuf * p.g; i += nthr) s.segmax[i] = 0;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -325,6 +375,7 @@ __device__ __forceinline__ void build_lut(const SweepParams &p, const SmemTail &
         s.meta[0] = 1;
         s.meta[1] = __float_as_int(lo);
         s.meta[2] = __float_as_int(scale);
+        s.meta[6] = __float_as_int(klo <= khi ? s.tau_s[khi] : ninf);  // the last finite threshold (-inf if none)
         // direct binning: all thresholds finite, checked cell by cell after the barrier
         float dscale = 0.0f;
         const bool finite = (klo == 0 && khi == K - 1);
@@ -410,11 +461,13 @@ struct BinCtx {
     unsigned C;
     const unsigned short *lut;
     const unsigned char *tau_b;
+    uint32_t lut_a, tau_a;    // the same two as shared-window addresses
     unsigned K4;
     bool one;                 // the table guarantees at most one threshold to step over
     float dscale, dshift;     // direct binning (only used when the grid qualifies)
     unsigned K;
     float tau_first, tau_last;
+    float tau_top;            // the last FINITE threshold: running sums below it have a cell inside the tables
     uint32_t arrive_one;      // always 1, opaque to the compiler (ties a stage release to a warp vote)
 };
 
@@ -427,6 +480,8 @@ __device__ __forceinline__ BinCtx make_bin_ctx(const SweepParams &p, const SmemT
     c.C = (unsigned)p.lut_cells;
     c.lut = s.lut;
     c.tau_b = reinterpret_cast<const unsigned char *>(s.tau_s);
+    c.lut_a = smem_addr(s.lut);
+    c.tau_a = smem_addr(s.tau_s);
     c.K4 = 4u * (unsigned)p.K;
     c.one = s.meta[0] != 0;
     c.dscale = __int_as_float(s.meta[4]);
@@ -434,6 +489,7 @@ __device__ __forceinline__ BinCtx make_bin_ctx(const SweepParams &p, const SmemT
     c.K = (unsigned)p.K;
     c.tau_first = s.tau_s[0];
     c.tau_last = s.tau_s[p.K - 1];
+    c.tau_top = __int_as_float(s.meta[6]);
     c.arrive_one = (uint32_t)p.one;
     return c;
 }
@@ -463,7 +519,7 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
                                               unsigned char *hist_b, unsigned fmax_delta, float &P, unsigned &prev,
                                               int &cnt0, float &fin0, uint64_t *release_bar)
 {
-    constexpr int GS = NQ >= 2 ? 8 : 4;  // samples per group
+    constexpr int GS = (4 * NQ) % 8 == 0 ? 8 : 4;  // samples per group (a chunk is a whole number of groups)
     // Running sums of the whole chunk, in place.
 #pragma unroll
     for (int q = 0; q < NQ; ++q) {
@@ -571,6 +627,111 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
             }
         }
     }
+}
+
+
+// ------------------------------------------------------------------------------------------
+// The short form of consume_chunk, for rows all of whose chunks are full (4*NQ samples each) and grids on which the
+// table or the cell arithmetic is at most one threshold short of the bin (`one`).  Nothing in it asks whether a lane
+// has a row of its own: such a lane shadows the last row of the tile (same shared-memory data, so the votes need no
+// validity term) and is handed the spare histogram copy, which nothing reads, and counters that are dropped.
+// ------------------------------------------------------------------------------------------
+// The groups of a chunk that hold samples to bin.  CLAMP = false when every lane's running sums of the chunk are
+// below the last finite threshold: cell() is monotone, so the cell index then cannot pass that threshold's and needs
+// no upper bound (negative and NaN inputs convert to 0 either way).
+// `bin` gives the shared-window address of a sample's bin in this thread's histogram copy: the cell arithmetic or
+// the table proposes the bin, the threshold itself decides (tau_s[K] = +inf).
+template <int NS, int GS, int RULE, bool BATCH, bool DIRECT, bool CLAMP>
+__device__ __forceinline__ void bin_groups(const float (&s)[NS], const BinCtx &c, uint32_t hist_a, unsigned fmax_delta,
+                                           unsigned &prev, int &cnt0, float &fin0)
+{
+    auto bin = [&](float x) -> uint32_t {
+        uint32_t off;
+        if (DIRECT) {
+            unsigned cell = __float2uint_rz(__fmaf_rn(x, c.dscale, c.dshift));
+            if (CLAMP) cell = min(cell, c.K);
+            off = 4u * cell;
+        } else {
+            unsigned cell = __float2uint_rz(__fmul_rn(__fsub_rn(x, c.lut_lo), c.lut_scale));
+            if (CLAMP) cell = min(cell, c.C);
+            off = lds_u16(c.lut_a + 2u * cell);
+        }
+        const uint32_t ha = hist_a + off;
+        return (x >= lds_f32(c.tau_a + off)) ? ha + 4u : ha;
+    };
+#pragma unroll
+    for (int g = 0; g < NS; g += GS) {
+        if (g + GS < NS && __all_sync(0xffffffffu, s[g + GS - 1] < c.tau_first)) {  // (the last group is never low here)
+            cnt0 += GS;
+            if (RULE == 1) fin0 = fmaxf(fin0, s[g + GS - 1]);
+            continue;
+        }
+        if (RULE == 0) {
+            if (BATCH) {
+                uint32_t ha[GS];
+#pragma unroll
+                for (int e = 0; e < GS; ++e) ha[e] = bin(s[g + e]);
+#pragma unroll
+                for (int e = 0; e < GS; ++e) red_shared_inc(ha[e]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < GS; ++e) red_shared_inc(bin(s[g + e]));
+            }
+        } else {
+            // `prev` is the ADDRESS of the bin of the running time before the next micro-batch (hist_a = bin 0)
+            uint32_t ha[GS];
+#pragma unroll
+            for (int e = 0; e < GS; ++e) ha[e] = bin(s[g + e]);
+#pragma unroll
+            for (int e = 0; e < GS; ++e) {
+                // bin 0 stays in registers (count and largest finish time), every other bin is updated in place; a
+                // predicated form without the branch measured 15-20 % slower (its increments are serialised)
+                if (prev != hist_a) {
+                    red_shared_inc(prev);
+                    red_shared_max(prev + fmax_delta, __float_as_int(s[g + e]));
+                } else {
+                    ++cnt0;
+                    fin0 = fmaxf(fin0, s[g + e]);
+                }
+                prev = ha[e];
+            }
+        }
+    }
+}
+
+template <int NQ, int RULE, bool BATCH, bool DIRECT>
+__device__ __forceinline__ void consume_full(const float4 (&v)[NQ], int lane, const BinCtx &c, uint32_t hist_a,
+                                             unsigned fmax_delta, float &P, unsigned &prev, int &cnt0, float &fin0,
+                                             uint64_t *release_bar)
+{
+    constexpr int NS = 4 * NQ;
+    constexpr int GS = (NS % 8 == 0) ? 8 : 4;  // samples per group
+    const float before = P;  // running sum before the chunk
+    float s[NS];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        P = __fadd_rn(P, v[q].x); s[4 * q + 0] = P;
+        P = __fadd_rn(P, v[q].y); s[4 * q + 1] = P;
+        P = __fadd_rn(P, v[q].z); s[4 * q + 2] = P;
+        P = __fadd_rn(P, v[q].w); s[4 * q + 3] = P;
+    }
+    // The vote needs every lane's last running sum, i.e. every shared-memory read of the stage by this warp has
+    // returned; the count operand of the arrive depends on the vote (arrive_one is 1), so the release cannot move
+    // ahead of the reads.
+    const bool chunk_low = __all_sync(0xffffffffu, P < c.tau_first);
+    if (lane == 0) mbar_arrive_count(release_bar, chunk_low ? 1u : c.arrive_one);
+    if (chunk_low) {
+        cnt0 += NS;
+        if (RULE == 1) fin0 = fmaxf(fin0, P);
+        return;
+    }
+    // Every lane at or above the last threshold before the chunk: under the paper's rule all its samples fall into
+    // the bin nobody reads, under the start-before-tau rule none of its micro-batches is started.
+    if (__all_sync(0xffffffffu, RULE == 0 ? before >= c.tau_last : prev >= hist_a + c.K4)) return;
+    if (__all_sync(0xffffffffu, P < c.tau_top))
+        bin_groups<NS, GS, RULE, BATCH, DIRECT, false>(s, c, hist_a, fmax_delta, prev, cnt0, fin0);
+    else
+        bin_groups<NS, GS, RULE, BATCH, DIRECT, true>(s, c, hist_a, fmax_delta, prev, cnt0, fin0);
 }
 
 }  // namespace

@@ -167,8 +167,10 @@ __global__ void __launch_bounds__(kMaxRowsPerPass + 64, 2) dc_sweep_flat(const S
             atomicAdd(myhist, cnt0);
             if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
         }
-        rowmax = warp_max(rowmax);
-        if (lane == 0) s.smax[32 * b + warp] = rowmax;
+        {   // largest row total of the trial (non-negative floats order like their bit patterns)
+            const unsigned wm = __reduce_max_sync(0xffffffffu, (unsigned)__float_as_int(rowmax));
+            if (lane == 0) atomicMax(&s.segmax[b], (int)wm);
+        }
         buffer_barrier_arrive<kBarReady>(b, bar_threads);
     }
 }

@@ -47,168 +47,285 @@ __device__ __forceinline__ void buffer_barrier_arrive(int b, int threads)
     else bar_arrive_imm<BASE + 1>(threads);
 }
 
-// The epilogue warp's loop (all 32 lanes).  Bins are taken 32 at a time: lane l sums bin k0+l over the
-// copies (and clears it), a warp scan gives the prefix, a carry links the blocks of 32.
+// The epilogue warp's loop (all 32 lanes) over the block's tiles; a tile holds p.g whole trials (1 unless trials are
+// small), each with histograms of its own.  Bins are taken 128 (or 32) at a time: a lane sums its bins over the
+// copies (and clears them), a warp scan gives the prefix, a carry links the steps.
 template <int RULE>
 __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTail &s, int lane, int ncw)
 {
-    const int K = p.K, H = p.hist_copies, HS = p.hist_stride;
+    const int K = p.K, H = p.hist_copies, HS = p.hist_stride, G = p.g;
     const int bar_threads = ncw * 32 + 32;
+    const long long tiles = (p.T + G - 1) / G;
     int j = 0;
-    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
+    for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++j) {
         const int b = j & 1;
-        buffer_barrier_sync<kBarReady>(b, bar_threads);  // every consumer has finished trial t
-        int *hist = s.hist + b * H * HS;
-        float *fmax = s.fmax + b * H * HS;  // rule 1 only
-        const float Tmax = warp_max(lane < ncw ? s.smax[32 * b + lane] : 0.0f);
-        const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
-        float *step_row = p.out_step + t * K;
-        int32_t *done_row = p.out_done + t * K;
-        int carry = 0;
-        float fm_carry = 0.0f;
-        // Four consecutive bins per lane, 128 bins per step, with 16-byte accesses throughout (when the shapes and
-        // pointers allow): a quarter of the scans and well under half the instructions of the scalar loop below.
-        for (int k0 = 0; p.epi_vec && k0 < K; k0 += 128) {
-            const int k = k0 + 4 * lane;
-            const bool in = k < K;  // K is a multiple of 4: a lane's four bins are all inside or all outside
-            int4 h = make_int4(0, 0, 0, 0);
-            float4 fm = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            if (in) {
+        buffer_barrier_sync<kBarReady>(b, bar_threads);  // every consumer has finished this tile
+        if (p.epi_sub > 0) {
+            // Several small trials per step: L = K/4 lanes (a power of two) take one trial, four bins each, and the
+            // scans run inside groups of L lanes; 32/L trials go through the warp at once.
+            const int L = p.epi_sub, per_step = 32 / L;
+            const int sub = lane & (L - 1), k = 4 * sub;
+            for (int seg0 = 0; seg0 < G; seg0 += per_step) {
+                const int seg = seg0 + lane / L;
+                const long long t = tile * G + seg;
+                const bool in = seg < G && t < p.T;
+                int4 h = make_int4(0, 0, 0, 0);
+                float4 fm = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                float Tmax = 0.0f;
+                if (in) {
+                    for (int c = 0; c < H; ++c) {
+                        int4 *hp = reinterpret_cast<int4 *>(s.hist + ((b * G + seg) * H + c) * HS + k);
+                        const int4 v = *hp;
+                        *hp = make_int4(0, 0, 0, 0);
+                        h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
+                        if (RULE == 1) {
+                            float4 *fp = reinterpret_cast<float4 *>(s.fmax + ((b * G + seg) * H + c) * HS + k);
+                            const float4 f = *fp;
+                            *fp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                            fm.x = fmaxf(fm.x, f.x); fm.y = fmaxf(fm.y, f.y); fm.z = fmaxf(fm.z, f.z); fm.w = fmaxf(fm.w, f.w);
+                        }
+                    }
+                    Tmax = __int_as_float(s.segmax[b * G + seg]);
+                }
+                h.y += h.x; h.z += h.y; h.w += h.z;  // inclusive inside the lane
+                int incl = h.w;
+                for (int o = 1; o < L; o <<= 1) {
+                    const int u = __shfl_up_sync(0xffffffffu, incl, o, L);
+                    if (sub >= o) incl += u;
+                }
+                const int base = incl - h.w;  // everything before this lane's bins, within its trial
+                float4 st;
+                if (RULE == 0) {
+                    const float4 tq = *reinterpret_cast<const float4 *>(s.tau_s + k);
+                    st.x = fminf(tq.x, Tmax); st.y = fminf(tq.y, Tmax); st.z = fminf(tq.z, Tmax); st.w = fminf(tq.w, Tmax);
+                } else {
+                    fm.y = fmaxf(fm.y, fm.x); fm.z = fmaxf(fm.z, fm.y); fm.w = fmaxf(fm.w, fm.z);
+                    float fincl = fm.w;
+                    for (int o = 1; o < L; o <<= 1) {
+                        const float u = __shfl_up_sync(0xffffffffu, fincl, o, L);
+                        if (sub >= o) fincl = fmaxf(fincl, u);
+                    }
+                    float before = __shfl_up_sync(0xffffffffu, fincl, 1, L);
+                    before = sub > 0 ? before : 0.0f;
+                    st.x = fmaxf(before, fm.x); st.y = fmaxf(before, fm.y); st.z = fmaxf(before, fm.z); st.w = fmaxf(before, fm.w);
+                }
+                if (in) {
+                    const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
+                    *reinterpret_cast<int4 *>(p.out_done + t * K + k) = make_int4(base + h.x, base + h.y, base + h.z, base + h.w);
+                    *reinterpret_cast<float4 *>(p.out_step + t * K + k) =
+                        make_float4(__fadd_rn(st.x, t_comm), __fadd_rn(st.y, t_comm), __fadd_rn(st.z, t_comm), __fadd_rn(st.w, t_comm));
+                    if (sub == 0) {  // the two bins past the last threshold, the trial's maximum, the synchronous time
+                        for (int c = 0; c < H; ++c) {
+                            s.hist[((b * G + seg) * H + c) * HS + K] = 0;
+                            s.hist[((b * G + seg) * H + c) * HS + K + 1] = 0;
+                            if (RULE == 1) {
+                                s.fmax[((b * G + seg) * H + c) * HS + K] = 0.0f;
+                                s.fmax[((b * G + seg) * H + c) * HS + K + 1] = 0.0f;
+                            }
+                        }
+                        s.segmax[b * G + seg] = 0;
+                        if (p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
+                    }
+                }
+            }
+            buffer_barrier_arrive<kBarFree>(b, bar_threads);  // buffer b is clear again
+            continue;
+        }
+        for (int seg = 0; seg < G; ++seg) {
+            const long long t = tile * G + seg;
+            if (t >= p.T) break;  // (nothing was added for trials past the last one)
+            int *hist = s.hist + (b * G + seg) * H * HS;
+            float *fmax = s.fmax + (b * G + seg) * H * HS;  // rule 1 only
+            const float Tmax = __int_as_float(s.segmax[b * G + seg]);
+            const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
+            float *step_row = p.out_step + t * K;
+            int32_t *done_row = p.out_done + t * K;
+            int carry = 0;
+            float fm_carry = 0.0f;
+            // Four consecutive bins per lane, 128 bins per step, with 16-byte accesses throughout (when the shapes
+            // and pointers allow): a quarter of the scans and well under half the instructions of the scalar loop.
+            for (int k0 = 0; p.epi_vec && k0 < K; k0 += 128) {
+                const int k = k0 + 4 * lane;
+                const bool in = k < K;  // K is a multiple of 4: a lane's four bins are all inside or all outside
+                int4 h = make_int4(0, 0, 0, 0);
+                float4 fm = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                if (in) {
 #pragma unroll 2
-                for (int c = 0; c < H; ++c) {
-                    int4 *hp = reinterpret_cast<int4 *>(hist + c * HS + k);
-                    const int4 v = *hp;
-                    *hp = make_int4(0, 0, 0, 0);
-                    h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
-                    if (RULE == 1) {
-                        float4 *fp = reinterpret_cast<float4 *>(fmax + c * HS + k);
-                        const float4 f = *fp;
-                        *fp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                        fm.x = fmaxf(fm.x, f.x); fm.y = fmaxf(fm.y, f.y); fm.z = fmaxf(fm.z, f.z); fm.w = fmaxf(fm.w, f.w);
+                    for (int c = 0; c < H; ++c) {
+                        int4 *hp = reinterpret_cast<int4 *>(hist + c * HS + k);
+                        const int4 v = *hp;
+                        *hp = make_int4(0, 0, 0, 0);
+                        h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
+                        if (RULE == 1) {
+                            float4 *fp = reinterpret_cast<float4 *>(fmax + c * HS + k);
+                            const float4 f = *fp;
+                            *fp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                            fm.x = fmaxf(fm.x, f.x); fm.y = fmaxf(fm.y, f.y); fm.z = fmaxf(fm.z, f.z); fm.w = fmaxf(fm.w, f.w);
+                        }
                     }
                 }
-            }
-            h.y += h.x; h.z += h.y; h.w += h.z;  // inclusive inside the lane
-            const int incl = warp_inclusive_scan(h.w, lane);
-            const int base = carry + incl - h.w;  // everything before this lane's bins
-            carry += __shfl_sync(0xffffffffu, incl, 31);
-            float4 st;
-            if (RULE == 0) {
-                const float4 tq = in ? *reinterpret_cast<const float4 *>(s.tau_s + k) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                st.x = fminf(tq.x, Tmax); st.y = fminf(tq.y, Tmax); st.z = fminf(tq.z, Tmax); st.w = fminf(tq.w, Tmax);
-            } else {
-                // max_n W_n(k) = max_{j <= k} fmax[j]
-                fm.y = fmaxf(fm.y, fm.x); fm.z = fmaxf(fm.z, fm.y); fm.w = fmaxf(fm.w, fm.z);
-                const float fincl = warp_inclusive_max_scan(fm.w, lane);
-                float before = __shfl_up_sync(0xffffffffu, fincl, 1);
-                before = fmaxf(fm_carry, lane > 0 ? before : 0.0f);
-                fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fincl, 31));
-                st.x = fmaxf(before, fm.x); st.y = fmaxf(before, fm.y); st.z = fmaxf(before, fm.z); st.w = fmaxf(before, fm.w);
-            }
-            if (in) {
-                *reinterpret_cast<int4 *>(done_row + k) = make_int4(base + h.x, base + h.y, base + h.z, base + h.w);
-                *reinterpret_cast<float4 *>(step_row + k) =
-                    make_float4(__fadd_rn(st.x, t_comm), __fadd_rn(st.y, t_comm), __fadd_rn(st.z, t_comm), __fadd_rn(st.w, t_comm));
-            }
-        }
-        // Otherwise: 32 bins at a time, lane l sums bin k0+l over the copies (and clears it), a warp scan gives the
-        // prefix, a carry links the blocks of 32.
-        for (int k0 = p.epi_vec ? K : 0; k0 < K; k0 += 32) {
-            const int k = k0 + lane;
-            int h = 0;
-            float fm = 0.0f;
-            if (k < K) {
-                for (int c = 0; c < H; ++c) {
-                    h += hist[c * HS + k];
-                    hist[c * HS + k] = 0;
-                    if (RULE == 1) {
-                        fm = fmaxf(fm, fmax[c * HS + k]);
-                        fmax[c * HS + k] = 0.0f;
-                    }
+                h.y += h.x; h.z += h.y; h.w += h.z;  // inclusive inside the lane
+                const int incl = warp_inclusive_scan(h.w, lane);
+                const int base = carry + incl - h.w;  // everything before this lane's bins
+                carry += __shfl_sync(0xffffffffu, incl, 31);
+                float4 st;
+                if (RULE == 0) {
+                    const float4 tq = in ? *reinterpret_cast<const float4 *>(s.tau_s + k) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    st.x = fminf(tq.x, Tmax); st.y = fminf(tq.y, Tmax); st.z = fminf(tq.z, Tmax); st.w = fminf(tq.w, Tmax);
+                } else {
+                    // max_n W_n(k) = max_{j <= k} fmax[j]
+                    fm.y = fmaxf(fm.y, fm.x); fm.z = fmaxf(fm.z, fm.y); fm.w = fmaxf(fm.w, fm.z);
+                    const float fincl = warp_inclusive_max_scan(fm.w, lane);
+                    float before = __shfl_up_sync(0xffffffffu, fincl, 1);
+                    before = fmaxf(fm_carry, lane > 0 ? before : 0.0f);
+                    fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fincl, 31));
+                    st.x = fmaxf(before, fm.x); st.y = fmaxf(before, fm.y); st.z = fmaxf(before, fm.z); st.w = fmaxf(before, fm.w);
+                }
+                if (in) {
+                    *reinterpret_cast<int4 *>(done_row + k) = make_int4(base + h.x, base + h.y, base + h.z, base + h.w);
+                    *reinterpret_cast<float4 *>(step_row + k) =
+                        make_float4(__fadd_rn(st.x, t_comm), __fadd_rn(st.y, t_comm), __fadd_rn(st.z, t_comm), __fadd_rn(st.w, t_comm));
                 }
             }
-            const int incl = warp_inclusive_scan(h, lane);
-            float step;
-            if (RULE == 0) {
-                step = __fadd_rn(fminf(k < K ? s.tau_s[k] : 0.0f, Tmax), t_comm);
-            } else {
-                const float fm_incl = warp_inclusive_max_scan(fm, lane);
-                step = __fadd_rn(fmaxf(fm_carry, fm_incl), t_comm);
-                fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fm_incl, 31));
+            // Otherwise: 32 bins at a time, lane l sums bin k0+l over the copies (and clears it), a warp scan gives the
+            // prefix, a carry links the blocks of 32.
+            for (int k0 = p.epi_vec ? K : 0; k0 < K; k0 += 32) {
+                const int k = k0 + lane;
+                int h = 0;
+                float fm = 0.0f;
+                if (k < K) {
+                    for (int c = 0; c < H; ++c) {
+                        h += hist[c * HS + k];
+                        hist[c * HS + k] = 0;
+                        if (RULE == 1) {
+                            fm = fmaxf(fm, fmax[c * HS + k]);
+                            fmax[c * HS + k] = 0.0f;
+                        }
+                    }
+                }
+                const int incl = warp_inclusive_scan(h, lane);
+                float step;
+                if (RULE == 0) {
+                    step = __fadd_rn(fminf(k < K ? s.tau_s[k] : 0.0f, Tmax), t_comm);
+                } else {
+                    const float fm_incl = warp_inclusive_max_scan(fm, lane);
+                    step = __fadd_rn(fmaxf(fm_carry, fm_incl), t_comm);
+                    fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fm_incl, 31));
+                }
+                if (k < K) {
+                    done_row[k] = carry + incl;
+                    step_row[k] = step;
+                }
+                carry += __shfl_sync(0xffffffffu, incl, 31);
             }
-            if (k < K) {
-                done_row[k] = carry + incl;
-                step_row[k] = step;
+            for (int c = lane; c < H; c += 32) {  // the two bins past the last threshold
+                hist[c * HS + K] = 0;
+                hist[c * HS + K + 1] = 0;
             }
-            carry += __shfl_sync(0xffffffffu, incl, 31);
-        }
-        for (int c = lane; c < H; c += 32) {  // the two bins past the last threshold
-            hist[c * HS + K] = 0;
-            hist[c * HS + K + 1] = 0;
-        }
-        if (RULE == 1) {
-            for (int c = lane; c < H; c += 32) {
-                fmax[c * HS + K] = 0.0f;
-                fmax[c * HS + K + 1] = 0.0f;
+            if (RULE == 1) {
+                for (int c = lane; c < H; c += 32) {
+                    fmax[c * HS + K] = 0.0f;
+                    fmax[c * HS + K + 1] = 0.0f;
+                }
+            }
+            if (lane == 0) {
+                s.segmax[b * G + seg] = 0;
+                if (p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
             }
         }
-        if (lane == 0 && p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
         buffer_barrier_arrive<kBarFree>(b, bar_threads);  // buffer b is clear again
     }
 }
 
-// The consumer threads' loop over the block's trials (tiled kernel).
-template <int NQ, int RULE, bool BATCH, bool DIRECT>
+// The consumer threads' loop over the block's tiles (tiled kernel).  A tile is p.g whole trials when trials are
+// small (thread r owns row r of the g*N rows, which belongs to trial r / N of the tile), else one trial whose
+// workers are taken in p.passes passes of p.rows rows.  LEAN = every chunk of a row is full (consume_full).
+template <int NQ, int RULE, bool BATCH, bool DIRECT, bool LEAN>
 __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTail &s, const BinCtx &ctx, unsigned char *stage0,
                                              uint64_t *full, uint64_t *empty, int tid, int lane, int warp, int ncw,
-                                             int *myhist0, unsigned fmax_delta, unsigned off_zero)
+                                             unsigned fmax_delta, unsigned off_zero)
 {
-    const int S = p.stages;
+    const int S = p.stages, G = p.g;
     const int bar_threads = ncw * 32 + 32;
-    const int hist_buf_ints = p.hist_copies * p.hist_stride;
+    const int seg_ints = p.hist_copies * p.hist_stride;  // one trial's histograms
+    // Threads past the last row of the tile shadow rows of the tile (different ones, so that what they add to the
+    // spare histogram copy spreads over its bins like real rows do).
+    const int row = tid < p.rows ? tid : tid % p.rows;
+    const int seg = G > 1 ? row / p.N : 0;
+    const int copy = (warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1));
+    int *myhist0 = s.hist + seg * seg_ints + copy * p.hist_stride;
     // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
-    // (threads past the last row of the box read the last row instead: always inside the stage)
-    const uint32_t row_off = (uint32_t)min(tid, p.rows - 1) * (uint32_t)p.pitch;
+    const uint32_t row_off = (uint32_t)row * (uint32_t)p.pitch;
     const uint32_t swz = ((row_off >> 7) & (uint32_t)p.swz_mask) << 4;
+    uint32_t qoff[NQ];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) qoff[q] = row_off + ((uint32_t)(q * 16) ^ swz);
+    // the spare histogram copy (after all real ones, never read): where lanes without a row of their own add
+    const uint32_t spare_a = smem_addr(s.hist + (hist_slots(p) - 1) * p.hist_stride);
+    const uint32_t stage0_a = smem_addr(stage0);
+    const long long tiles = (p.T + G - 1) / G;
     int st = 0;
     uint32_t ph = 0;
     int j = 0;
-    for (long long t = blockIdx.x; t < p.T; t += gridDim.x, ++j) {
+    for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++j) {
         const int b = j & 1;
         if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
-        int *myhist = myhist0 + b * hist_buf_ints;
+        int *myhist = myhist0 + b * G * seg_ints;
         unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
+        const bool in_tile = (tid < p.rows) && (tile * G + seg < p.T);  // this thread's trial exists
         float rowmax = 0.0f, fin0 = 0.0f;
         int cnt0 = 0;
         for (int pass = 0; pass < p.passes; ++pass) {
-            const bool valid = (tid < p.rows) && (pass * p.rows + tid < p.N);
-            float P = 0.0f;
-            unsigned prev = off_zero;  // rule 1: bin (byte offset) of the running time before the next micro-batch
+            const bool valid = in_tile && (pass * p.rows + tid < p.N || G > 1);
+            float P = 0.0f, pass_fin0 = 0.0f;
+            int pass_cnt0 = 0;
+            const uint32_t hist_a = valid ? smem_addr(hist_b) : spare_a;  // (short loop) where this lane adds in this pass
+            // rule 1: bin of the running time before the next micro-batch, as a byte offset (general loop) or as the
+            // address of that bin in this lane's histogram copy (short loop)
+            unsigned prev = LEAN ? hist_a + off_zero : off_zero;
             for (int c = 0; c < p.chunks; ++c) {
                 mbar_wait(&full[st], ph, kErrLoadNeverArrived);
-                const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes + row_off;
+                const unsigned char *stage = stage0 + (size_t)st * p.stage_bytes;
+                const uint32_t stage_a = stage0_a + (uint32_t)st * (uint32_t)p.stage_bytes;
                 uint64_t *empty_bar = &empty[st];
                 if (++st == S) {
                     st = 0;
                     ph ^= 1u;
                 }
-                const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
                 float4 v[NQ];
+                if (LEAN) {
 #pragma unroll
-                for (int q = 0; q < NQ; ++q) {
-                    if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + ((uint32_t)(q * 16) ^ swz));
-                    else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    for (int q = 0; q < NQ; ++q) v[q] = lds_stage_f32x4(stage_a + qoff[q]);
+                    consume_full<NQ, RULE, BATCH, DIRECT>(v, lane, ctx, hist_a, fmax_delta, P, prev, pass_cnt0, pass_fin0, empty_bar);
+                } else {
+                    const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
+#pragma unroll
+                    for (int q = 0; q < NQ; ++q) {
+                        if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + qoff[q]);
+                        else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    }
+                    consume_chunk<NQ, RULE, BATCH, DIRECT>(v, 4 * nq, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, empty_bar);
                 }
-                consume_chunk<NQ, RULE, BATCH, DIRECT>(v, 4 * nq, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, empty_bar);
             }
-            if (valid) rowmax = fmaxf(rowmax, P);
+            if (valid) {
+                rowmax = fmaxf(rowmax, P);
+                if (LEAN) {  // (a lane without a row in this pass drops what it counted: the row's owner has it)
+                    cnt0 += pass_cnt0;
+                    fin0 = fmaxf(fin0, pass_fin0);
+                }
+            }
         }
         if (cnt0 > 0) {
             atomicAdd(myhist, cnt0);
             if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
         }
-        rowmax = warp_max(rowmax);
-        if (lane == 0) s.smax[32 * b + warp] = rowmax;
+        // largest row total of the trial: running sums are non-negative, so their bit patterns order like integers
+        if (G > 1) {
+            if (in_tile) atomicMax(&s.segmax[b * G + seg], __float_as_int(rowmax));
+        } else {
+            const unsigned wm = __reduce_max_sync(0xffffffffu, (unsigned)__float_as_int(rowmax));
+            if (lane == 0) atomicMax(&s.segmax[b], (int)wm);
+        }
         buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
     }
 }
@@ -231,13 +348,15 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     const int S = p.stages;
 
     // The producer thread sets up the barriers and fills the whole ring before the block builds its tables: the
-    // first tiles are on their way from HBM while the thresholds are read and the lookup table is built.
-    // (tile = one chunk of one pass of one trial; the block's tiles in order: trial, pass, chunk)
+    // first boxes are on their way from HBM while the thresholds are read and the lookup table is built.
+    // (box = one chunk of one pass of one tile; the block's boxes in order: tile, pass, chunk.  With several trials
+    // per tile the box is {chunk, all N workers, g trials}; trials past the last one are zero-filled.)
+    const long long tiles = (p.T + p.g - 1) / p.g;
     long long prod_t = blockIdx.x;
     int prod_pass = 0, prod_c = 0, prod_issued = 0;
     auto issue_tile = [&](int st) {
         mbar_arrive_expect_tx(&full[st], (uint32_t)(p.rows * p.pitch));
-        tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, prod_c * p.bw, prod_pass * p.rows, (int)prod_t, &full[st]);
+        tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, prod_c * p.bw, prod_pass * p.rows, (int)(prod_t * p.g), &full[st]);
         if (++prod_c == p.chunks) {
             prod_c = 0;
             if (++prod_pass == p.passes) {
@@ -253,7 +372,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        while (prod_issued < S && prod_t < p.T) issue_tile(prod_issued++);
+        while (prod_issued < S && prod_t < tiles) issue_tile(prod_issued++);
     }
     load_thresholds(p, s, tid, blockDim.x);
     __syncthreads();  // also: the initialised barriers are visible to every thread
@@ -264,7 +383,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
         if (lane == 0) {
             int st = 0;
             uint32_t ph = 1;  // parity of the current use of stage st (every stage has been used once)
-            while (prod_t < p.T) {
+            while (prod_t < tiles) {
                 mbar_wait(&empty[st], ph ^ 1u, kErrStageNeverFreed);
                 issue_tile(st);
                 if (++st == S) {
@@ -281,16 +400,19 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     }
 
     // ---------------- consumers
-    int *myhist0 = s.hist + ((warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1))) * p.hist_stride;
-    // rule 1: byte distance from a histogram entry to the finish-time maximum of the same buffer, copy and bin
+    // rule 1: byte distance from a histogram entry to the finish-time maximum of the same buffer, trial, copy and bin
     const unsigned fmax_delta = (unsigned)(reinterpret_cast<unsigned char *>(s.fmax) - reinterpret_cast<unsigned char *>(s.hist));
     const BinCtx ctx = make_bin_ctx(p, s);
     const bool one = ctx.one;
     const unsigned off_zero = RULE == 1 ? bin_of_zero(ctx) : 0u;  // rule 1 only
-    if (s.meta[3] != 0 && one && p.direct_bins != 0)
-        tiled_trials<NQ, RULE, BATCH, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, myhist0, fmax_delta, off_zero);
-    else
-        tiled_trials<NQ, RULE, BATCH, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, myhist0, fmax_delta, off_zero);
+    const bool direct = s.meta[3] != 0 && one && p.direct_bins != 0;
+    if (p.lean != 0 && one) {
+        if (direct) tiled_trials<NQ, RULE, BATCH, true, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
+        else tiled_trials<NQ, RULE, BATCH, false, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
+    } else {
+        if (direct) tiled_trials<NQ, RULE, BATCH, true, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
+        else tiled_trials<NQ, RULE, BATCH, false, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
+    }
 }
 
 }  // namespace

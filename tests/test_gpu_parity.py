@@ -78,6 +78,12 @@ EDGE_SHAPES = [
     (2, 256, 32, 4096),              # the largest grid
     (300, 5, 16, 3),                 # many short trials, more trials than blocks in flight
     (1, 1000, 8, 1),                 # one trial only
+    # several whole trials of few workers share a tile (the last tile holds fewer trials than the others)
+    (1000, 8, 4, 16), (1000, 8, 12, 16), (1000, 8, 32, 7), (333, 5, 4, 33), (333, 5, 12, 64), (333, 5, 32, 9),
+    (77, 33, 4, 16), (77, 33, 12, 40), (77, 33, 32, 128), (50, 128, 4, 5), (50, 128, 12, 64), (50, 128, 32, 256),
+    (5000, 3, 8, 20), (700, 1, 16, 4), (900, 100, 48, 64), (650, 64, 36, 30),
+    # row lengths cut into equal chunks of 12, 16 or 24 floats (36, 48, 72, 80) and one that is not (100)
+    (6, 300, 48, 40), (5, 256, 72, 64), (4, 150, 80, 33), (40, 260, 36, 50),
 ]
 
 

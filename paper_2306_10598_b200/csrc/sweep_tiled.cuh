@@ -47,192 +47,218 @@ __device__ __forceinline__ void buffer_barrier_arrive(int b, int threads)
     else bar_arrive_imm<BASE + 1>(threads);
 }
 
-// The epilogue warp's loop (all 32 lanes) over the block's tiles; a tile holds p.g whole trials (1 unless trials are
-// small), each with histograms of its own.  Bins are taken 128 (or 32) at a time: a lane sums its bins over the
-// copies (and clears them), a warp scan gives the prefix, a carry links the steps.
+// One finished trial (all 32 lanes of a warp): its histograms (p.hist_copies copies at `hist`, finish-time maxima at
+// `fmax` under rule 1) become out_done / out_step / out_sync of trial t, and are cleared.  Bins are taken 128 (or 32)
+// at a time: a lane sums its bins over the copies (and clears them), a warp scan gives the prefix, a carry links the
+// steps.  `segmax` holds the bit pattern of the trial's largest row total.
+template <int RULE>
+__device__ __forceinline__ void epilogue_trial(const SweepParams &p, const SmemTail &s, int *hist, float *fmax, int *segmax,
+                                               long long t, int lane)
+{
+    const int K = p.K, H = p.hist_copies, HS = p.hist_stride;
+    const float Tmax = __int_as_float(*segmax);
+    const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
+    float *step_row = p.out_step + t * K;
+    int32_t *done_row = p.out_done + t * K;
+    int carry = 0;
+    float fm_carry = 0.0f;
+    // Four consecutive bins per lane, 128 bins per step, with 16-byte accesses throughout (when the shapes
+    // and pointers allow): a quarter of the scans and well under half the instructions of the scalar loop.
+    for (int k0 = 0; p.epi_vec && k0 < K; k0 += 128) {
+        const int k = k0 + 4 * lane;
+        const bool in = k < K;  // K is a multiple of 4: a lane's four bins are all inside or all outside
+        int4 h = make_int4(0, 0, 0, 0);
+        float4 fm = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (in) {
+#pragma unroll 2
+            for (int c = 0; c < H; ++c) {
+                int4 *hp = reinterpret_cast<int4 *>(hist + c * HS + k);
+                const int4 v = *hp;
+                *hp = make_int4(0, 0, 0, 0);
+                h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
+                if (RULE == 1) {
+                    float4 *fp = reinterpret_cast<float4 *>(fmax + c * HS + k);
+                    const float4 f = *fp;
+                    *fp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    fm.x = fmaxf(fm.x, f.x); fm.y = fmaxf(fm.y, f.y); fm.z = fmaxf(fm.z, f.z); fm.w = fmaxf(fm.w, f.w);
+                }
+            }
+        }
+        h.y += h.x; h.z += h.y; h.w += h.z;  // inclusive inside the lane
+        const int incl = warp_inclusive_scan(h.w, lane);
+        const int base = carry + incl - h.w;  // everything before this lane's bins
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+        float4 st;
+        if (RULE == 0) {
+            const float4 tq = in ? *reinterpret_cast<const float4 *>(s.tau_s + k) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            st.x = fminf(tq.x, Tmax); st.y = fminf(tq.y, Tmax); st.z = fminf(tq.z, Tmax); st.w = fminf(tq.w, Tmax);
+        } else {
+            // max_n W_n(k) = max_{j <= k} fmax[j]
+            fm.y = fmaxf(fm.y, fm.x); fm.z = fmaxf(fm.z, fm.y); fm.w = fmaxf(fm.w, fm.z);
+            const float fincl = warp_inclusive_max_scan(fm.w, lane);
+            float before = __shfl_up_sync(0xffffffffu, fincl, 1);
+            before = fmaxf(fm_carry, lane > 0 ? before : 0.0f);
+            fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fincl, 31));
+            st.x = fmaxf(before, fm.x); st.y = fmaxf(before, fm.y); st.z = fmaxf(before, fm.z); st.w = fmaxf(before, fm.w);
+        }
+        if (in) {
+            *reinterpret_cast<int4 *>(done_row + k) = make_int4(base + h.x, base + h.y, base + h.z, base + h.w);
+            *reinterpret_cast<float4 *>(step_row + k) =
+                make_float4(__fadd_rn(st.x, t_comm), __fadd_rn(st.y, t_comm), __fadd_rn(st.z, t_comm), __fadd_rn(st.w, t_comm));
+        }
+    }
+    // Otherwise: 32 bins at a time, lane l sums bin k0+l over the copies (and clears it), a warp scan gives the
+    // prefix, a carry links the blocks of 32.
+    for (int k0 = p.epi_vec ? K : 0; k0 < K; k0 += 32) {
+        const int k = k0 + lane;
+        int h = 0;
+        float fm = 0.0f;
+        if (k < K) {
+            for (int c = 0; c < H; ++c) {
+                h += hist[c * HS + k];
+                hist[c * HS + k] = 0;
+                if (RULE == 1) {
+                    fm = fmaxf(fm, fmax[c * HS + k]);
+                    fmax[c * HS + k] = 0.0f;
+                }
+            }
+        }
+        const int incl = warp_inclusive_scan(h, lane);
+        float step;
+        if (RULE == 0) {
+            step = __fadd_rn(fminf(k < K ? s.tau_s[k] : 0.0f, Tmax), t_comm);
+        } else {
+            const float fm_incl = warp_inclusive_max_scan(fm, lane);
+            step = __fadd_rn(fmaxf(fm_carry, fm_incl), t_comm);
+            fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fm_incl, 31));
+        }
+        if (k < K) {
+            done_row[k] = carry + incl;
+            step_row[k] = step;
+        }
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    for (int c = lane; c < H; c += 32) {  // the two bins past the last threshold
+        hist[c * HS + K] = 0;
+        hist[c * HS + K + 1] = 0;
+    }
+    if (RULE == 1) {
+        for (int c = lane; c < H; c += 32) {
+            fmax[c * HS + K] = 0.0f;
+            fmax[c * HS + K + 1] = 0.0f;
+        }
+    }
+    if (lane == 0) {
+        *segmax = 0;
+        if (p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
+    }
+}
+
+// Several small trials in one step of a warp: L = p.epi_sub = K/4 lanes (a power of two) take one trial, four bins
+// each, and the scans run inside groups of L lanes, so 32/L trials of a tile (seg0, seg0 + 1, ...) go through the warp
+// at once.  `slot0` = index of the tile's first trial among the histogram slots.
+template <int RULE>
+__device__ __forceinline__ void epilogue_small_trials(const SweepParams &p, const SmemTail &s, int slot0, long long t0, int seg0,
+                                                      int lane)
+{
+    const int K = p.K, H = p.hist_copies, HS = p.hist_stride, G = p.g;
+    const int L = p.epi_sub;
+    const int sub = lane & (L - 1), k = 4 * sub;
+    const int seg = seg0 + lane / L;
+    const long long t = t0 + seg;
+    const bool in = seg < G && t < p.T;
+    int4 h = make_int4(0, 0, 0, 0);
+    float4 fm = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    float Tmax = 0.0f;
+    if (in) {
+        for (int c = 0; c < H; ++c) {
+            int4 *hp = reinterpret_cast<int4 *>(s.hist + ((slot0 + seg) * H + c) * HS + k);
+            const int4 v = *hp;
+            *hp = make_int4(0, 0, 0, 0);
+            h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
+            if (RULE == 1) {
+                float4 *fp = reinterpret_cast<float4 *>(s.fmax + ((slot0 + seg) * H + c) * HS + k);
+                const float4 f = *fp;
+                *fp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                fm.x = fmaxf(fm.x, f.x); fm.y = fmaxf(fm.y, f.y); fm.z = fmaxf(fm.z, f.z); fm.w = fmaxf(fm.w, f.w);
+            }
+        }
+        Tmax = __int_as_float(s.segmax[slot0 + seg]);
+    }
+    h.y += h.x; h.z += h.y; h.w += h.z;  // inclusive inside the lane
+    int incl = h.w;
+    for (int o = 1; o < L; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, incl, o, L);
+        if (sub >= o) incl += u;
+    }
+    const int base = incl - h.w;  // everything before this lane's bins, within its trial
+    float4 st;
+    if (RULE == 0) {
+        const float4 tq = *reinterpret_cast<const float4 *>(s.tau_s + k);
+        st.x = fminf(tq.x, Tmax); st.y = fminf(tq.y, Tmax); st.z = fminf(tq.z, Tmax); st.w = fminf(tq.w, Tmax);
+    } else {
+        fm.y = fmaxf(fm.y, fm.x); fm.z = fmaxf(fm.z, fm.y); fm.w = fmaxf(fm.w, fm.z);
+        float fincl = fm.w;
+        for (int o = 1; o < L; o <<= 1) {
+            const float u = __shfl_up_sync(0xffffffffu, fincl, o, L);
+            if (sub >= o) fincl = fmaxf(fincl, u);
+        }
+        float before = __shfl_up_sync(0xffffffffu, fincl, 1, L);
+        before = sub > 0 ? before : 0.0f;
+        st.x = fmaxf(before, fm.x); st.y = fmaxf(before, fm.y); st.z = fmaxf(before, fm.z); st.w = fmaxf(before, fm.w);
+    }
+    if (in) {
+        const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
+        *reinterpret_cast<int4 *>(p.out_done + t * K + k) = make_int4(base + h.x, base + h.y, base + h.z, base + h.w);
+        *reinterpret_cast<float4 *>(p.out_step + t * K + k) =
+            make_float4(__fadd_rn(st.x, t_comm), __fadd_rn(st.y, t_comm), __fadd_rn(st.z, t_comm), __fadd_rn(st.w, t_comm));
+        if (sub == 0) {  // the two bins past the last threshold, the trial's maximum, the synchronous time
+            for (int c = 0; c < H; ++c) {
+                s.hist[((slot0 + seg) * H + c) * HS + K] = 0;
+                s.hist[((slot0 + seg) * H + c) * HS + K + 1] = 0;
+                if (RULE == 1) {
+                    s.fmax[((slot0 + seg) * H + c) * HS + K] = 0.0f;
+                    s.fmax[((slot0 + seg) * H + c) * HS + K + 1] = 0.0f;
+                }
+            }
+            s.segmax[slot0 + seg] = 0;
+            if (p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
+        }
+    }
+}
+
+// The trials of one finished tile, shared out over `nw` warps (this is warp `w` of them): whole trials, or groups of
+// small trials per step.  slot0 = index of the tile's first trial among the histogram slots.
+template <int RULE>
+__device__ __forceinline__ void epilogue_tile(const SweepParams &p, const SmemTail &s, int slot0, long long tile, int w, int nw,
+                                              int lane)
+{
+    const int G = p.g, seg_ints = p.hist_copies * p.hist_stride;
+    const long long t0 = tile * G;
+    if (p.epi_sub > 0) {
+        const int per_step = 32 / p.epi_sub;
+        for (int seg0 = w * per_step; seg0 < G; seg0 += nw * per_step) epilogue_small_trials<RULE>(p, s, slot0, t0, seg0, lane);
+    } else {
+        for (int seg = w; seg < G && t0 + seg < p.T; seg += nw)  // (nothing was added for trials past the last one)
+            epilogue_trial<RULE>(p, s, s.hist + (slot0 + seg) * seg_ints, s.fmax + (slot0 + seg) * seg_ints,
+                                 s.segmax + slot0 + seg, t0 + seg, lane);
+    }
+}
+
+// The epilogue warp's loop (all 32 lanes) over the block's tiles when a tile is one trial: the consumers fill
+// histogram buffer j&1 for their j-th trial and go straight on while this warp turns the other buffer into outputs.
+// (Tiles of several small trials are finished by the consumer warps themselves, see tiled_trials.)
 template <int RULE>
 __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTail &s, int lane, int ncw)
 {
-    const int K = p.K, H = p.hist_copies, HS = p.hist_stride, G = p.g;
+    if (p.nbuf == 1) return;
     const int bar_threads = ncw * 32 + 32;
-    const long long tiles = (p.T + G - 1) / G;
+    const long long tiles = (p.T + p.g - 1) / p.g;
     int j = 0;
     for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++j) {
         const int b = j & 1;
         buffer_barrier_sync<kBarReady>(b, bar_threads);  // every consumer has finished this tile
-        if (p.epi_sub > 0) {
-            // Several small trials per step: L = K/4 lanes (a power of two) take one trial, four bins each, and the
-            // scans run inside groups of L lanes; 32/L trials go through the warp at once.
-            const int L = p.epi_sub, per_step = 32 / L;
-            const int sub = lane & (L - 1), k = 4 * sub;
-            for (int seg0 = 0; seg0 < G; seg0 += per_step) {
-                const int seg = seg0 + lane / L;
-                const long long t = tile * G + seg;
-                const bool in = seg < G && t < p.T;
-                int4 h = make_int4(0, 0, 0, 0);
-                float4 fm = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                float Tmax = 0.0f;
-                if (in) {
-                    for (int c = 0; c < H; ++c) {
-                        int4 *hp = reinterpret_cast<int4 *>(s.hist + ((b * G + seg) * H + c) * HS + k);
-                        const int4 v = *hp;
-                        *hp = make_int4(0, 0, 0, 0);
-                        h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
-                        if (RULE == 1) {
-                            float4 *fp = reinterpret_cast<float4 *>(s.fmax + ((b * G + seg) * H + c) * HS + k);
-                            const float4 f = *fp;
-                            *fp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                            fm.x = fmaxf(fm.x, f.x); fm.y = fmaxf(fm.y, f.y); fm.z = fmaxf(fm.z, f.z); fm.w = fmaxf(fm.w, f.w);
-                        }
-                    }
-                    Tmax = __int_as_float(s.segmax[b * G + seg]);
-                }
-                h.y += h.x; h.z += h.y; h.w += h.z;  // inclusive inside the lane
-                int incl = h.w;
-                for (int o = 1; o < L; o <<= 1) {
-                    const int u = __shfl_up_sync(0xffffffffu, incl, o, L);
-                    if (sub >= o) incl += u;
-                }
-                const int base = incl - h.w;  // everything before this lane's bins, within its trial
-                float4 st;
-                if (RULE == 0) {
-                    const float4 tq = *reinterpret_cast<const float4 *>(s.tau_s + k);
-                    st.x = fminf(tq.x, Tmax); st.y = fminf(tq.y, Tmax); st.z = fminf(tq.z, Tmax); st.w = fminf(tq.w, Tmax);
-                } else {
-                    fm.y = fmaxf(fm.y, fm.x); fm.z = fmaxf(fm.z, fm.y); fm.w = fmaxf(fm.w, fm.z);
-                    float fincl = fm.w;
-                    for (int o = 1; o < L; o <<= 1) {
-                        const float u = __shfl_up_sync(0xffffffffu, fincl, o, L);
-                        if (sub >= o) fincl = fmaxf(fincl, u);
-                    }
-                    float before = __shfl_up_sync(0xffffffffu, fincl, 1, L);
-                    before = sub > 0 ? before : 0.0f;
-                    st.x = fmaxf(before, fm.x); st.y = fmaxf(before, fm.y); st.z = fmaxf(before, fm.z); st.w = fmaxf(before, fm.w);
-                }
-                if (in) {
-                    const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
-                    *reinterpret_cast<int4 *>(p.out_done + t * K + k) = make_int4(base + h.x, base + h.y, base + h.z, base + h.w);
-                    *reinterpret_cast<float4 *>(p.out_step + t * K + k) =
-                        make_float4(__fadd_rn(st.x, t_comm), __fadd_rn(st.y, t_comm), __fadd_rn(st.z, t_comm), __fadd_rn(st.w, t_comm));
-                    if (sub == 0) {  // the two bins past the last threshold, the trial's maximum, the synchronous time
-                        for (int c = 0; c < H; ++c) {
-                            s.hist[((b * G + seg) * H + c) * HS + K] = 0;
-                            s.hist[((b * G + seg) * H + c) * HS + K + 1] = 0;
-                            if (RULE == 1) {
-                                s.fmax[((b * G + seg) * H + c) * HS + K] = 0.0f;
-                                s.fmax[((b * G + seg) * H + c) * HS + K + 1] = 0.0f;
-                            }
-                        }
-                        s.segmax[b * G + seg] = 0;
-                        if (p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
-                    }
-                }
-            }
-            buffer_barrier_arrive<kBarFree>(b, bar_threads);  // buffer b is clear again
-            continue;
-        }
-        for (int seg = 0; seg < G; ++seg) {
-            const long long t = tile * G + seg;
-            if (t >= p.T) break;  // (nothing was added for trials past the last one)
-            int *hist = s.hist + (b * G + seg) * H * HS;
-            float *fmax = s.fmax + (b * G + seg) * H * HS;  // rule 1 only
-            const float Tmax = __int_as_float(s.segmax[b * G + seg]);
-            const float t_comm = p.t_comm_vec ? p.t_comm_vec[t] : p.t_comm;
-            float *step_row = p.out_step + t * K;
-            int32_t *done_row = p.out_done + t * K;
-            int carry = 0;
-            float fm_carry = 0.0f;
-            // Four consecutive bins per lane, 128 bins per step, with 16-byte accesses throughout (when the shapes
-            // and pointers allow): a quarter of the scans and well under half the instructions of the scalar loop.
-            for (int k0 = 0; p.epi_vec && k0 < K; k0 += 128) {
-                const int k = k0 + 4 * lane;
-                const bool in = k < K;  // K is a multiple of 4: a lane's four bins are all inside or all outside
-                int4 h = make_int4(0, 0, 0, 0);
-                float4 fm = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                if (in) {
-#pragma unroll 2
-                    for (int c = 0; c < H; ++c) {
-                        int4 *hp = reinterpret_cast<int4 *>(hist + c * HS + k);
-                        const int4 v = *hp;
-                        *hp = make_int4(0, 0, 0, 0);
-                        h.x += v.x; h.y += v.y; h.z += v.z; h.w += v.w;
-                        if (RULE == 1) {
-                            float4 *fp = reinterpret_cast<float4 *>(fmax + c * HS + k);
-                            const float4 f = *fp;
-                            *fp = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                            fm.x = fmaxf(fm.x, f.x); fm.y = fmaxf(fm.y, f.y); fm.z = fmaxf(fm.z, f.z); fm.w = fmaxf(fm.w, f.w);
-                        }
-                    }
-                }
-                h.y += h.x; h.z += h.y; h.w += h.z;  // inclusive inside the lane
-                const int incl = warp_inclusive_scan(h.w, lane);
-                const int base = carry + incl - h.w;  // everything before this lane's bins
-                carry += __shfl_sync(0xffffffffu, incl, 31);
-                float4 st;
-                if (RULE == 0) {
-                    const float4 tq = in ? *reinterpret_cast<const float4 *>(s.tau_s + k) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    st.x = fminf(tq.x, Tmax); st.y = fminf(tq.y, Tmax); st.z = fminf(tq.z, Tmax); st.w = fminf(tq.w, Tmax);
-                } else {
-                    // max_n W_n(k) = max_{j <= k} fmax[j]
-                    fm.y = fmaxf(fm.y, fm.x); fm.z = fmaxf(fm.z, fm.y); fm.w = fmaxf(fm.w, fm.z);
-                    const float fincl = warp_inclusive_max_scan(fm.w, lane);
-                    float before = __shfl_up_sync(0xffffffffu, fincl, 1);
-                    before = fmaxf(fm_carry, lane > 0 ? before : 0.0f);
-                    fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fincl, 31));
-                    st.x = fmaxf(before, fm.x); st.y = fmaxf(before, fm.y); st.z = fmaxf(before, fm.z); st.w = fmaxf(before, fm.w);
-                }
-                if (in) {
-                    *reinterpret_cast<int4 *>(done_row + k) = make_int4(base + h.x, base + h.y, base + h.z, base + h.w);
-                    *reinterpret_cast<float4 *>(step_row + k) =
-                        make_float4(__fadd_rn(st.x, t_comm), __fadd_rn(st.y, t_comm), __fadd_rn(st.z, t_comm), __fadd_rn(st.w, t_comm));
-                }
-            }
-            // Otherwise: 32 bins at a time, lane l sums bin k0+l over the copies (and clears it), a warp scan gives the
-            // prefix, a carry links the blocks of 32.
-            for (int k0 = p.epi_vec ? K : 0; k0 < K; k0 += 32) {
-                const int k = k0 + lane;
-                int h = 0;
-                float fm = 0.0f;
-                if (k < K) {
-                    for (int c = 0; c < H; ++c) {
-                        h += hist[c * HS + k];
-                        hist[c * HS + k] = 0;
-                        if (RULE == 1) {
-                            fm = fmaxf(fm, fmax[c * HS + k]);
-                            fmax[c * HS + k] = 0.0f;
-                        }
-                    }
-                }
-                const int incl = warp_inclusive_scan(h, lane);
-                float step;
-                if (RULE == 0) {
-                    step = __fadd_rn(fminf(k < K ? s.tau_s[k] : 0.0f, Tmax), t_comm);
-                } else {
-                    const float fm_incl = warp_inclusive_max_scan(fm, lane);
-                    step = __fadd_rn(fmaxf(fm_carry, fm_incl), t_comm);
-                    fm_carry = fmaxf(fm_carry, __shfl_sync(0xffffffffu, fm_incl, 31));
-                }
-                if (k < K) {
-                    done_row[k] = carry + incl;
-                    step_row[k] = step;
-                }
-                carry += __shfl_sync(0xffffffffu, incl, 31);
-            }
-            for (int c = lane; c < H; c += 32) {  // the two bins past the last threshold
-                hist[c * HS + K] = 0;
-                hist[c * HS + K + 1] = 0;
-            }
-            if (RULE == 1) {
-                for (int c = lane; c < H; c += 32) {
-                    fmax[c * HS + K] = 0.0f;
-                    fmax[c * HS + K + 1] = 0.0f;
-                }
-            }
-            if (lane == 0) {
-                s.segmax[b * G + seg] = 0;
-                if (p.out_sync != nullptr) p.out_sync[t] = __fadd_rn(Tmax, t_comm);
-            }
-        }
+        epilogue_tile<RULE>(p, s, b * p.g, tile, 0, 1, lane);
         buffer_barrier_arrive<kBarFree>(b, bar_threads);  // buffer b is clear again
     }
 }
@@ -267,9 +293,10 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
     int st = 0;
     uint32_t ph = 0;
     int j = 0;
+    const bool own_epilogue = p.nbuf == 1;  // tiles of several small trials: the consumer warps finish them themselves
     for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++j) {
-        const int b = j & 1;
-        if (j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
+        const int b = own_epilogue ? 0 : (j & 1);
+        if (!own_epilogue && j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
         int *myhist = myhist0 + b * G * seg_ints;
         unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
         const bool in_tile = (tid < p.rows) && (tile * G + seg < p.T);  // this thread's trial exists
@@ -326,7 +353,15 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
             const unsigned wm = __reduce_max_sync(0xffffffffu, (unsigned)__float_as_int(rowmax));
             if (lane == 0) atomicMax(&s.segmax[b], (int)wm);
         }
-        buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
+        if (own_epilogue) {
+            // every consumer has added its rows; each warp then turns a share of the tile's trials into outputs and
+            // clears their histograms; nobody starts the next tile before all of that is done
+            bar_sync_imm<kConsumerBarrier>(ncw * 32);
+            epilogue_tile<RULE>(p, s, 0, tile, warp, ncw, lane);
+            bar_sync_imm<kConsumerBarrier>(ncw * 32);
+        } else {
+            buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
+        }
     }
 }
 

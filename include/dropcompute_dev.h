@@ -42,6 +42,8 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  *                        row is full (tiled kernel)
  *   DC_TUNE_TILE_TRIALS  the most trials of few workers (N <= 128) that may share one tile of the tiled kernel
  *                        (1 = one trial per tile)
+ *   DC_TUNE_WHOLE_LINES  1 = rows shorter than 128 bytes are always fetched row by row, 2 (and 0) = as whole
+ *                        128-byte lines wherever the passes of every trial start and end on a line (tiled kernel)
  * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
  */
 #define DC_TUNE_STAGES 1
@@ -56,6 +58,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
 #define DC_TUNE_FLAT_MAX_M 11
 #define DC_TUNE_LEAN_LOOP 12
 #define DC_TUNE_TILE_TRIALS 13
+#define DC_TUNE_WHOLE_LINES 14
 int dc_tune(int32_t key, int32_t value);
 
 /*

@@ -129,6 +129,7 @@ struct Tune {
     int flat_max_m = 0;    // 0 = automatic (kFlatAutoMaxM), else the longest row the flat kernel is given (<= kFlatMaxM)
     int flat_tile_warps = 0, flat_groups = 0, flat_depth = 0;  // flat kernel; all three or none
     int lean = 0;          // 0 = automatic (on), 1 = off, 2 = on: the short consumer loop for rows of full chunks
+    int whole_lines = 0;   // 0 = automatic (on), 1 = off: rows shorter than 128 bytes fetched as whole 128-byte lines
     int tile_trials = 0;   // 0 = automatic, else the most trials of few workers that share a tile
 };
 std::mutex g_tune_lock;
@@ -396,6 +397,34 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         if (p.pitch == 128) { swz = CU_TENSOR_MAP_SWIZZLE_128B; p.swz_mask = 7; }
         else if (p.pitch == 64) { swz = CU_TENSOR_MAP_SWIZZLE_64B; p.swz_mask = 3; }
         else if (p.pitch == 32) { swz = CU_TENSOR_MAP_SWIZZLE_32B; p.swz_mask = 1; }
+        p.box_y = p.rows;
+        // Rows shorter than a 128-byte line: consecutive rows are contiguous in memory, so when every pass of every
+        // trial starts and ends on a line the tensor is described to the copy unit as lines of 32 floats and a tile
+        // is so many whole lines (a quarter to an eighth of the requests of row-sized pieces).  The tile in shared
+        // memory is the same dense copy of its rows; of "no swizzle" and the 128-byte swizzle the one with fewer
+        // bank conflicts for "lane r reads 16 bytes of row r" is taken.
+        const bool whole_lines = tune.whole_lines != 1 && M < 32 && (N * M) % 32 == 0 && ((int64_t)p.rows * M) % 32 == 0 &&
+                                 (p.g > 1 || N % p.rows == 0);
+        if (whole_lines) {
+            int worst[2] = {0, 0};
+            for (int mode = 0; mode < 2; ++mode) {
+                for (int q = 0; q < nq; ++q) {
+                    for (int r0 = 0; r0 < 32 && r0 < p.rows; r0 += 8) {
+                        int hits[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                        for (int r = r0; r < r0 + 8 && r < p.rows; ++r) {
+                            unsigned chunk = (unsigned)(r * (int)M / 4 + q);
+                            if (mode == 1) chunk ^= (chunk >> 3) & 7u;
+                            const int hcount = ++hits[chunk & 7u];
+                            if (hcount > worst[mode]) worst[mode] = hcount;
+                        }
+                    }
+                }
+            }
+            const bool use_swizzle = worst[1] < worst[0];
+            swz = use_swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE;
+            p.swz_mask = use_swizzle ? 7 : 0;
+            p.box_y = (int)((int64_t)p.rows * M / 32);
+        }
         p.stage_bytes = ((p.rows * p.pitch + 1023) / 1024) * 1024;
         size_t smem = 0;
         {
@@ -404,9 +433,16 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         }
 
         CUtensorMap map;
-        const cuuint64_t gdim[3] = {(cuuint64_t)M, (cuuint64_t)N, (cuuint64_t)T};
-        const cuuint64_t gstride[2] = {(cuuint64_t)M * 4, (cuuint64_t)N * (cuuint64_t)M * 4};
-        const cuuint32_t box[3] = {(cuuint32_t)p.bw, (cuuint32_t)(p.g > 1 ? N : p.rows), (cuuint32_t)p.g};
+        cuuint64_t gdim[3] = {(cuuint64_t)M, (cuuint64_t)N, (cuuint64_t)T};
+        cuuint64_t gstride[2] = {(cuuint64_t)M * 4, (cuuint64_t)N * (cuuint64_t)M * 4};
+        cuuint32_t box[3] = {(cuuint32_t)p.bw, (cuuint32_t)(p.g > 1 ? N : p.rows), (cuuint32_t)p.g};
+        if (whole_lines) {  // [T][N*M/32 lines][32 floats]
+            gdim[0] = 32;
+            gdim[1] = (cuuint64_t)(N * M / 32);
+            gstride[0] = 128;
+            box[0] = 32;
+            box[1] = (cuuint32_t)((p.g > 1 ? N : (int64_t)p.rows) * M / 32);
+        }
         const cuuint32_t estr[3] = {1, 1, 1};
         if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(lat), gdim, gstride, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -954,6 +990,10 @@ int dc_tune(int32_t key, int32_t value)
     }
     if (key == DC_TUNE_LEAN_LOOP && value >= 0 && value <= 2) {
         tune.lean = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_WHOLE_LINES && value >= 0 && value <= 2) {
+        tune.whole_lines = value;
         return DC_OK;
     }
     if (key == DC_TUNE_TILE_TRIALS && value >= 0 && value <= kMaxRowsPerPass) {

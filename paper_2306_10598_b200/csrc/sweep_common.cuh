@@ -60,6 +60,8 @@ struct SweepParams {
     int short_launch;  // host only: under 1 GiB of latencies (see simulate_impl)
     int epi_vec;       // staged kernels: the epilogue warp may take four bins per lane with 16-byte accesses
                        // (K a multiple of 4, out_step / out_done 16-byte aligned, hist_stride a multiple of 4)
+    int box_y;         // tiled kernel: height of one pass in the tensor map's second coordinate (rows, or 128-byte lines
+                       // when rows shorter than a line are fetched as whole lines)
     int g;             // staged kernels: trials per tile (several whole trials of few workers share a tile; else 1)
     int epi_sub;       // tiled kernel, g > 1: lanes of the epilogue warp per trial (K/4, a power of two), or 0 for one
                        // trial at a time

@@ -280,12 +280,16 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
     const int seg = G > 1 ? row / p.N : 0;
     const int copy = (warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1));
     int *myhist0 = s.hist + seg * seg_ints + copy * p.hist_stride;
-    // byte offset of this thread's quad q inside a stage: row_off + ((16 q) ^ swz)
+    // Byte offset of this thread's quad q inside a stage.  The tile is a dense copy of its rows; the hardware
+    // swizzle XORs bits 4..6 of an offset with (bits 7..9 & swz_mask), which moves 16-byte quads inside 128-byte lines
+    // (rows may be shorter than a line, or not a divisor of it, when they are fetched as whole lines).
     const uint32_t row_off = (uint32_t)row * (uint32_t)p.pitch;
-    const uint32_t swz = ((row_off >> 7) & (uint32_t)p.swz_mask) << 4;
     uint32_t qoff[NQ];
 #pragma unroll
-    for (int q = 0; q < NQ; ++q) qoff[q] = row_off + ((uint32_t)(q * 16) ^ swz);
+    for (int q = 0; q < NQ; ++q) {
+        const uint32_t o = row_off + (uint32_t)(q * 16);
+        qoff[q] = o ^ (((o >> 7) & (uint32_t)p.swz_mask) << 4);
+    }
     // the spare histogram copy (after all real ones, never read): where lanes without a row of their own add
     const uint32_t spare_a = smem_addr(s.hist + (hist_slots(p) - 1) * p.hist_stride);
     const uint32_t stage0_a = smem_addr(stage0);
@@ -391,7 +395,7 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     int prod_pass = 0, prod_c = 0, prod_issued = 0;
     auto issue_tile = [&](int st) {
         mbar_arrive_expect_tx(&full[st], (uint32_t)(p.rows * p.pitch));
-        tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, prod_c * p.bw, prod_pass * p.rows, (int)(prod_t * p.g), &full[st]);
+        tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, prod_c * p.bw, prod_pass * p.box_y, (int)(prod_t * p.g), &full[st]);
         if (++prod_c == p.chunks) {
             prod_c = 0;
             if (++prod_pass == p.passes) {

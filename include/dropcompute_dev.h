@@ -44,6 +44,8 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  *                        (1 = one trial per tile)
  *   DC_TUNE_WHOLE_LINES  1 = rows shorter than 128 bytes are always fetched row by row, 2 (and 0) = as whole
  *                        128-byte lines wherever the passes of every trial start and end on a line (tiled kernel)
+ *   DC_TUNE_EVEN_GRID    1 (and 0) = as many blocks as the GPU holds at once, 2 = the fewest blocks that need no more
+ *                        rounds over the trials than that (tiled kernel)
  * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
  */
 #define DC_TUNE_STAGES 1
@@ -59,6 +61,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
 #define DC_TUNE_LEAN_LOOP 12
 #define DC_TUNE_TILE_TRIALS 13
 #define DC_TUNE_WHOLE_LINES 14
+#define DC_TUNE_EVEN_GRID 15
 int dc_tune(int32_t key, int32_t value);
 
 /*

@@ -98,14 +98,15 @@ bool device_info(DeviceInfo *out)
     return true;
 }
 
-// Blocks for `units` equal pieces of work (trials, or tiles of several trials) that the blocks take round-robin:
-// no more than `resident` (what fits the GPU at once), and of those the FEWEST that still finish in the same number
-// of rounds.  The last round then has no idle blocks to wait for, and a bandwidth-bound kernel loses nothing by
-// running on a few blocks less (4096 trials on 444 resident blocks: ten rounds either way; 410 blocks all work
-// through all ten, whereas with 444 blocks 344 of them sit out the tenth).
-long long even_grid(long long units, long long resident)
+// Blocks for `units` equal pieces of work (trials, or tiles of several trials) that the blocks take round-robin: as
+// many as fit the GPU at once (`resident`).  mode 2 (DC_TUNE_EVEN_GRID) takes the FEWEST blocks that still finish in
+// the same number of rounds instead, so that no block sits out the last round; that pays only where the kernel is
+// bound by memory bandwidth alone, and measured 0-8 % slower on the workloads here, whose blocks are bound by their
+// own pace: the blocks left over in the last round run faster when they have the GPU to themselves.
+long long even_grid(long long units, long long resident, int mode = 0)
 {
     if (units <= resident) return units;
+    if (mode != 2) return resident;
     const long long rounds = (units + resident - 1) / resident;
     return (units + rounds - 1) / rounds;
 }
@@ -130,6 +131,7 @@ struct Tune {
     int flat_tile_warps = 0, flat_groups = 0, flat_depth = 0;  // flat kernel; all three or none
     int lean = 0;          // 0 = automatic (on), 1 = off, 2 = on: the short consumer loop for rows of full chunks
     int whole_lines = 0;   // 0 = automatic (on), 1 = off: rows shorter than 128 bytes fetched as whole 128-byte lines
+    int even_grid = 0;     // 0 = automatic (1), 1 = as many blocks as fit the GPU, 2 = the fewest blocks with as many rounds
     int tile_trials = 0;   // 0 = automatic, else the most trials of few workers that share a tile
 };
 std::mutex g_tune_lock;
@@ -211,7 +213,7 @@ int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size
             last[dev].occ = occ;
         }
     }
-    const long long grid = even_grid(T, (long long)occ * di.sms);
+    const long long grid = even_grid(T, (long long)occ * di.sms, p.grid_mode);
     kernel<<<(unsigned)grid, block, smem, stream>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }
@@ -344,6 +346,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
     p.batch_lookups = 0;
     p.rule = rule;
     p.aux_copies = rule == DC_RULE_START_BEFORE_TAU ? p.hist_copies : 0;
+    p.grid_mode = tune.even_grid;
 
     if (tiled_ok(lat, M)) {
         EncodeTiledFn encode = get_encode_fn();
@@ -990,6 +993,10 @@ int dc_tune(int32_t key, int32_t value)
     }
     if (key == DC_TUNE_LEAN_LOOP && value >= 0 && value <= 2) {
         tune.lean = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_EVEN_GRID && value >= 0 && value <= 2) {
+        tune.even_grid = value;
         return DC_OK;
     }
     if (key == DC_TUNE_WHOLE_LINES && value >= 0 && value <= 2) {

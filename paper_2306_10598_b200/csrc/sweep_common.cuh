@@ -58,6 +58,7 @@ struct SweepParams {
     int tile_warps;    // flat kernel: warps per group (rows / 32)
     int direct_bins;   // staged kernels: 1 = bin evenly spaced thresholds arithmetically instead of through the table
     int short_launch;  // host only: under 1 GiB of latencies (see simulate_impl)
+    int grid_mode;     // host only: DC_TUNE_EVEN_GRID
     int epi_vec;       // staged kernels: the epilogue warp may take four bins per lane with 16-byte accesses
                        // (K a multiple of 4, out_step / out_done 16-byte aligned, hist_stride a multiple of 4)
     int box_y;         // tiled kernel: height of one pass in the tensor map's second coordinate (rows, or 128-byte lines

@@ -185,11 +185,11 @@ int launch_flat(const SweepParams &p, int block, size_t smem, long long T, const
     return launch_flat_q<RULE, BATCH, 8>(p, block, smem, T, di, stream);
 }
 
-template <int NQ, int RULE, bool BATCH>
+template <int NQ, int RULE, bool BATCH, bool WIDE = false>
 int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
                    cudaStream_t stream)
 {
-    auto kernel = dc_sweep_tiled<NQ, RULE, BATCH>;
+    auto kernel = dc_sweep_tiled<NQ, RULE, BATCH, WIDE>;
     // Per instantiation and device: the largest dynamic shared memory opted into so far, and the occupancy of
     // the last (block, smem) asked for -- repeated calls with one shape then cost no runtime queries.
     static std::mutex lock;
@@ -222,7 +222,16 @@ template <int NQ, int RULE>
 int launch_tiled(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
                  cudaStream_t stream)
 {
-    // rule 1 has one binning path only
+    // rule 1 has one binning path only; tiles of two whole trials are compiled for chunks of 12 and 16 floats
+    if constexpr (NQ == 3 || NQ == 4) {
+        if (block > kMaxRowsPerPass + 64) {
+            if constexpr (RULE == 0) {
+                if (p.batch_lookups) return launch_tiled_b<NQ, RULE, true, true>(map, p, block, smem, T, di, stream);
+            }
+            return launch_tiled_b<NQ, RULE, false, true>(map, p, block, smem, T, di, stream);
+        }
+    }
+    if (block > kMaxRowsPerPass + 64) return DC_ERR_RANGE;
     if constexpr (RULE == 0) {
         if (p.batch_lookups) return launch_tiled_b<NQ, RULE, true>(map, p, block, smem, T, di, stream);
     }
@@ -392,6 +401,18 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
                 p.g = (int)g;
                 p.passes = 1;
                 p.rows = (int)(g * N);
+            }
+        } else if (N < kMaxRowsPerPass && (nq_inst == 3 || nq_inst == 4) && p.chunks == 1 && tune.tile_trials != 1 &&
+                   T >= 8 * (int64_t)di.sms && K <= 512) {
+            // Two whole trials per tile when that leaves clearly fewer idle lanes than one (200 workers: 24 of 224
+            // lanes idle alone, 16 of 416 as a pair).  Rows of one chunk only: measured 3-6 % faster there (200
+            // workers, 12 and 16 samples), level or slower on rows of two chunks.
+            const double idle1 = 1.0 - (double)N / (double)(((N + 31) / 32) * 32);
+            const double idle2 = 1.0 - (double)(2 * N) / (double)(((2 * N + 31) / 32) * 32);
+            if (idle1 - idle2 >= 0.04) {
+                p.g = 2;
+                p.passes = 1;
+                p.rows = (int)(2 * N);
             }
         }
         const int row_threads_t = ((p.rows + 31) / 32) * 32;

@@ -369,8 +369,10 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
     }
 }
 
-template <int NQ, int RULE, bool BATCH>
-__global__ void __launch_bounds__(kMaxRowsPerPass + 64, NQ <= 4 ? 3 : 2)
+// WIDE = tiles of two trials of 129-256 workers each (up to 512 rows, 16 consumer warps): fewer idle lanes in the last
+// warp of a trial and half the hand-overs per trial.
+template <int NQ, int RULE, bool BATCH, bool WIDE>
+__global__ void __launch_bounds__(WIDE ? 2 * kMaxRowsPerPass + 64 : kMaxRowsPerPass + 64, WIDE ? 2 : (NQ <= 4 ? 3 : 2))
 dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 {
     extern __shared__ unsigned char smem_raw[];

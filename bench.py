@@ -457,7 +457,11 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
-    ap.add_argument("--workload", default="bandwidth_stress", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--workload", default="bandwidth_stress",
+                    help="one of " + ", ".join(sorted(W.WORKLOADS)) + "; or c3:<law> for the paper's own synthetic setting "
+                         "(App. C.3: 12 accumulations of 0.45 s + eps; laws: " + ", ".join(sorted(W.C3_NOISE)) +
+                         "), or b1 (App. B.1 delay); these two take --workers and --trials")
+    ap.add_argument("--workers", type=int, default=200, help="workers N of a c3:<law> or b1 workload")
     ap.add_argument("--trials", type=int, default=0, help="override the number of trials (profiling small cases)")
     ap.add_argument("--rule", type=int, default=0, choices=(0, 1),
                     help="completion rule: 0 = Algorithm 2 (finish before tau, the benchmark), 1 = start before tau")
@@ -467,9 +471,18 @@ def main():
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="skip the extra per-workload sweep timings that the default run adds to its JSON line")
     args = ap.parse_args()
-    w = W.WORKLOADS[args.workload]
-    if args.trials:
-        w = w.with_trials(args.trials)
+    if args.workload.startswith("c3:"):
+        w = W.c3_workload(args.workload[3:], N=args.workers, T=args.trials or 16384)
+        args.trials = w.T
+    elif args.workload == "b1":
+        w = W.b1_workload(N=args.workers, T=args.trials or 16384)
+        args.trials = w.T
+    else:
+        if args.workload not in W.WORKLOADS:
+            ap.error(f"unknown workload {args.workload!r}")
+        w = W.WORKLOADS[args.workload]
+        if args.trials:
+            w = w.with_trials(args.trials)
     if args.impl == "reference":
         return run_reference(args, w)
     return run_ours(args, w)

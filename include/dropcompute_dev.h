@@ -46,6 +46,8 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
  *                        128-byte lines wherever the passes of every trial start and end on a line (tiled kernel)
  *   DC_TUNE_EVEN_GRID    1 (and 0) = as many blocks as the GPU holds at once, 2 = the fewest blocks that need no more
  *                        rounds over the trials than that (tiled kernel)
+ *   DC_TUNE_L2_PROMOTION granularity at which the copy unit's reads are promoted in L2: 1 = none, 2 = 64, 3 = 128,
+ *                        4 (and 0) = 256 bytes (tiled kernel)
  * Returns DC_ERR_UNSUPPORTED for an unknown key or value.
  */
 #define DC_TUNE_STAGES 1
@@ -62,6 +64,7 @@ int dc_simulate_plan(const float *latencies, int64_t T, int64_t N, int64_t M, in
 #define DC_TUNE_TILE_TRIALS 13
 #define DC_TUNE_WHOLE_LINES 14
 #define DC_TUNE_EVEN_GRID 15
+#define DC_TUNE_L2_PROMOTION 16
 int dc_tune(int32_t key, int32_t value);
 
 /*

@@ -302,7 +302,7 @@ def dc_sweep_host(latencies_host: torch.Tensor, taus_host: torch.Tensor, t_comm:
 
 TUNE_STAGES, TUNE_LANE_COPIES, TUNE_WARP_GROUPS, TUNE_BOX_FLOATS, TUNE_BATCH_LOOKUPS, TUNE_DIRECT_BINS = 1, 2, 3, 4, 5, 6
 TUNE_FLAT_TILE_WARPS, TUNE_FLAT_GROUPS, TUNE_FLAT_DEPTH, TUNE_FLAT_MAX_M = 7, 8, 9, 11
-TUNE_LEAN_LOOP, TUNE_TILE_TRIALS, TUNE_WHOLE_LINES, TUNE_EVEN_GRID = 12, 13, 14, 15
+TUNE_LEAN_LOOP, TUNE_TILE_TRIALS, TUNE_WHOLE_LINES, TUNE_EVEN_GRID, TUNE_L2_PROMOTION = 12, 13, 14, 15, 16
 
 
 def dc_tune(key: int, value: int) -> None:

@@ -131,6 +131,7 @@ struct Tune {
     int flat_tile_warps = 0, flat_groups = 0, flat_depth = 0;  // flat kernel; all three or none
     int lean = 0;          // 0 = automatic (on), 1 = off, 2 = on: the short consumer loop for rows of full chunks
     int whole_lines = 0;   // 0 = automatic (on), 1 = off: rows shorter than 128 bytes fetched as whole 128-byte lines
+    int l2_promotion = 0;  // 0 = automatic (256 bytes), 1 = none, 2 = 64, 3 = 128, 4 = 256 bytes
     int even_grid = 0;     // 0 = automatic (1), 1 = as many blocks as fit the GPU, 2 = the fewest blocks with as many rounds
     int tile_trials = 0;   // 0 = automatic, else the most trials of few workers that share a tile
 };
@@ -469,7 +470,10 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         }
         const cuuint32_t estr[3] = {1, 1, 1};
         if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(lat), gdim, gstride, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                   tune.l2_promotion == 1 ? CU_TENSOR_MAP_L2_PROMOTION_NONE
+                   : tune.l2_promotion == 2 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
+                   : tune.l2_promotion == 3 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return DC_ERR_CUDA;
 
@@ -1014,6 +1018,10 @@ int dc_tune(int32_t key, int32_t value)
     }
     if (key == DC_TUNE_LEAN_LOOP && value >= 0 && value <= 2) {
         tune.lean = value;
+        return DC_OK;
+    }
+    if (key == DC_TUNE_L2_PROMOTION && value >= 0 && value <= 4) {
+        tune.l2_promotion = value;
         return DC_OK;
     }
     if (key == DC_TUNE_EVEN_GRID && value >= 0 && value <= 2) {

@@ -386,6 +386,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         p.pitch = p.bw * 4;
         const int nq = p.bw / 4;
         // the kernel is compiled for 1, 2, 3, 4, 6 and 8 quads per chunk; other chunk lengths run in the next size up
+        // (each further size costs a quarter more build time and measured 3 % on the rows it would serve)
         const int nq_inst = nq <= 4 ? nq : (nq <= 6 ? 6 : 8);
         p.lean = (tune.lean != 1 && last_cols == p.bw && nq == nq_inst) ? 1 : 0;
         // Several whole trials of few workers share a tile: g trials of N rows each, g N <= 256, as many as it takes

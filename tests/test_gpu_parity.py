@@ -82,8 +82,9 @@ EDGE_SHAPES = [
     (1000, 8, 4, 16), (1000, 8, 12, 16), (1000, 8, 32, 7), (333, 5, 4, 33), (333, 5, 12, 64), (333, 5, 32, 9),
     (77, 33, 4, 16), (77, 33, 12, 40), (77, 33, 32, 128), (50, 128, 4, 5), (50, 128, 12, 64), (50, 128, 32, 256),
     (5000, 3, 8, 20), (700, 1, 16, 4), (900, 100, 48, 64), (650, 64, 36, 30),
-    # row lengths cut into equal chunks of 12, 16 or 24 floats (36, 48, 72, 80) and one that is not (100)
-    (6, 300, 48, 40), (5, 256, 72, 64), (4, 150, 80, 33), (40, 260, 36, 50),
+    # row lengths cut into equal chunks of 12, 16 or 24 floats (36, 48, 72, 80) and ones that are not (100, 56, 44, 88, 20, 28)
+    (6, 300, 48, 40), (5, 256, 72, 64), (4, 150, 80, 33), (40, 260, 36, 50), (7, 200, 100, 64), (5, 90, 56, 20),
+    (6, 130, 44, 30), (3, 70, 88, 64), (9, 64, 20, 16), (9, 64, 28, 16),
 ]
 
 

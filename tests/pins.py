@@ -252,7 +252,7 @@ def pin_per_iteration_comm(lib, order="rows"):
 
 def pin_fp32_left_to_right(lib, order="rows"):
     """The running sum is binary32 with one rounding per addition, taken m = 1..M in order
-    (Algorithm 2's inner loop; the precision is this build's reading)."""
+    (Algorithm 2's inner loop; the precision is a reading taken where the paper is silent)."""
     e = 2.0 ** -24
     nxt = np.float32(1.0 + 2.0 ** -23)
     # 1 + 2^-24 ties to even = 1, three times over: the sum never leaves 1.0

@@ -67,7 +67,7 @@ def _bind(lib):
     p = ctypes.c_void_p
     for name in ("dco_sweep_definition", "dco_sweep_rows"):
         fn = getattr(lib, name)
-        fn.argtypes = [p, i64, i64, i64, p, i64, f32, p, i32, p, p, p]
+        fn.argtypes = [p, i64, i64, i64, p, i64, f32, p, i32, p, p, p, p]
         fn.restype = i32
     lib.dco_reduce_trials.argtypes = [p, p, p, i64, i64, i64, i64, p, p]
     lib.dco_reduce_trials.restype = i32
@@ -123,13 +123,14 @@ def _f32c(a, ndim):
     return a
 
 
-def sweep(lat, taus, t_comm: float, rule: int = 0, order: str = "rows", lib=None) -> Sweep:
+def sweep(lat, taus, t_comm: float, rule: int = 0, order: str = "rows", lib=None, worker_scale=None) -> Sweep:
     """Per-(iteration, tau) step time and completed count.
 
     ``order='definition'`` writes out each iteration's table of finish times and reads every quantity off
     it, one threshold at a time (Sec. 4.3's definitions as they stand);
     ``order='rows'`` reads every sample once (same predicate, same integers).
-    ``t_comm`` is one number, or an array of T numbers (Algorithm 2's per-iteration T_i^c)."""
+    ``t_comm`` is one number, or an array of T numbers (Algorithm 2's per-iteration T_i^c).
+    ``worker_scale``: None, or N positive numbers s_n: worker n works against its own threshold s_n * tau_k."""
     lib = lib or load()
     lat = _f32c(lat, 3)
     taus = _f32c(taus, 1)
@@ -143,8 +144,12 @@ def sweep(lat, taus, t_comm: float, rule: int = 0, order: str = "rows", lib=None
     if np.ndim(t_comm) > 0:
         tc_vec = np.ascontiguousarray(t_comm, dtype=np.float32)
         assert tc_vec.shape == (T,)
+    sc = None
+    if worker_scale is not None:
+        sc = np.ascontiguousarray(worker_scale, dtype=np.float32)
+        assert sc.shape == (N,)
     rc = fn(lat.ctypes.data, T, N, M, taus.ctypes.data, K, np.float32(0.0 if tc_vec is not None else t_comm),
-            None if tc_vec is None else tc_vec.ctypes.data, rule,
+            None if tc_vec is None else tc_vec.ctypes.data, rule, None if sc is None else sc.ctypes.data,
             step.ctypes.data, done.ctypes.data, sync.ctypes.data)
     if rc != 0:
         raise ValueError(f"oracle sweep failed with status {rc}")

@@ -25,6 +25,11 @@
  *   - statistics over iterations are binary64;
  *   - argmax takes the first maximum and never selects a NaN.
  *
+ * Heterogeneous workers (App. C.2 remarks that workers may differ, each with its own mu_n, sigma_n): optionally
+ * worker n works against its own threshold s_n * tau_k (one binary32 product) instead of the common tau_k; its time
+ * is then min{s_n tau_k, T_n} and the step takes the maximum of those over workers.  With all s_n = 1 this is the
+ * common-threshold case bit for bit.
+ *
  * rule 0 is the paper's (a micro-batch counts iff it FINISHES before tau).
  * rule 1 is the variant described in the paper's Limitations paragraph, where
  * the timeout is only looked at between accumulations: a micro-batch is run
@@ -70,7 +75,7 @@
  * ------------------------------------------------------------------------- */
 int dco_sweep_definition(const float *lat, int64_t T, int64_t N, int64_t M,
                          const float *taus, int64_t K, float t_comm, const float *t_comm_per_iter, int rule,
-                         float *out_step, int32_t *out_done, float *out_sync)
+                         const float *worker_scale, float *out_step, int32_t *out_done, float *out_sync)
 {
     if (!lat || !taus || !out_step || !out_done || !out_sync) return 1;
     if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return 2;
@@ -91,7 +96,34 @@ int dco_sweep_definition(const float *lat, int64_t T, int64_t N, int64_t M,
         float slowest_full = 0.0f; /* T = max_n T_n^{(M)} */
         for (int64_t n = 0; n < N; ++n) slowest_full = fmaxf(slowest_full, finish[n * M + (M - 1)]);
         out_sync[i] = slowest_full + tc;
-        for (int64_t k = 0; k < K; ++k) {
+        for (int64_t k = 0; k < K && worker_scale; ++k) {
+            /* heterogeneous workers: worker n works against its own threshold s_n * tau_k (one binary32 product) */
+            int64_t completed = 0;
+            float slowest = 0.0f; /* max_n of the worker's time under its threshold */
+            for (int64_t n = 0; n < N; ++n) {
+                const float *f = finish + n * M;
+                const float own_tau = worker_scale[n] * taus[k];
+                float worker_time;
+                if (rule == 0) {
+                    for (int64_t m = 0; m < M; ++m) completed += (f[m] < own_tau) ? 1 : 0;
+                    worker_time = fminf(own_tau, f[M - 1]); /* min{tau, T_n} of Sec. 4.3, per worker */
+                } else {
+                    int64_t last_run = -1;
+                    for (int64_t m = 0; m < M; ++m) {
+                        const float start = (m == 0) ? 0.0f : f[m - 1];
+                        if (start < own_tau) {
+                            completed += 1;
+                            last_run = m;
+                        }
+                    }
+                    worker_time = last_run >= 0 ? f[last_run] : 0.0f;
+                }
+                slowest = (n == 0) ? worker_time : fmaxf(slowest, worker_time);
+            }
+            out_done[i * K + k] = (int32_t)completed;
+            out_step[i * K + k] = slowest + tc;
+        }
+        for (int64_t k = 0; k < K && !worker_scale; ++k) {
             const float tau = taus[k];
             int64_t completed = 0;
             float slowest_cut = 0.0f; /* rule 1: max_n (finish time of the last micro-batch worker n ran) */
@@ -130,7 +162,7 @@ int dco_sweep_definition(const float *lat, int64_t T, int64_t N, int64_t M,
  * ------------------------------------------------------------------------- */
 int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
                    const float *taus, int64_t K, float t_comm, const float *t_comm_per_iter, int rule,
-                   float *out_step, int32_t *out_done, float *out_sync)
+                   const float *worker_scale, float *out_step, int32_t *out_done, float *out_sync)
 {
     if (!lat || !taus || !out_step || !out_done || !out_sync) return 1;
     if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return 2;
@@ -141,17 +173,42 @@ int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
         int64_t *cnt = (int64_t *)malloc((size_t)K * sizeof(int64_t));
         float *wmax = (float *)malloc((size_t)K * sizeof(float));   /* rule 1: slowest worker's time per threshold */
         float *wlast = (float *)malloc((size_t)K * sizeof(float));  /* rule 1: this worker's time per threshold */
-        if (!cnt || !wmax || !wlast) {
+        float *own = (float *)malloc((size_t)K * sizeof(float));    /* heterogeneous workers: this worker's thresholds */
+        if (!cnt || !wmax || !wlast || !own) {
 #pragma omp atomic write
             failed = 1;
         }
 #pragma omp for schedule(dynamic, 1)
         for (int64_t i = 0; i < T; ++i) {
-            if (!cnt || !wmax || !wlast) continue;
+            if (!cnt || !wmax || !wlast || !own) continue;
             const float tc = t_comm_per_iter ? t_comm_per_iter[i] : t_comm;
             float slowest_full = 0.0f;
             for (int64_t k = 0; k < K; ++k) { cnt[k] = 0; wmax[k] = 0.0f; }
-            for (int64_t n = 0; n < N; ++n) {
+            for (int64_t n = 0; n < N && worker_scale; ++n) {
+                /* heterogeneous workers: worker n against its own thresholds s_n * tau_k; wmax[k] collects the
+                 * maximum over workers of each worker's time under its threshold (both rules) */
+                const float *row = lat + (i * N + n) * M;
+                float elapsed = 0.0f;
+                for (int64_t k = 0; k < K; ++k) { own[k] = worker_scale[n] * taus[k]; wlast[k] = 0.0f; }
+                for (int64_t m = 0; m < M; ++m) {
+                    const float start = elapsed;
+                    elapsed = elapsed + row[m];
+                    for (int64_t k = 0; k < K; ++k) {
+                        if (rule == 0) {
+                            cnt[k] += (elapsed < own[k]) ? 1 : 0;
+                        } else if (start < own[k]) {
+                            cnt[k] += 1;
+                            wlast[k] = elapsed;
+                        }
+                    }
+                }
+                slowest_full = fmaxf(slowest_full, elapsed);
+                for (int64_t k = 0; k < K; ++k) {
+                    const float worker_time = (rule == 0) ? fminf(own[k], elapsed) : wlast[k];
+                    wmax[k] = (n == 0) ? worker_time : fmaxf(wmax[k], worker_time);
+                }
+            }
+            for (int64_t n = 0; n < N && !worker_scale; ++n) {
                 const float *row = lat + (i * N + n) * M;
                 float elapsed = 0.0f;
                 if (rule == 1) for (int64_t k = 0; k < K; ++k) wlast[k] = 0.0f;
@@ -175,13 +232,17 @@ int dco_sweep_rows(const float *lat, int64_t T, int64_t N, int64_t M,
             }
             out_sync[i] = slowest_full + tc;
             for (int64_t k = 0; k < K; ++k) {
-                out_step[i * K + k] = (rule == 0) ? (fminf(taus[k], slowest_full) + tc) : (wmax[k] + tc);
+                if (worker_scale)
+                    out_step[i * K + k] = wmax[k] + tc;
+                else
+                    out_step[i * K + k] = (rule == 0) ? (fminf(taus[k], slowest_full) + tc) : (wmax[k] + tc);
                 out_done[i * K + k] = (int32_t)cnt[k];
             }
         }
         free(cnt);
         free(wmax);
         free(wlast);
+        free(own);
     }
     return failed ? 6 : 0;
 }

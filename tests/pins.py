@@ -28,10 +28,10 @@ def _np(t):
     return t.numpy() if hasattr(t, "numpy") else np.asarray(t)
 
 
-def _stats(lib, lat, taus, t_comm, rule=0, order="rows"):
+def _stats(lib, lat, taus, t_comm, rule=0, order="rows", worker_scale=None):
     lat = _np(lat)
     T, N, M = lat.shape
-    sw = oracle.sweep(lat, taus, t_comm, rule=rule, order=order, lib=lib)
+    sw = oracle.sweep(lat, taus, t_comm, rule=rule, order=order, lib=lib, worker_scale=worker_scale)
     st = oracle.reduce_trials(sw.step, sw.done, sw.sync, N, M, lib=lib)
     return sw, st
 
@@ -405,6 +405,69 @@ def pin_bailey_against_quadrature(lib, order="rows"):
     assert abs(oracle.bailey_mean_max(0.5, 0.2, 9, 400, lib=lib) - (0.6 * z + 4.5)) <= 1e-12
 
 
+def pin_worker_scales(lib, order="rows"):
+    """Heterogeneous workers (App. C.2: workers may differ): worker n works against its own threshold s_n tau_k, its
+    time is min{s_n tau_k, T_n} (Sec. 4.3, per worker) and the step is the slowest worker's time plus T^c.
+    Exhaustive enumeration in rational arithmetic with dyadic scales (every product exact), the all-ones case equal
+    to the common-threshold code bit for bit, and a worker whose latencies and scale are both doubled keeps its
+    decisions."""
+    vals = [Fraction(1, 4), Fraction(1, 2)]
+    t_comm = Fraction(1, 8)
+    taus = [Fraction(-1, 4), Fraction(1, 8), Fraction(1, 4), Fraction(1, 2), Fraction(3, 4), Fraction(1), Fraction(3, 2), Fraction(4)]
+    for (N, M, scales), rule in itertools.product((((2, 3, (Fraction(1), Fraction(1, 2)))), (3, 2, (Fraction(2), Fraction(1), Fraction(1, 2))),
+                                                   (1, 3, (Fraction(1, 2),))), (0, 1)):
+        outcomes = list(itertools.product(vals, repeat=N * M))
+        T = len(outcomes)
+        want_done, want_step = [], []
+        for o in outcomes:
+            finish = [list(itertools.accumulate(o[n * M:(n + 1) * M])) for n in range(N)]
+            d_row, s_row = [], []
+            for tau in taus:
+                d, times = 0, []
+                for n, f in enumerate(finish):
+                    own = scales[n] * tau
+                    if rule == 0:
+                        d += sum(1 for x in f if x < own)
+                        times.append(min(own, f[-1]))
+                    else:
+                        start = [Fraction(0)] + f[:-1]
+                        ran = [x for b, x in zip(start, f) if b < own]
+                        d += len(ran)
+                        times.append(ran[-1] if ran else Fraction(0))
+                d_row.append(d)
+                s_row.append(max(times) + t_comm)
+            want_done.append(d_row)
+            want_step.append(s_row)
+        lat = np.array([[float(x) for x in o] for o in outcomes], np.float32).reshape(T, N, M)
+        taus_f = np.array([float(t) for t in taus], np.float32)
+        sc = np.array([float(x) for x in scales], np.float32)
+        sw = oracle.sweep(lat, taus_f, float(t_comm), rule=rule, order=order, lib=lib, worker_scale=sc)
+        assert np.array_equal(sw.done, np.array(want_done, np.int32)), (N, M, rule)
+        assert np.array_equal(sw.step, np.array([[float(x) for x in r] for r in want_step], np.float32)), (N, M, rule)
+    # all scales one: the common-threshold results, bit for bit; and the synchronous time never depends on the scales
+    rng = np.random.default_rng(23)
+    lat = _np(W.iid_latencies("shifted_exp", 9, 7, 6, 24, shift=0.05, mean=0.03))
+    taus_f = np.sort(rng.uniform(-0.1, 1.2 * lat.sum(-1).max(), 13)).astype(np.float32)
+    for rule in (0, 1):
+        a = oracle.sweep(lat, taus_f, 0.07, rule=rule, order=order, lib=lib)
+        b = oracle.sweep(lat, taus_f, 0.07, rule=rule, order=order, lib=lib, worker_scale=np.ones(7, np.float32))
+        assert np.array_equal(a.done, b.done) and np.array_equal(a.step, b.step) and np.array_equal(a.sync, b.sync)
+        # worker 3 twice as slow and given twice the threshold: its own decisions do not change (powers of two are exact)
+        sc = rng.uniform(0.5, 1.5, 7).astype(np.float32)
+        one = oracle.sweep(lat[:, 3:4], taus_f, 0.07, rule=rule, order=order, lib=lib, worker_scale=sc[3:4])
+        lat2, sc2 = lat.copy(), sc.copy()
+        lat2[:, 3] *= 2.0
+        sc2[3] *= 2.0
+        two = oracle.sweep(lat2[:, 3:4], taus_f, 0.07, rule=rule, order=order, lib=lib, worker_scale=sc2[3:4])
+        assert np.array_equal(one.done, two.done)
+        c = oracle.sweep(lat, taus_f, 0.07, rule=rule, order=order, lib=lib, worker_scale=sc)
+        assert np.array_equal(c.sync, a.sync)
+        # the counts are the sum of the workers' own counts
+        per = sum(oracle.sweep(lat[:, n:n + 1], taus_f, 0.07, rule=rule, order=order, lib=lib, worker_scale=sc[n:n + 1]).done
+                  for n in range(7))
+        assert np.array_equal(per, c.done)
+
+
 def pin_closed_form(lib, order="rows"):
     """App. C.2: Phi and Phi^-1 against scipy, Eq. 4/12, Eq. 5/10, Eq. 11 and the analytic tau*; then the
     closed forms against the simulator itself where they are exact (normal micro-batches: Eq. 5) or good
@@ -447,8 +510,8 @@ ALL_PINS = (
     pin_exp_max_harmonic, pin_normal_max_quadrature, pin_done_frac_normal_eq5, pin_done_frac_erlang,
     pin_enumeration, pin_hand_example, pin_per_iteration_comm, pin_fp32_left_to_right, pin_m1_sort, pin_invariants, pin_argmax,
     pin_definition_equals_rows, pin_independence_and_bailey, pin_bailey_against_quadrature, pin_closed_form,
-    pin_start_rule_memoryless,
+    pin_start_rule_memoryless, pin_worker_scales,
 )
 # a quick subset that still kills every planted mistake (used by the mutation test)
-FAST_PINS = (pin_hand_example, pin_per_iteration_comm, pin_enumeration, pin_fp32_left_to_right, pin_m1_sort, pin_argmax,
+FAST_PINS = (pin_worker_scales, pin_hand_example, pin_per_iteration_comm, pin_enumeration, pin_fp32_left_to_right, pin_m1_sort, pin_argmax,
              pin_bailey_against_quadrature, pin_closed_form, pin_invariants, pin_exp_max_harmonic)

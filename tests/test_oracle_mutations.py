@@ -15,14 +15,14 @@ MUTANTS = [
     ("non_strict_compare", [("completed += (f[m] < tau) ? 1 : 0;", "completed += (f[m] <= tau) ? 1 : 0;", 1),
                             ("cnt[k] += (elapsed < taus[k]) ? 1 : 0;", "cnt[k] += (elapsed <= taus[k]) ? 1 : 0;", 1)]),
     ("last_worker_not_max", [("slowest_full = fmaxf(slowest_full, finish[n * M + (M - 1)]);", "slowest_full = finish[n * M + (M - 1)];", 1),
-                             ("slowest_full = fmaxf(slowest_full, elapsed);", "slowest_full = elapsed;", 1)]),
-    ("double_accumulator", [("float elapsed = 0.0f;", "double elapsed = 0.0;", 3)]),
+                             ("slowest_full = fmaxf(slowest_full, elapsed);", "slowest_full = elapsed;", 2)]),
+    ("double_accumulator", [("float elapsed = 0.0f;", "double elapsed = 0.0;", 4)]),
     ("no_min_with_tau", [("(fminf(tau, slowest_full) + tc)", "(tau + tc)", 1),
                          ("(fminf(taus[k], slowest_full) + tc)", "(taus[k] + tc)", 1)]),
     ("sync_without_comm", [("out_sync[i] = slowest_full + tc;", "out_sync[i] = slowest_full;", 2)]),
     ("step_without_comm", [("(fminf(tau, slowest_full) + tc)", "(fminf(tau, slowest_full))", 1),
                            ("(fminf(taus[k], slowest_full) + tc)", "(fminf(taus[k], slowest_full))", 1)]),
-    ("transposed_layout", [("const float *row = lat + (i * N + n) * M;", "const float *row = lat + (i * M + n) * N;", 3)]),
+    ("transposed_layout", [("const float *row = lat + (i * N + n) * M;", "const float *row = lat + (i * M + n) * N;", 4)]),
     ("skips_first_microbatch", [("elapsed = elapsed + row[m];\n                finish[n * M + m] = elapsed;",
                                  "if (m > 0) elapsed = elapsed + row[m];\n                finish[n * M + m] = elapsed;", 1),
                                 ("for (int64_t m = 0; m < M; ++m) {\n                    if (rule == 0) {",
@@ -39,10 +39,15 @@ MUTANTS = [
     ("bailey_weights_swapped", [("(1.0 - g) * dco_phi_inv(1.0 - 1.0 / (double)N) + g * dco_phi_inv(", "g * dco_phi_inv(1.0 - 1.0 / (double)N) + (1.0 - g) * dco_phi_inv(", 1)]),
     ("eq5_variance_not_scaled_by_m", [("sqrt((double)m * sigma * sigma)", "sqrt(sigma * sigma)", 1)]),
     ("eq11_numerator_without_comm", [("* (ET + t_comm) / step", "* ET / step", 1)]),
-    ("rule1_inclusive", [("const float start = (m == 0) ? 0.0f : f[m - 1];", "const float start = f[m];", 1),
+    ("rule1_inclusive", [("const float start = (m == 0) ? 0.0f : f[m - 1];", "const float start = f[m];", 2),
                          ("if (start < taus[k]) {", "if (elapsed < taus[k]) {", 1)]),
-    ("rule1_time_is_start_of_last", [("last_run >= 0 ? f[last_run] : 0.0f", "last_run > 0 ? f[last_run - 1] : 0.0f", 1),
-                                     ("wlast[k] = elapsed;", "wlast[k] = start;", 1)]),
+    ("rule1_time_is_start_of_last", [("last_run >= 0 ? f[last_run] : 0.0f", "last_run > 0 ? f[last_run - 1] : 0.0f", 2),
+                                     ("wlast[k] = elapsed;", "wlast[k] = start;", 2)]),
+    ("scale_of_the_wrong_worker", [("worker_scale[n] * taus[k]", "worker_scale[0] * taus[k]", 2)]),
+    ("scaled_worker_time_ignores_its_threshold", [("worker_time = fminf(own_tau, f[M - 1]);", "worker_time = f[M - 1];", 1),
+                                                  ("(rule == 0) ? fminf(own[k], elapsed) : wlast[k]", "(rule == 0) ? elapsed : wlast[k]", 1)]),
+    ("scaled_step_starts_from_zero", [("slowest = (n == 0) ? worker_time : fmaxf(slowest, worker_time);", "slowest = fmaxf(slowest, worker_time);", 1),
+                                      ("wmax[k] = (n == 0) ? worker_time : fmaxf(wmax[k], worker_time);", "wmax[k] = fmaxf(wmax[k], worker_time);", 1)]),
     ("rule1_last_worker_not_max", [("slowest_cut = fmaxf(slowest_cut, last_run >= 0 ? f[last_run] : 0.0f);",
                                     "slowest_cut = last_run >= 0 ? f[last_run] : 0.0f;", 1),
                                    ("wmax[k] = fmaxf(wmax[k], wlast[k]);", "wmax[k] = wlast[k];", 1)]),

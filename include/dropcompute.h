@@ -124,6 +124,28 @@ int dc_simulate_tc(const float *latencies, int64_t T, int64_t N, int64_t M,
                    int32_t rule, void *stream);
 
 /*
+ * dc_simulate_scaled — dc_simulate_ex for workers that are not identical (App. C.2 remarks that each worker may have
+ * its own mu_n, sigma_n): worker n works against its own thresholds
+ *
+ *   theta[n][k] = fl32( worker_scale[n] * taus[k] )          (one fp32 product; worker_scale[n] > 0, finite)
+ *
+ * instead of the common taus[k].  With DC_RULE_FINISH_BEFORE_TAU:
+ *   out_done[t][k] = #{ (n,m) : P_{t,n,m} < theta[n][k] }
+ *   out_step[t][k] = fl32( max_n fminf(theta[n][k], P_{t,n,M-1}) + t_comm )     (Sec. 4.3's min{tau, T_n}, per worker)
+ * and with DC_RULE_START_BEFORE_TAU micro-batch m of worker n is run iff P_{t,n,m-1} < theta[n][k], W_n is the finish
+ * time of the last one it ran and out_step[t][k] = fl32( max_n W_n + t_comm ).  out_sync as in dc_simulate_ex (it does not
+ * depend on the scales).  worker_scale = all ones gives dc_simulate_ex's results bit for bit.
+ *   worker_scale  DEVICE, [N] fp32, 4-byte aligned
+ * Everything else as dc_simulate_ex; dc_reduce_trials and dc_argmax_tau work on the outputs unchanged.  A plain kernel
+ * (ordinary loads, one block per trial, a cursor per row): 0.9-2.1 TB/s on the workloads here, a sixth to a third of
+ * dc_simulate_ex's rate.
+ */
+int dc_simulate_scaled(const float *latencies, int64_t T, int64_t N, int64_t M,
+                       const float *taus, int32_t K, const float *worker_scale, float t_comm,
+                       float *out_step, int32_t *out_done, float *out_sync,
+                       int32_t rule, void *stream);
+
+/*
  * dc_simulate_split — dc_simulate_ex for FEW trials of MANY workers.  The sweep kernels give a whole trial to
  * one thread block, so fewer trials than about twice the number of SMs leave most of the GPU idle.  This entry
  * point sweeps every trial as G groups of N/G workers (G a divisor of N chosen by the library; no data is

@@ -25,7 +25,7 @@ NSTATS = 5
 STAT_NAMES = ("mean_step", "done_frac", "thr", "thr_mean", "s_eff")
 
 EXPORTS = (
-    "dc_simulate", "dc_simulate_ex", "dc_simulate_tc", "dc_simulate_split_workspace_bytes", "dc_simulate_split",
+    "dc_simulate", "dc_simulate_ex", "dc_simulate_tc", "dc_simulate_scaled", "dc_simulate_split_workspace_bytes", "dc_simulate_split",
     "dc_reduce_workspace_bytes", "dc_reduce_trials", "dc_reduce_trials_static",
     "dc_argmax_tau", "dc_sweep_device",
     "dc_closed_form", "dc_sweep_host_workspace_bytes", "dc_sweep_host", "dc_check_inputs", "dc_device_status",
@@ -52,6 +52,8 @@ _lib.dc_simulate.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _p, _p, _p]
 _lib.dc_simulate_ex.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _p, _p, _p, _i32, _p]
 _lib.dc_simulate_tc.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _p, _p, _p, _p, _i32, _p]
 _lib.dc_simulate_tc.restype = ctypes.c_int
+_lib.dc_simulate_scaled.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _p, _f32, _p, _p, _p, _i32, _p]
+_lib.dc_simulate_scaled.restype = ctypes.c_int
 _lib.dc_simulate_split_workspace_bytes.argtypes = [_i64, _i64, _i64, _i32]
 _lib.dc_simulate_split_workspace_bytes.restype = _sz
 _lib.dc_simulate_split.argtypes = [_p, _i64, _i64, _i64, _p, _i32, _f32, _p, _p, _p, _i32, _p, _sz, _p]
@@ -151,6 +153,22 @@ def dc_simulate_tc(latencies: torch.Tensor, taus: torch.Tensor, t_comm_trials: t
                                    _dev(out_step, torch.float32, "out_step"), _dev(out_done, torch.int32, "out_done"),
                                    None if out_sync is None else _dev(out_sync, torch.float32, "out_sync"),
                                    int(rule), _stream(latencies)), "dc_simulate_tc")
+
+
+def dc_simulate_scaled(latencies: torch.Tensor, taus: torch.Tensor, worker_scale: torch.Tensor, t_comm: float,
+                       out_step: torch.Tensor, out_done: torch.Tensor, out_sync: Optional[torch.Tensor],
+                       rule: int = RULE_FINISH_BEFORE_TAU) -> None:
+    """``dc_simulate_scaled``: worker n works against its own thresholds worker_scale[n] * taus[k] (worker_scale [N] fp32)."""
+    T, N, M = latencies.shape
+    K = taus.shape[0]
+    assert tuple(out_step.shape) == (T, K) and tuple(out_done.shape) == (T, K) and tuple(worker_scale.shape) == (N,)
+    assert out_sync is None or tuple(out_sync.shape) == (T,)
+    with torch.cuda.device(latencies.device):
+        _check(_lib.dc_simulate_scaled(_dev(latencies, torch.float32, "latencies"), T, N, M, _dev(taus, torch.float32, "taus"),
+                                       K, _dev(worker_scale, torch.float32, "worker_scale"), float(t_comm),
+                                       _dev(out_step, torch.float32, "out_step"), _dev(out_done, torch.int32, "out_done"),
+                                       None if out_sync is None else _dev(out_sync, torch.float32, "out_sync"),
+                                       int(rule), _stream(latencies)), "dc_simulate_scaled")
 
 
 def dc_simulate_split_workspace_bytes(T: int, N: int, M: int, K: int) -> int:

@@ -46,6 +46,7 @@
 #include "sweep_tiled.cuh"
 #include "sweep_flat.cuh"
 #include "sweep_plain.cuh"
+#include "sweep_scaled.cuh"
 #include "stats_kernels.cuh"
 
 namespace {
@@ -633,6 +634,28 @@ int dc_simulate_tc(const float *latencies, int64_t T, int64_t N, int64_t M, cons
     return simulate_impl(latencies, T, N, M, taus, K, 0.0f, t_comm_trials, out_step, out_done, out_sync, rule, stream);
 }
 
+int dc_simulate_scaled(const float *latencies, int64_t T, int64_t N, int64_t M, const float *taus, int32_t K,
+                       const float *worker_scale, float t_comm, float *out_step, int32_t *out_done, float *out_sync, int32_t rule,
+                       void *stream_v)
+{
+    if (!worker_scale) return DC_ERR_NULL;
+    const int rc = validate_simulate(latencies, T, N, M, taus, K, out_step, out_done, rule);
+    if (rc != DC_OK) return rc;
+    if ((reinterpret_cast<uintptr_t>(worker_scale) & 3) || (out_sync && (reinterpret_cast<uintptr_t>(out_sync) & 3))) return DC_ERR_ALIGN;
+    DeviceInfo di;
+    if (!device_info(&di)) return DC_ERR_CUDA;
+    const size_t smem = scaled_smem_bytes(K);
+    if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
+    auto kernel = rule == DC_RULE_FINISH_BEFORE_TAU ? dc_sweep_scaled<0> : dc_sweep_scaled<1>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kScaledThreads, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
+    const long long grid = even_grid(T, (long long)occ * di.sms);
+    kernel<<<(unsigned)grid, kScaledThreads, smem, static_cast<cudaStream_t>(stream_v)>>>(latencies, taus, worker_scale, T, (int)N, (int)M, K,
+                                                                                      t_comm, out_step, out_done, out_sync);
+    return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
 // Groups per trial for dc_simulate_split: the smallest divisor G of N that gives T*G >= two blocks per SM while
 // leaving at least 64 workers per group (else the largest divisor that leaves 64); 1 when nothing is gained.
 static int64_t split_groups(int64_t T, int64_t N, int sms)
@@ -1044,7 +1067,7 @@ int dc_launch_count(int32_t entry_point, int64_t T, int64_t N, int64_t M, int32_
 {
     if (T <= 0 || N <= 0 || M <= 0 || K <= 0) return -DC_ERR_SHAPE;
     switch (entry_point) {
-    case DC_ENTRY_SIMULATE: return 1;
+    case DC_ENTRY_SIMULATE: return 1;  // (dc_simulate_scaled too)
     case DC_ENTRY_SIMULATE_SPLIT: {
         DeviceInfo di;
         if (!device_info(&di)) return -DC_ERR_CUDA;

@@ -826,3 +826,43 @@ def test_two_host_threads_on_two_streams(api):
         api.dc_tune(api.TUNE_DIRECT_BINS, 0)
     assert not errors, errors
     api.dc_device_status()
+
+
+@pytest.mark.parametrize("rule", [0, 1])
+@pytest.mark.parametrize("T,N,M,K", [(9, 8, 4, 16), (5, 300, 36, 40), (4, 33, 129, 17), (40, 200, 12, 64), (3, 1000, 7, 300),
+                                      (6, 1, 5, 3), (2, 70, 16, 4096)])
+def test_heterogeneous_workers_match_oracle(api, T, N, M, K, rule):
+    """dc_simulate_scaled: worker n against its own thresholds s_n tau_k (App. C.2: workers need not be identical), both
+    rules, grids with negative, repeated and infinite thresholds; with all scales one it must give dc_simulate_ex's bits."""
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=600 + T + N, shift=0.01, mean=0.02).numpy()
+    taus = grid_for(lat, K, seed=K + 21)
+    rng = np.random.default_rng(N + M)
+    scale = rng.uniform(0.6, 1.6, N).astype(np.float32)
+    scale[rng.integers(N)] = 1.0
+    lat_d, taus_d = torch.from_numpy(lat).cuda(), torch.from_numpy(taus).cuda()
+    step = torch.empty((T, K), dtype=torch.float32, device="cuda")
+    done = torch.empty((T, K), dtype=torch.int32, device="cuda")
+    sync = torch.empty((T,), dtype=torch.float32, device="cuda")
+    for sc in (scale, np.ones(N, np.float32)):
+        ref = oracle.sweep(lat, taus, 0.07, rule=rule, worker_scale=sc,
+                           order="definition" if T * N * M * K < 10 ** 7 else "rows")
+        step.fill_(-1.0)
+        done.fill_(-1)
+        api.dc_simulate_scaled(lat_d, taus_d, torch.from_numpy(sc).cuda(), 0.07, step, done, sync, rule)
+        torch.cuda.synchronize()
+        assert np.array_equal(done.cpu().numpy(), ref.done), "out_done differs"
+        assert np.array_equal(step.cpu().numpy().view(np.uint32), ref.step.view(np.uint32)), "out_step differs"
+        assert np.array_equal(sync.cpu().numpy().view(np.uint32), ref.sync.view(np.uint32)), "out_sync differs"
+    same = run_gpu(api, lat_d, taus_d, 0.07, rule=rule)          # all scales one == the common-threshold entry point
+    assert torch.equal(done, same.out_done) and torch.equal(step, same.out_step) and torch.equal(sync, same.out_sync)
+    # the statistics and tau* follow from the per-trial outputs as always
+    stats = torch.empty((api.NSTATS, K), dtype=torch.float64, device="cuda")
+    base = torch.empty(2, dtype=torch.float64, device="cuda")
+    ws = torch.empty(api.dc_reduce_workspace_bytes(T, K), dtype=torch.uint8, device="cuda")
+    api.dc_simulate_scaled(lat_d, taus_d, torch.from_numpy(scale).cuda(), 0.07, step, done, sync, rule)
+    api.dc_reduce_trials(step, done, sync, N, M, stats, base, ws)
+    torch.cuda.synchronize()
+    ref = oracle.sweep(lat, taus, 0.07, rule=rule, worker_scale=scale)
+    st = oracle.reduce_trials(ref.step, ref.done, ref.sync, N, M)
+    assert np.allclose(stats.cpu().numpy(), st.stats, rtol=RTOL_STATS, atol=0, equal_nan=True)
+    api.dc_device_status()

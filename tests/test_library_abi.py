@@ -78,6 +78,9 @@ def test_argument_errors_need_no_gpu(lib):
     # the later entry points
     assert lib.dc_simulate_tc(A, 1, 1, 1, A, 1, None, A, A, None, 0, None) == 1          # per-trial times missing
     assert lib.dc_simulate_tc(A, 1, 1, 1, A, 1, A + 2, A, A, None, 0, None) == 3
+    assert lib.dc_simulate_scaled(A, 1, 1, 1, A, 1, None, f, A, A, None, 0, None) == 1      # per-worker scales missing
+    assert lib.dc_simulate_scaled(A, 1, 1, 1, A, 1, A + 2, f, A, A, None, 0, None) == 3
+    assert lib.dc_simulate_scaled(A, 1, 1, 1, A, 1, A, f, A, A, None, 3, None) == 7
     assert lib.dc_reduce_trials_static(A, A, A, 4, 1025, 1, 1, A, A, None) == 4           # beyond the built-in scratch
     assert lib.dc_reduce_trials_static(A, A, A, 0, 4, 1, 1, A, A, None) == 2
     d = ctypes.c_double

@@ -96,14 +96,17 @@ def test_static_reduce_requests_no_device_memory(api):
     step, done, sync = _sweep_outputs(api, 300, 20, 8, 64, seed=60)
     got = torch.empty((api.NSTATS, 64), dtype=torch.float64, device="cuda")
     got_base = torch.empty(2, dtype=torch.float64, device="cuda")
+    import gc
     api.dc_reduce_trials_static(step, done, sync, 20, 8, got, got_base)      # warm-up
     torch.cuda.synchronize()
+    gc.collect()                                                             # tensors of earlier tests go now, not mid-measurement
     before = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), _device_free_bytes())
     for _ in range(3):
         api.dc_reduce_trials_static(step, done, sync, 20, 8, got, got_base)
     torch.cuda.synchronize()
     after = (torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), _device_free_bytes())
-    assert before == after, (before, after)
+    assert after[0] <= before[0], (before, after)          # nothing new handed out by torch's pool
+    assert after[1:] == before[1:], (before, after)        # the pool did not grow, the device's free memory did not move
 
 
 def test_static_reduce_at_the_top_of_its_scratch(api):

@@ -211,7 +211,8 @@ def time_other_workloads(api, dev, peak: float, max_trials: int = 0):
     """The four smaller workloads under both completion rules and the bench workload under rule 1: one
     dc_simulate_ex launch each, 3 warm-ups and 10 timed launches, under the same regime as the headline
     measurement (a 256 MiB buffer is written between launches when the input is smaller than 512 MB; larger
-    inputs exceed the L2 cache by themselves), with a plain read-only pass over the same bytes beside each."""
+    inputs exceed the L2 cache by themselves), with a plain read-only pass over the same bytes beside each.  Three of
+    the workloads are also run through dc_simulate_scaled (rows with an "entry" key)."""
     rows = []
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     sink = torch.zeros((1,), dtype=torch.float32, device=dev)
@@ -255,6 +256,17 @@ def time_other_workloads(api, dev, peak: float, max_trials: int = 0):
                          "sweep_ms": avg_ms, "sweep_ms_best": best_ms, "hbm_gbs": gbs, "frac": gbs / peak,
                          "read_only_pass_ms": probe_ms, "sweep_over_read_only_pass": avg_ms / probe_ms,
                          "l2": "inputs larger than L2" if fl is None else "256 MiB buffer written between launches"})
+        if name in ("paper_scale", "extrapolation", "correlated"):
+            # workers with thresholds of their own (s_n tau_k, s_n uniform on [0.8, 1.2]): dc_simulate_scaled
+            scale = torch.from_numpy(W.worker_scales(w.N, w.seed)).to(dev)
+            for rule in rules:
+                avg_ms, best_ms = timed(lambda: api.dc_simulate_scaled(lat, taus, scale, w.t_comm, step, done, sync, rule))
+                gbs = (alg_bytes + 4 * w.N) / (avg_ms * 1e-3) / 1e9
+                rows.append({"workload": name, "rule": rule, "T": w.T, "N": w.N, "M": w.M, "K": w.K,
+                             "entry": "dc_simulate_scaled", "kernel": "dc_sweep_scaled",
+                             "sweep_ms": avg_ms, "sweep_ms_best": best_ms, "hbm_gbs": gbs, "frac": gbs / peak,
+                             "read_only_pass_ms": probe_ms, "sweep_over_read_only_pass": avg_ms / probe_ms,
+                             "l2": "inputs larger than L2" if fl is None else "256 MiB buffer written between launches"})
         del lat, step, done, sync
         torch.cuda.empty_cache()
     api.dc_device_status()

@@ -648,10 +648,12 @@ int dc_simulate_scaled(const float *latencies, int64_t T, int64_t N, int64_t M, 
     if (smem > (size_t)di.max_smem_optin) return DC_ERR_RANGE;
     auto kernel = rule == DC_RULE_FINISH_BEFORE_TAU ? dc_sweep_scaled<0> : dc_sweep_scaled<1>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DC_ERR_CUDA;
+    // a block is one thread per worker, in whole warps, up to kScaledThreads (more workers: several rows per thread)
+    const int block = (int)min((int64_t)kScaledThreads, ((N + 31) / 32) * 32);
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, kScaledThreads, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, block, smem) != cudaSuccess || occ < 1) return DC_ERR_CUDA;
     const long long grid = even_grid(T, (long long)occ * di.sms);
-    kernel<<<(unsigned)grid, kScaledThreads, smem, static_cast<cudaStream_t>(stream_v)>>>(latencies, taus, worker_scale, T, (int)N, (int)M, K,
+    kernel<<<(unsigned)grid, block, smem, static_cast<cudaStream_t>(stream_v)>>>(latencies, taus, worker_scale, T, (int)N, (int)M, K,
                                                                                       t_comm, out_step, out_done, out_sync);
     return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
 }

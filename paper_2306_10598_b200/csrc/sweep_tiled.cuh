@@ -5,19 +5,22 @@
 namespace {
 
 // ------------------------------------------------------------------------------------------
-// Tiled kernel: TMA-staged rows, persistent over trials.  Warp roles inside a block:
-//   warps 0 .. ncw-1   consumers: thread r owns row (pass*rows + r) of the current trial
+// Tiled kernel: TMA-staged rows, persistent over tiles.  A tile is one pass of a trial (up to 256 rows), or g whole
+// trials of few workers each (g N <= 256 rows; two trials of up to 256 rows in the WIDE instantiations).
+// Warp roles inside a block:
+//   warps 0 .. ncw-1   consumers: thread r owns row r of the current tile
 //   warp  ncw          producer: one thread streams the block's tiles through the ring of stages
-//   warp  ncw+1        epilogue: turns a finished trial's histograms into out_done / out_step / out_sync
-// The histograms (and the per-warp maxima) are double-buffered: consumers fill buffer j&1 for their j-th
-// trial and go straight on to the next trial while the epilogue warp sums, scans, writes and clears the
-// buffer.  Named barriers hand the buffers over: kBarReady+b (consumers arrive, epilogue waits) and
-// kBarFree+b (epilogue arrives, consumers wait before reusing the buffer two trials later).
+//   warp  ncw+1        epilogue: turns a finished tile's histograms into out_done / out_step / out_sync
+// The histograms (and the maxima) are double-buffered: consumers fill buffer j&1 for their j-th tile and go
+// straight on to the next one while the epilogue warp sums, scans, writes and clears the buffer.  Named barriers
+// hand the buffers over: kBarReady+b (consumers arrive, epilogue waits) and kBarFree+b (epilogue arrives,
+// consumers wait before reusing the buffer two tiles later).  Tiles of many small trials are finished by the
+// consumer warps themselves instead (one buffer, the epilogue warp returns at once).
 // NQ = 16-byte quads of a row per chunk held in registers (box width = 4*NQ floats at most).
-// A consumer thread adds its row's samples in order; per group of eight, if every lane of the warp is
-// still below the first threshold the samples are bin 0 (one register add); if every lane is at or
-// above the last threshold they are in the bin nobody reads; otherwise each running sum is binned
-// through the lookup table.
+// A consumer thread adds its row's samples in order; per group of samples, if every lane of the warp is still
+// below the first threshold the samples are bin 0 (one register add); if every lane is at or above the last
+// threshold they are in the bin nobody reads; otherwise each running sum is binned through the lookup table (or
+// by arithmetic on evenly spaced thresholds) and settled by exact comparisons with the thresholds.
 // ------------------------------------------------------------------------------------------
 constexpr int kBarReady = 2;  // +0, +1
 constexpr int kBarFree = 4;   // +0, +1

@@ -81,6 +81,13 @@ def make_taus(w: Workload) -> np.ndarray:
     return grid.astype(np.float32)
 
 
+def worker_scales(N: int, seed: int = 0, spread: float = 0.2) -> np.ndarray:
+    """Per-worker threshold scales s_n for the heterogeneous-worker sweep: fp32, uniform on [1 - spread, 1 + spread]
+    (a fleet whose workers' paces differ by up to +-spread), drawn with numpy's seeded generator."""
+    rng = np.random.default_rng(7_000_003 * (seed + 1) + N)
+    return rng.uniform(1.0 - spread, 1.0 + spread, N).astype(np.float32)
+
+
 # --- the laws -------------------------------------------------------------
 # Every function fills out[t0:t1] (a [n_trials, N, M] fp32 view) using generator g.
 

@@ -62,7 +62,8 @@ def test_gpu_arm_prints_one_json_line_with_roofline_and_e2e():
 @pytest.mark.gpu
 def test_default_workload_line_carries_the_other_workloads():
     """The default run (the bench workload under the paper's rule) also times the four smaller workloads under both
-    rules and the bench workload under the start-before-tau rule, and reports them in the same JSON line."""
+    rules, the bench workload under the start-before-tau rule and the heterogeneous-worker sweep on three of them,
+    and reports them in the same JSON line."""
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "3", "--warmup", "3", "--no-e2e",
                           "--no-cpu-baseline", "--other-trials", "96"], capture_output=True, text=True, timeout=900, cwd=ROOT)
     assert out.returncode == 0, out.stderr[-2000:]
@@ -71,10 +72,13 @@ def test_default_workload_line_carries_the_other_workloads():
     d = json.loads(lines[0])
     assert d["config"]["workload"] == "bandwidth_stress" and d["config"]["rule"] == 0
     rows = d["other_workloads"]
-    got = sorted((r["workload"], r["rule"]) for r in rows if "rule" in r)
+    got = sorted((r["workload"], r["rule"]) for r in rows if "rule" in r and "entry" not in r)
     assert got == sorted([(n, r) for n in ("tiny", "paper_scale", "extrapolation", "correlated") for r in (0, 1)]
                          + [("bandwidth_stress", 1)])
+    scaled = sorted((r["workload"], r["rule"]) for r in rows if r.get("entry") == "dc_simulate_scaled")
+    assert scaled == sorted((n, r) for n in ("paper_scale", "extrapolation", "correlated") for r in (0, 1))
     for r in rows:
         for key in ("kernel", "sweep_ms", "hbm_gbs", "frac", "read_only_pass_ms", "sweep_over_read_only_pass"):
             assert key in r and (r[key] is not None), (r["workload"], key)
-        assert r["sweep_ms"] > 0 and r["kernel"] == "dc_sweep_tiled"
+        assert r["sweep_ms"] > 0
+        assert r["kernel"] == ("dc_sweep_scaled" if "entry" in r else "dc_sweep_tiled")

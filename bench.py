@@ -311,6 +311,8 @@ def run_ours(args, w: W.Workload):
     k_star = torch.empty((), dtype=torch.int32, device=dev)
     tau_star = torch.empty((), dtype=torch.float32, device=dev)
     value = torch.empty((), dtype=torch.float64, device=dev)
+    # --worker-scales: the heterogeneous-worker sweep (worker n against s_n tau_k) in place of the common-threshold one
+    scale = torch.from_numpy(W.worker_scales(N, wr.seed)).to(dev) if args.worker_scales else None
     flush = None
     if wr.latency_bytes < (512 << 20):  # inputs not much larger than L2: write a 256 MiB buffer between steps
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -320,7 +322,10 @@ def run_ours(args, w: W.Workload):
             flush.zero_()
         if ev:
             ev[0].record()
-        api.dc_simulate_ex(lat, taus, wr.t_comm, out_step, out_done, out_sync, args.rule)
+        if scale is not None:
+            api.dc_simulate_scaled(lat, taus, scale, wr.t_comm, out_step, out_done, out_sync, args.rule)
+        else:
+            api.dc_simulate_ex(lat, taus, wr.t_comm, out_step, out_done, out_sync, args.rule)
         if ev:
             ev[1].record()
         api.dc_reduce_trials(out_step, out_done, out_sync, N, M, stats, baseline, ws)
@@ -376,10 +381,12 @@ def run_ours(args, w: W.Workload):
     samples = T * N * M
     value_sps = world * args.steps * samples / (total_ms * 1e-3)
     sim_avg_s = (sum(sim_ms) / len(sim_ms)) * 1e-3
-    alg_bytes = 4 * samples + 8 * T * K + 4 * T
+    alg_bytes = 4 * samples + 8 * T * K + 4 * T + (4 * N if scale is not None else 0)
     peak, peak_kind = measured_hbm_peak()
     achieved = alg_bytes / sim_avg_s / 1e9
-    traffic = read_traffic(w.name, api.dc_kernel_version()) if not args.trials else None
+    traffic = read_traffic(w.name, api.dc_kernel_version()) if not (args.trials or args.worker_scales) else None
+    kernel_name = ("dc_sweep_scaled" if scale is not None
+                   else ("dc_sweep_tiled", "dc_sweep_plain", "dc_sweep_flat")[api.dc_simulate_plan(lat, K)])
 
     line = {
         "metric": METRIC, "value": value_sps, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
@@ -388,12 +395,13 @@ def run_ours(args, w: W.Workload):
         "config": {"workload": w.name, "T": T, "N": N, "M": M, "K": K, "t_comm": wr.t_comm,
                    "latency_bytes": wr.latency_bytes,
                    "l2": "inputs larger than L2" if flush is None else "256 MiB buffer written between steps",
-                   "parallelism": f"{world} x independent trials", "rule": args.rule},
+                   "parallelism": f"{world} x independent trials", "rule": args.rule,
+                   "entry": "dc_simulate_scaled (s_n uniform on [0.8, 1.2])" if scale is not None else "dc_simulate_ex"},
         "hbm_gbs": achieved,
         "sweep_ms": sim_avg_s * 1e3,
         "sweep_ms_best": min(sim_ms),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": traffic, "kernel": ("dc_sweep_tiled", "dc_sweep_plain", "dc_sweep_flat")[api.dc_simulate_plan(lat, K)],
+                     "traffic": traffic, "kernel": kernel_name,
                      "peak_kind": f"of {peak_kind} (a copy: half reads, half writes; this kernel almost only reads, which HBM "
                                   "does a little faster, so the fraction can pass 1)",
                      "algorithmic_bytes_per_launch": alg_bytes,
@@ -416,7 +424,7 @@ def run_ours(args, w: W.Workload):
 
     # ---- end to end: samples in pinned host memory, through dc_sweep_host -------------------------
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.worker_scales:   # (dc_sweep_host runs the common-threshold sweep)
         avail = host_mem_available_bytes()
         Te = T
         if wr.latency_bytes > 0.6 * avail / max(world, 1):
@@ -449,9 +457,10 @@ def run_ours(args, w: W.Workload):
         del host, wsh
     line["e2e"] = e2e
 
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.worker_scales:
         line["cpu_baseline"] = cpu_baseline(wr, lat, taus_np)
-    if rank == 0 and world == 1 and not args.no_other_workloads and w.name == "bandwidth_stress" and not args.trials and args.rule == 0:
+    if (rank == 0 and world == 1 and not args.no_other_workloads and w.name == "bandwidth_stress" and not args.trials
+            and args.rule == 0 and not args.worker_scales):
         del lat
         torch.cuda.empty_cache()
         line["other_workloads"] = time_other_workloads(api, dev, peak, args.other_trials)
@@ -477,6 +486,9 @@ def main():
     ap.add_argument("--trials", type=int, default=0, help="override the number of trials (profiling small cases)")
     ap.add_argument("--rule", type=int, default=0, choices=(0, 1),
                     help="completion rule: 0 = Algorithm 2 (finish before tau, the benchmark), 1 = start before tau")
+    ap.add_argument("--worker-scales", action="store_true",
+                    help="time dc_simulate_scaled (workers with thresholds s_n tau_k of their own) instead of dc_simulate_ex; "
+                         "the end-to-end and CPU legs are skipped")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--other-trials", type=int, default=0, help="cap the trials of those extra workloads (for tests)")

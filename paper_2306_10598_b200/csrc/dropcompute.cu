@@ -187,11 +187,11 @@ int launch_flat(const SweepParams &p, int block, size_t smem, long long T, const
     return launch_flat_q<RULE, BATCH, 8>(p, block, smem, T, di, stream);
 }
 
-template <int NQ, int RULE, bool BATCH, bool WIDE = false>
-int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
+template <int NQ, int RULE, bool BATCH, bool WIDE, bool LEAN>
+int launch_tiled_k(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
                    cudaStream_t stream)
 {
-    auto kernel = dc_sweep_tiled<NQ, RULE, BATCH, WIDE>;
+    auto kernel = dc_sweep_tiled<NQ, RULE, BATCH, WIDE, LEAN>;
     // Per instantiation and device: the largest dynamic shared memory opted into so far, and the occupancy of
     // the last (block, smem) asked for -- repeated calls with one shape then cost no runtime queries.
     static std::mutex lock;
@@ -218,6 +218,17 @@ int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size
     const long long grid = even_grid(T, (long long)occ * di.sms, p.grid_mode);
     kernel<<<(unsigned)grid, block, smem, stream>>>(map, p);
     return cudaGetLastError() == cudaSuccess ? DC_OK : DC_ERR_CUDA;
+}
+
+// Rows of full chunks get the kernel with the short consumer loop, the others the kernel with the general one; tiles of
+// two whole trials (WIDE) only exist for rows of one full chunk.
+template <int NQ, int RULE, bool BATCH, bool WIDE = false>
+int launch_tiled_b(const CUtensorMap &map, const SweepParams &p, int block, size_t smem, long long T, const DeviceInfo &di,
+                   cudaStream_t stream)
+{
+    if (p.lean) return launch_tiled_k<NQ, RULE, BATCH, WIDE, true>(map, p, block, smem, T, di, stream);
+    if constexpr (WIDE) return DC_ERR_RANGE;
+    else return launch_tiled_k<NQ, RULE, BATCH, false, false>(map, p, block, smem, T, di, stream);
 }
 
 template <int NQ, int RULE>
@@ -405,7 +416,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
                 p.passes = 1;
                 p.rows = (int)(g * N);
             }
-        } else if (N < kMaxRowsPerPass && (nq_inst == 3 || nq_inst == 4) && p.chunks == 1 && tune.tile_trials != 1 &&
+        } else if (N < kMaxRowsPerPass && (nq_inst == 3 || nq_inst == 4) && p.chunks == 1 && p.lean && tune.tile_trials != 1 &&
                    T >= 8 * (int64_t)di.sms && K <= 512) {
             // Two whole trials per tile when that leaves clearly fewer idle lanes than one (200 workers: 24 of 224
             // lanes idle alone, 16 of 416 as a pair).  Rows of one chunk only: measured 3-6 % faster there (200

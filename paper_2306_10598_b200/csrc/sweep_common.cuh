@@ -634,8 +634,7 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
 
 
 // ------------------------------------------------------------------------------------------
-// The short form of consume_chunk, for rows all of whose chunks are full (4*NQ samples each) and grids on which the
-// table or the cell arithmetic is at most one threshold short of the bin (`one`).  Nothing in it asks whether a lane
+// The short form of consume_chunk, for rows all of whose chunks are full (4*NQ samples each).  Nothing in it asks whether a lane
 // has a row of its own: such a lane shadows the last row of the tile (same shared-memory data, so the votes need no
 // validity term) and is handed the spare histogram copy, which nothing reads, and counters that are dropped.
 // ------------------------------------------------------------------------------------------
@@ -644,7 +643,9 @@ __device__ __forceinline__ void consume_chunk(float4 (&v)[NQ], int ns, bool vali
 // no upper bound (negative and NaN inputs convert to 0 either way).
 // `bin` gives the shared-window address of a sample's bin in this thread's histogram copy: the cell arithmetic or
 // the table proposes the bin, the threshold itself decides (tau_s[K] = +inf).
-template <int NS, int GS, int RULE, bool BATCH, bool DIRECT, bool CLAMP>
+// ONE = the proposal is at most one threshold short (no cell of the table holds two finite thresholds; always so for
+// the cell arithmetic); otherwise the thresholds are stepped over one by one.
+template <int NS, int GS, int RULE, bool BATCH, bool DIRECT, bool CLAMP, bool ONE>
 __device__ __forceinline__ void bin_groups(const float (&s)[NS], const BinCtx &c, uint32_t hist_a, unsigned fmax_delta,
                                            unsigned &prev, int &cnt0, float &fin0)
 {
@@ -658,6 +659,10 @@ __device__ __forceinline__ void bin_groups(const float (&s)[NS], const BinCtx &c
             unsigned cell = __float2uint_rz(__fmul_rn(__fsub_rn(x, c.lut_lo), c.lut_scale));
             if (CLAMP) cell = min(cell, c.C);
             off = lds_u16(c.lut_a + 2u * cell);
+        }
+        if (!ONE) {
+            while (off < c.K4 && x >= lds_f32(c.tau_a + off)) off += 4u;  // (tau_s[K] = +inf ends it too)
+            return hist_a + off;
         }
         const uint32_t ha = hist_a + off;
         return (x >= lds_f32(c.tau_a + off)) ? ha + 4u : ha;
@@ -702,7 +707,7 @@ __device__ __forceinline__ void bin_groups(const float (&s)[NS], const BinCtx &c
     }
 }
 
-template <int NQ, int RULE, bool BATCH, bool DIRECT>
+template <int NQ, int RULE, bool BATCH, bool DIRECT, bool ONE>
 __device__ __forceinline__ void consume_full(const float4 (&v)[NQ], int lane, const BinCtx &c, uint32_t hist_a,
                                              unsigned fmax_delta, float &P, unsigned &prev, int &cnt0, float &fin0,
                                              uint64_t *release_bar)
@@ -732,9 +737,9 @@ __device__ __forceinline__ void consume_full(const float4 (&v)[NQ], int lane, co
     // the bin nobody reads, under the start-before-tau rule none of its micro-batches is started.
     if (__all_sync(0xffffffffu, RULE == 0 ? before >= c.tau_last : prev >= hist_a + c.K4)) return;
     if (__all_sync(0xffffffffu, P < c.tau_top))
-        bin_groups<NS, GS, RULE, BATCH, DIRECT, false>(s, c, hist_a, fmax_delta, prev, cnt0, fin0);
+        bin_groups<NS, GS, RULE, BATCH, DIRECT, false, ONE>(s, c, hist_a, fmax_delta, prev, cnt0, fin0);
     else
-        bin_groups<NS, GS, RULE, BATCH, DIRECT, true>(s, c, hist_a, fmax_delta, prev, cnt0, fin0);
+        bin_groups<NS, GS, RULE, BATCH, DIRECT, true, ONE>(s, c, hist_a, fmax_delta, prev, cnt0, fin0);
 }
 
 }  // namespace

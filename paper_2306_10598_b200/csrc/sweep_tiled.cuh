@@ -269,7 +269,7 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
 // The consumer threads' loop over the block's tiles (tiled kernel).  A tile is p.g whole trials when trials are
 // small (thread r owns row r of the g*N rows, which belongs to trial r / N of the tile), else one trial whose
 // workers are taken in p.passes passes of p.rows rows.  LEAN = every chunk of a row is full (consume_full).
-template <int NQ, int RULE, bool BATCH, bool DIRECT, bool LEAN>
+template <int NQ, int RULE, bool BATCH, bool DIRECT, bool LEAN, bool ONE = true>
 __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTail &s, const BinCtx &ctx, unsigned char *stage0,
                                              uint64_t *full, uint64_t *empty, int tid, int lane, int warp, int ncw,
                                              unsigned fmax_delta, unsigned off_zero)
@@ -330,7 +330,7 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
                 if (LEAN) {
 #pragma unroll
                     for (int q = 0; q < NQ; ++q) v[q] = lds_stage_f32x4(stage_a + qoff[q]);
-                    consume_full<NQ, RULE, BATCH, DIRECT>(v, lane, ctx, hist_a, fmax_delta, P, prev, pass_cnt0, pass_fin0, empty_bar);
+                    consume_full<NQ, RULE, BATCH, DIRECT, ONE>(v, lane, ctx, hist_a, fmax_delta, P, prev, pass_cnt0, pass_fin0, empty_bar);
                 } else {
                     const int nq = (c == p.chunks - 1) ? p.nq_last : NQ;
 #pragma unroll
@@ -374,7 +374,10 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
 
 // WIDE = tiles of two trials of 129-256 workers each (up to 512 rows, 16 consumer warps): fewer idle lanes in the last
 // warp of a trial and half the hand-overs per trial.
-template <int NQ, int RULE, bool BATCH, bool WIDE>
+// LEAN = every chunk of every row is full: the kernel holds the short consumer loop only (three forms: cell
+// arithmetic, table, table with several thresholds per cell); otherwise the general loop only (two forms).  Keeping
+// the two apart keeps each kernel's code small: with both loops in one kernel the general one measured 5-17 % slower.
+template <int NQ, int RULE, bool BATCH, bool WIDE, bool LEAN>
 __global__ void __launch_bounds__(WIDE ? 2 * kMaxRowsPerPass + 64 : kMaxRowsPerPass + 64, WIDE ? 2 : (NQ <= 4 ? 3 : 2))
 dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
 {
@@ -450,9 +453,10 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     const bool one = ctx.one;
     const unsigned off_zero = RULE == 1 ? bin_of_zero(ctx) : 0u;  // rule 1 only
     const bool direct = s.meta[3] != 0 && one && p.direct_bins != 0;
-    if (p.lean != 0 && one) {
-        if (direct) tiled_trials<NQ, RULE, BATCH, true, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
-        else tiled_trials<NQ, RULE, BATCH, false, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
+    if constexpr (LEAN) {
+        if (direct) tiled_trials<NQ, RULE, BATCH, true, true, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
+        else if (one) tiled_trials<NQ, RULE, BATCH, false, true, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
+        else tiled_trials<NQ, RULE, BATCH, false, true, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
     } else {
         if (direct) tiled_trials<NQ, RULE, BATCH, true, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
         else tiled_trials<NQ, RULE, BATCH, false, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);

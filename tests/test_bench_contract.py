@@ -82,3 +82,20 @@ def test_default_workload_line_carries_the_other_workloads():
             assert key in r and (r[key] is not None), (r["workload"], key)
         assert r["sweep_ms"] > 0
         assert r["kernel"] == ("dc_sweep_scaled" if "entry" in r else "dc_sweep_tiled")
+
+
+@pytest.mark.gpu
+def test_worker_scales_run_times_the_heterogeneous_sweep():
+    """`--worker-scales` puts dc_simulate_scaled in the step: the line names that entry point and kernel, counts the
+    scales in its algorithmic bytes and carries no end-to-end or CPU leg (both are about the common-threshold sweep)."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "paper_scale", "--trials", "512",
+                          "--worker-scales", "--steps", "3", "--warmup", "3", "--no-other-workloads"],
+                         capture_output=True, text=True, timeout=900, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["config"]["entry"].startswith("dc_simulate_scaled") and d["roofline"]["kernel"] == "dc_sweep_scaled"
+    assert d["roofline"]["algorithmic_bytes_per_launch"] == 4 * 512 * 200 * 32 + 8 * 512 * 64 + 4 * 512 + 4 * 200
+    assert d["roofline"]["traffic"] is None and d["e2e"] is None and "cpu_baseline" not in d
+    assert d["gpu_launches"] == 3 * 4 and d["value"] > 0 and 0 <= d["result"]["k_star"] < 64

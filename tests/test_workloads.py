@@ -50,3 +50,12 @@ def test_appendix_b1_delay():
     assert float(x.min()) >= 1.0 and float(x.max()) <= 1.0 + W.B1_BETA + 1e-6     # at most 6.5 times the base
     assert abs(float(x.mean()) - 1.5) < 0.01                                      # 'x1.5 longer on average'
     assert 0.0005 < float((x >= 1.0 + W.B1_BETA - 1e-6).double().mean()) < 0.005  # the bound is rarely hit
+
+
+def test_worker_scales_are_seeded_and_in_range():
+    a = W.worker_scales(200, seed=3)
+    assert a.dtype == np.float32 and a.shape == (200,)
+    assert np.array_equal(a, W.worker_scales(200, seed=3)) and not np.array_equal(a, W.worker_scales(200, seed=4))
+    assert a.min() >= 0.8 and a.max() <= 1.2 and a.std() > 0.05
+    b = W.worker_scales(64, spread=0.5)
+    assert b.min() >= 0.5 and b.max() <= 1.5

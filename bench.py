@@ -273,6 +273,53 @@ def time_other_workloads(api, dev, peak: float, max_trials: int = 0):
     return rows
 
 
+def shape_grid(args):
+    """`--shape-grid`: a table (text, not the JSON line) of GB/s of latency bytes per dc_simulate_ex launch over worker
+    counts N and micro-batch counts M at fixed numbers of latency bytes, rule 0 / rule 1.  Uniform latencies, 64 evenly
+    spaced thresholds over [0.6, 1.4] x the mean row total, median of five launches by CUDA events, a 256 MiB buffer
+    written between launches.  Shows what few workers per trial, very short rows and ragged row lengths cost."""
+    from paper_2306_10598_b200 import build
+    build.build_library()
+    from paper_2306_10598_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    K = 64
+
+    def cell(T, N, M, rule):
+        g = torch.Generator(device=dev).manual_seed(1)
+        lat = torch.rand(T, N, M, device=dev, generator=g) * 0.01 + 0.02
+        taus = torch.linspace(0.6 * 0.025 * M, 1.4 * 0.025 * M, K, device=dev)
+        step = torch.empty(T, K, dtype=torch.float32, device=dev)
+        done = torch.empty(T, K, dtype=torch.int32, device=dev)
+        sync = torch.empty(T, dtype=torch.float32, device=dev)
+        ms = []
+        for i in range(7):
+            flush.fill_(i)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            api.dc_simulate_ex(lat, taus, 0.1, step, done, sync, rule)
+            e1.record()
+            torch.cuda.synchronize(dev)
+            if i >= 2:
+                ms.append(e0.elapsed_time(e1))
+        return 4 * T * N * M / statistics.median(ms) / 1e6
+
+    workers = (8, 32, 100, 200, 256, 300, 512, 1000, 2048, 5000)
+    micro = (4, 8, 12, 16, 24, 32, 48, 64, 100, 128, 256, 512)
+    for total in args.shape_grid:
+        print(f"{total:.1e} latency bytes; rows: workers N, columns: micro-batches M; GB/s under rule 0 / rule 1")
+        print("N\\M   " + "".join(f"{m:>12d}" for m in micro))
+        for N in workers:
+            cells = []
+            for M in micro:
+                T = max(1, int(total / (4 * N * M)))
+                cells.append(f"{cell(T, N, M, 0):6.0f}/{cell(T, N, M, 1):5.0f}")
+            print(f"{N:5d} " + "".join(f"{c:>12s}" for c in cells), flush=True)
+    api.dc_device_status()
+    return 0
+
+
 def run_ours(args, w: W.Workload):
     from paper_2306_10598_b200 import build
     if int(os.environ.get("LOCAL_RANK", "0")) == 0:
@@ -494,7 +541,12 @@ def main():
     ap.add_argument("--other-trials", type=int, default=0, help="cap the trials of those extra workloads (for tests)")
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="skip the extra per-workload sweep timings that the default run adds to its JSON line")
+    ap.add_argument("--shape-grid", type=float, nargs="+", default=None, metavar="BYTES",
+                    help="instead of the benchmark: print a table of sweep GB/s over worker and micro-batch counts at "
+                         "these numbers of latency bytes (e.g. 4e8 3e9), one GPU")
     args = ap.parse_args()
+    if args.shape_grid:
+        return shape_grid(args)
     if args.workload.startswith("c3:"):
         w = W.c3_workload(args.workload[3:], N=args.workers, T=args.trials or 16384)
         args.trials = w.T

@@ -112,6 +112,8 @@ long long even_grid(long long units, long long resident, int mode = 0)
     return (units + rounds - 1) / rounds;
 }
 
+constexpr int kPackedMinRounds = 3;  // packed tiles of several trials only when every resident block gets about this many
+
 int floor_pow2(int v)
 {
     int p = 1;
@@ -416,7 +418,49 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
                 p.passes = 1;
                 p.rows = (int)(g * N);
             }
-        } else if (N < kMaxRowsPerPass && (nq_inst == 3 || nq_inst == 4) && p.chunks == 1 && p.lean && tune.tile_trials != 1 &&
+        }
+        // Trials that do not fill whole warps leave lanes idle in the last warp of every pass (200 workers: 24 of 224;
+        // two trials of 100 workers likewise).  Packed tiles: G trials are one run of G N consecutive rows of the
+        // [T N][M] view, cut into P >= 2 equal passes of at most 256 rows (200 workers: 5 trials = 1000 rows = 4 passes
+        // of 250 rows on 256 lanes, 2.3 % idle instead of 10.7 %); a trial then starts in the middle of a pass.  Taken
+        // when it leaves clearly fewer lanes idle and there are enough tiles for a few rounds.  Measured on 100 and 200
+        // workers, 8192 and more trials: start-before-tau rule 12-20 % faster (its heavier per-trial epilogue also
+        // takes two trials per step instead of one); the paper's rule 4-17 % faster on rows of 12 samples, 10 % on rows
+        // of 100 (general loop), level to 4 % slower on rows of 32 and 64, which therefore stay as they were.
+        bool packed = false;
+        if (N < kMaxRowsPerPass && tune.tile_trials != 1 && (uint64_t)T * (uint64_t)N < (1ull << 31) - 4096) {
+            const int64_t hist_cap = (int64_t)kHistBudgetBytes / (2 * 4 * 4 * (int64_t)(K + 8));  // two buffers, four copies
+            int64_t gmax = min((int64_t)8, hist_cap);
+            // (the epilogue warp must keep up: with K/4 lanes per trial it takes several trials per step; otherwise at
+            // most three trials per tile, as choose_block_layout hands longer tiles to the consumer warps)
+            if (!(K % 4 == 0 && K <= 128 && ((K / 4) & (K / 4 - 1)) == 0)) gmax = min(gmax, (int64_t)3);
+            if (tune.tile_trials > 1 && gmax > tune.tile_trials) gmax = tune.tile_trials;
+            const double idle1 = 1.0 - (double)p.rows / (double)(((p.rows + 31) / 32) * 32);  // as chosen so far
+            double best_idle = idle1;
+            int best_g = 1, best_p = 1, best_rows = 0;
+            for (int64_t G = p.g + 1; G <= gmax; ++G) {
+                const int64_t P = (G * N + kMaxRowsPerPass - 1) / kMaxRowsPerPass;
+                if (P < 2) continue;
+                const int64_t rows = (G * N + P - 1) / P;
+                const double idle = 1.0 - (double)(G * N) / (double)(((rows + 31) / 32) * 32 * P);
+                if (idle < best_idle - 0.005) {
+                    best_idle = idle;
+                    best_g = (int)G;
+                    best_p = (int)P;
+                    best_rows = (int)rows;
+                }
+            }
+            // (under the paper's rule, rows of 32 samples and more in the short loop measured level to 4 % slower packed)
+            const bool pays = rule == DC_RULE_START_BEFORE_TAU || M <= 16 || !p.lean;
+            const bool enough = tune.tile_trials > 1 || (pays && T / best_g >= (int64_t)kPackedMinRounds * 3 * di.sms);
+            if (best_g > 1 && idle1 - best_idle >= 0.04 && enough) {
+                packed = true;
+                p.g = best_g;
+                p.passes = best_p;
+                p.rows = best_rows;
+            }
+        }
+        if (!packed && p.g == 1 && N > kMaxRowsPerPass / 2 && N < kMaxRowsPerPass && (nq_inst == 3 || nq_inst == 4) && p.chunks == 1 && p.lean && tune.tile_trials != 1 &&
                    T >= 8 * (int64_t)di.sms && K <= 512) {
             // Two whole trials per tile when that leaves clearly fewer idle lanes than one (200 workers: 24 of 224
             // lanes idle alone, 16 of 416 as a pair).  Rows of one chunk only: measured 3-6 % faster there (200
@@ -441,7 +485,7 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
         // is so many whole lines (a quarter to an eighth of the requests of row-sized pieces).  The tile in shared
         // memory is the same dense copy of its rows; of "no swizzle" and the 128-byte swizzle the one with fewer
         // bank conflicts for "lane r reads 16 bytes of row r" is taken.
-        const bool whole_lines = tune.whole_lines != 1 && M < 32 && (N * M) % 32 == 0 && ((int64_t)p.rows * M) % 32 == 0 &&
+        const bool whole_lines = !packed && tune.whole_lines != 1 && M < 32 && (N * M) % 32 == 0 && ((int64_t)p.rows * M) % 32 == 0 &&
                                  (p.g > 1 || N % p.rows == 0);
         if (whole_lines) {
             int worst[2] = {0, 0};
@@ -480,6 +524,17 @@ int simulate_impl(const float *lat, int64_t T, int64_t N, int64_t M, const float
             gstride[0] = 128;
             box[0] = 32;
             box[1] = (cuuint32_t)((p.g > 1 ? N : (int64_t)p.rows) * M / 32);
+        }
+        p.tile_y = 0;
+        p.tile_z = p.g;
+        if (packed) {  // [1][T N rows][M floats]: a tile's rows are consecutive whatever trial they belong to
+            gdim[1] = (cuuint64_t)T * (cuuint64_t)N;
+            gdim[2] = 1;
+            gstride[1] = (cuuint64_t)T * (cuuint64_t)N * (cuuint64_t)M * 4;
+            box[1] = (cuuint32_t)p.rows;
+            box[2] = 1;
+            p.tile_y = (int)(p.g * N);
+            p.tile_z = 0;
         }
         const cuuint32_t estr[3] = {1, 1, 1};
         if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(lat), gdim, gstride, box, estr,

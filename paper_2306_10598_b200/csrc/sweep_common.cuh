@@ -63,7 +63,10 @@ struct SweepParams {
                        // (K a multiple of 4, out_step / out_done 16-byte aligned, hist_stride a multiple of 4)
     int box_y;         // tiled kernel: height of one pass in the tensor map's second coordinate (rows, or 128-byte lines
                        // when rows shorter than a line are fetched as whole lines)
-    int g;             // staged kernels: trials per tile (several whole trials of few workers share a tile; else 1)
+    int g;             // staged kernels: trials per tile (several whole trials share a tile; else 1)
+    int tile_y, tile_z;  // tiled kernel: what one tile adds to the tensor map's second and third coordinate (0, 1 for a
+                       // tile of one trial; 0, g for g whole trials in one pass; g N, 0 for g trials whose rows are
+                       // taken as one run of g N consecutive rows of the [T N][M] view, cut into equal passes)
     int epi_sub;       // tiled kernel, g > 1: lanes of the epilogue warp per trial (K/4, a power of two), or 0 for one
                        // trial at a time
     int lean;          // tiled kernel: 1 = every chunk of a row is full, so the short form of the consumer loop applies

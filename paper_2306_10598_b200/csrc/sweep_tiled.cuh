@@ -5,8 +5,10 @@
 namespace {
 
 // ------------------------------------------------------------------------------------------
-// Tiled kernel: TMA-staged rows, persistent over tiles.  A tile is one pass of a trial (up to 256 rows), or g whole
-// trials of few workers each (g N <= 256 rows; two trials of up to 256 rows in the WIDE instantiations).
+// Tiled kernel: TMA-staged rows, persistent over tiles.  A tile is one trial taken in passes of up to 256 rows, or g
+// whole trials: of few workers each in one pass (g N <= 256 rows; two trials of up to 256 rows in the WIDE
+// instantiations), or as one run of g N consecutive rows cut into equal passes, where a trial may start in the middle
+// of a pass (the row -> trial map is then worked out per pass).
 // Warp roles inside a block:
 //   warps 0 .. ncw-1   consumers: thread r owns row r of the current tile
 //   warp  ncw          producer: one thread streams the block's tiles through the ring of stages
@@ -266,23 +268,22 @@ __device__ __forceinline__ void epilogue_warp(const SweepParams &p, const SmemTa
     }
 }
 
-// The consumer threads' loop over the block's tiles (tiled kernel).  A tile is p.g whole trials when trials are
-// small (thread r owns row r of the g*N rows, which belongs to trial r / N of the tile), else one trial whose
-// workers are taken in p.passes passes of p.rows rows.  LEAN = every chunk of a row is full (consume_full).
-template <int NQ, int RULE, bool BATCH, bool DIRECT, bool LEAN, bool ONE = true>
-__device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTail &s, const BinCtx &ctx, unsigned char *stage0,
+// The consumer threads' loop over the block's tiles (tiled kernel).  A tile is p.g whole trials (thread r owns row
+// pass * p.rows + r of the tile's g*N rows in pass `pass`, which belongs to trial (that row) / N of the tile), or one
+// trial whose workers are taken in p.passes passes of p.rows rows.  LEAN = every chunk of a row is full (consume_full).
+template <int NQ, int RULE, bool BATCH, bool DIRECT, bool LEAN, bool ONE, bool MULTI>
+__device__ __forceinline__ void tiled_trials_g(const SweepParams &p, const SmemTail &s, const BinCtx &ctx, unsigned char *stage0,
                                              uint64_t *full, uint64_t *empty, int tid, int lane, int warp, int ncw,
                                              unsigned fmax_delta, unsigned off_zero)
 {
-    const int S = p.stages, G = p.g;
+    const int S = p.stages, G = MULTI ? p.g : 1;  // (MULTI = several trials per tile: compiled apart, the one-trial loop carries none of it)
     const int bar_threads = ncw * 32 + 32;
     const int seg_ints = p.hist_copies * p.hist_stride;  // one trial's histograms
     // Threads past the last row of the tile shadow rows of the tile (different ones, so that what they add to the
     // spare histogram copy spreads over its bins like real rows do).
     const int row = tid < p.rows ? tid : tid % p.rows;
-    const int seg = G > 1 ? row / p.N : 0;
     const int copy = (warp % p.warp_groups) * p.lane_copies + (lane & (p.lane_copies - 1));
-    int *myhist0 = s.hist + seg * seg_ints + copy * p.hist_stride;
+    int *copy0 = s.hist + copy * p.hist_stride;  // this thread's copy in the histograms of buffer 0, trial 0
     // Byte offset of this thread's quad q inside a stage.  The tile is a dense copy of its rows; the hardware
     // swizzle XORs bits 4..6 of an offset with (bits 7..9 & swz_mask), which moves 16-byte quads inside 128-byte lines
     // (rows may be shorter than a line, or not a divisor of it, when they are fetched as whole lines).
@@ -304,13 +305,24 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
     for (long long tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++j) {
         const int b = own_epilogue ? 0 : (j & 1);
         if (!own_epilogue && j >= 2) buffer_barrier_sync<kBarFree>(b, bar_threads);  // the epilogue warp has cleared buffer b
-        int *myhist = myhist0 + b * G * seg_ints;
-        unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
-        const bool in_tile = (tid < p.rows) && (tile * G + seg < p.T);  // this thread's trial exists
         float rowmax = 0.0f, fin0 = 0.0f;
         int cnt0 = 0;
+        int *myhist = copy0 + b * G * seg_ints;
         for (int pass = 0; pass < p.passes; ++pass) {
-            const bool valid = in_tile && (pass * p.rows + tid < p.N || G > 1);
+            // This thread's row in this pass, the trial of the tile it belongs to, and whether both exist.  With
+            // several trials per tile the tile's rows are one run of G N rows taken p.rows at a time, so a thread's
+            // rows in different passes belong to different trials and everything it counts is handed over per pass.
+            int seg = 0;
+            bool valid;
+            if (G > 1) {
+                seg = (pass * p.rows + tid) / p.N;
+                valid = tid < p.rows && seg < G && tile * G + seg < p.T;
+                if (!valid) seg = 0;
+                myhist = copy0 + (b * G + seg) * seg_ints;
+            } else {
+                valid = tid < p.rows && pass * p.rows + tid < p.N;
+            }
+            unsigned char *hist_b = reinterpret_cast<unsigned char *>(myhist);
             float P = 0.0f, pass_fin0 = 0.0f;
             int pass_cnt0 = 0;
             const uint32_t hist_a = valid ? smem_addr(hist_b) : spare_a;  // (short loop) where this lane adds in this pass
@@ -338,25 +350,56 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
                         if (q < nq) v[q] = *reinterpret_cast<const float4 *>(stage + qoff[q]);
                         else v[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                     }
-                    consume_chunk<NQ, RULE, BATCH, DIRECT>(v, 4 * nq, valid, lane, ctx, hist_b, fmax_delta, P, prev, cnt0, fin0, empty_bar);
+                    consume_chunk<NQ, RULE, BATCH, DIRECT>(v, 4 * nq, valid, lane, ctx, hist_b, fmax_delta, P, prev, pass_cnt0, pass_fin0, empty_bar);
                 }
             }
-            if (valid) {
-                rowmax = fmaxf(rowmax, P);
-                if (LEAN) {  // (a lane without a row in this pass drops what it counted: the row's owner has it)
+            // (a lane without a row in this pass drops what it counted: the row's owner has it)
+            if (G > 1 && p.N >= 32) {
+                // The 32 consecutive rows of a warp belong to at most two trials: the lanes of each add up what they
+                // kept in registers (bin-0 counts; largest bin-0 finish time; largest total) and one lane hands it over
+                // (any copy of the trial's histograms will do, they are summed in the end).  Running sums are
+                // non-negative, so their bit patterns order like integers and 0 is "nothing".
+                const int s0 = __shfl_sync(0xffffffffu, seg, 0);
+                const bool in0 = valid && seg == s0, in1 = valid && seg != s0;
+                const unsigned others = __ballot_sync(0xffffffffu, in1);
+                auto hand_over = [&](bool in, int trial_seg, int lane_out) {
+                    const int cnt = __reduce_add_sync(0xffffffffu, in ? pass_cnt0 : 0);
+                    const int tot = __reduce_max_sync(0xffffffffu, in ? __float_as_int(P) : 0);
+                    const int fin = RULE == 1 ? __reduce_max_sync(0xffffffffu, in ? __float_as_int(pass_fin0) : 0) : 0;
+                    if (lane == lane_out) {
+                        int *h = copy0 + (b * G + trial_seg) * seg_ints;
+                        if (cnt > 0) {
+                            atomicAdd(h, cnt);
+                            if (RULE == 1) raise_max(reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(h) + fmax_delta), __int_as_float(fin));
+                        }
+                        if (tot > 0) atomicMax(&s.segmax[b * G + trial_seg], tot);
+                    }
+                };
+                hand_over(in0, s0, 0);
+                if (others != 0u) {
+                    const int src = __ffs(others) - 1;
+                    hand_over(in1, __shfl_sync(0xffffffffu, seg, src), src);
+                }
+            } else if (valid) {
+                if (G > 1) {
+                    if (pass_cnt0 > 0) {
+                        atomicAdd(myhist, pass_cnt0);
+                        if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), pass_fin0);
+                    }
+                    // largest row total of the trial: running sums are non-negative, so their bit patterns order like integers
+                    atomicMax(&s.segmax[b * G + seg], __float_as_int(P));
+                } else {
+                    rowmax = fmaxf(rowmax, P);
                     cnt0 += pass_cnt0;
                     fin0 = fmaxf(fin0, pass_fin0);
                 }
             }
         }
-        if (cnt0 > 0) {
-            atomicAdd(myhist, cnt0);
-            if (RULE == 1) raise_max(reinterpret_cast<float *>(hist_b + fmax_delta), fin0);
-        }
-        // largest row total of the trial: running sums are non-negative, so their bit patterns order like integers
-        if (G > 1) {
-            if (in_tile) atomicMax(&s.segmax[b * G + seg], __float_as_int(rowmax));
-        } else {
+        if (G == 1) {
+            if (cnt0 > 0) {
+                atomicAdd(myhist, cnt0);
+                if (RULE == 1) raise_max(reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(myhist) + fmax_delta), fin0);
+            }
             const unsigned wm = __reduce_max_sync(0xffffffffu, (unsigned)__float_as_int(rowmax));
             if (lane == 0) atomicMax(&s.segmax[b], (int)wm);
         }
@@ -370,6 +413,15 @@ __device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTai
             buffer_barrier_arrive<kBarReady>(b, bar_threads);  // hand buffer b to the epilogue warp
         }
     }
+}
+
+template <int NQ, int RULE, bool BATCH, bool DIRECT, bool LEAN, bool ONE = true>
+__device__ __forceinline__ void tiled_trials(const SweepParams &p, const SmemTail &s, const BinCtx &ctx, unsigned char *stage0,
+                                             uint64_t *full, uint64_t *empty, int tid, int lane, int warp, int ncw,
+                                             unsigned fmax_delta, unsigned off_zero)
+{
+    if (p.g > 1) tiled_trials_g<NQ, RULE, BATCH, DIRECT, LEAN, ONE, true>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
+    else tiled_trials_g<NQ, RULE, BATCH, DIRECT, LEAN, ONE, false>(p, s, ctx, stage0, full, empty, tid, lane, warp, ncw, fmax_delta, off_zero);
 }
 
 // WIDE = tiles of two trials of 129-256 workers each (up to 512 rows, 16 consumer warps): fewer idle lanes in the last
@@ -403,7 +455,8 @@ dc_sweep_tiled(const __grid_constant__ CUtensorMap lat_map, const SweepParams p)
     int prod_pass = 0, prod_c = 0, prod_issued = 0;
     auto issue_tile = [&](int st) {
         mbar_arrive_expect_tx(&full[st], (uint32_t)(p.rows * p.pitch));
-        tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, prod_c * p.bw, prod_pass * p.box_y, (int)(prod_t * p.g), &full[st]);
+        tma_load_3d(stage0 + (size_t)st * p.stage_bytes, &lat_map, prod_c * p.bw, prod_pass * p.box_y + (int)(prod_t * p.tile_y),
+                    (int)(prod_t * p.tile_z), &full[st]);
         if (++prod_c == p.chunks) {
             prod_c = 0;
             if (++prod_pass == p.passes) {

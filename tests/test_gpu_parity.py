@@ -456,6 +456,30 @@ def test_results_do_not_depend_on_tuning_or_timing(api):
 
 
 @pytest.mark.parametrize("rule", [0, 1])
+@pytest.mark.parametrize("T,N,M,K,cap", [(23, 200, 32, 64, 8), (7, 200, 12, 64, 8), (41, 129, 16, 16, 8), (12, 255, 8, 128, 8),
+                                         (9, 150, 100, 64, 8), (10, 200, 20, 100, 8), (16, 170, 36, 256, 8), (5, 200, 64, 64, 2),
+                                         (3, 131, 4, 8, 5), (2000, 200, 16, 64, 8)])
+def test_packed_tiles_match_oracle(api, T, N, M, K, cap, rule):
+    """Trials of 129-255 workers may be taken several at a time as one run of consecutive rows cut into equal passes
+    (a trial then starts in the middle of a pass and a thread's rows in different passes belong to different trials).
+    Small inputs never get that layout by themselves, so it is asked for through the tile-trials setting; the results
+    must be the oracle's bits, on evenly spaced and on irregular grids, whole and ragged last tiles, both loops."""
+    lat = W.iid_latencies("shifted_exp", T, N, M, seed=900 + N + M, shift=0.01, mean=0.02).numpy()
+    mean = M * 0.03
+    grids = [grid_for(lat, K, seed=K + N), np.linspace(0.7 * mean, 1.3 * mean, K, dtype=np.float64).astype(np.float32)]
+    lat_d = torch.from_numpy(lat).cuda()
+    try:
+        api.dc_tune(api.TUNE_TILE_TRIALS, cap)
+        for taus in grids:
+            ref = oracle.sweep(lat, taus, 0.05, rule=rule)
+            res = run_gpu(api, lat_d, torch.from_numpy(taus).cuda(), 0.05, rule=rule)
+            compare_sweep(res, ref, f"packed T={T} N={N} M={M} K={K}")
+    finally:
+        api.dc_tune(api.TUNE_TILE_TRIALS, 0)
+    api.dc_device_status()
+
+
+@pytest.mark.parametrize("rule", [0, 1])
 def test_direct_and_table_binning_agree_with_oracle(api, rule):
     """Evenly spaced grids are binned arithmetically, every other grid through the lookup table; both must
     give the oracle's bits.  Grids: exact dyadic steps with samples ON the thresholds, float32 linspace grids
